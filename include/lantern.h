@@ -1,0 +1,143 @@
+/*
+ * lantern.h -- C ABI of the LANTERN relaxed speculative-verification library (CUDA, sm_100a).
+ *
+ * The library implements the verification side of "LANTERN" (arXiv 2410.03355): the one-time
+ * latent-neighbourhood table B_k of a VQ codebook and, per verification step, the relaxed
+ * acceptance test over the TVD-bounded neighbourhood A_{k,delta}, the relaxed residual
+ * resampling on rejection, and the walk of a chain or tree of drafts to the first rejection.
+ *
+ * Notation (the paper's): q = target distribution, p = drafter distribution, x~ = draft token,
+ * B_k(x~) = k nearest codes of x~ in the codebook, itself included (Section 4.2),
+ * A_{k,delta}(x~) = the distance-ordered prefix of B_k(x~) whose moved mass stays below
+ * delta (Section 4.3; Algorithm 2).
+ *
+ * Conventions common to all calls
+ *   - Every data pointer is a DEVICE pointer owned by the caller; the library neither
+ *     allocates, frees nor keeps it.  `workspace` is caller-owned device scratch of at least
+ *     the size the matching *_workspace_bytes() call returns; its contents are undefined
+ *     before and after a call, and two calls in flight at once need distinct workspaces.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the default stream).  Work is
+ *     enqueued on it and the call returns without waiting for it.
+ *   - Return value: LANTERN_OK, or a negative code found on the host before anything is
+ *     launched (outputs untouched).  Faults that live in the data (a token out of range, a
+ *     NaN logit ...) never trap: they set bits in out_status[b] and give that sequence the
+ *     fallback result accept_len = number of drafts accepted before the fault, next_token = -1.
+ */
+#ifndef LANTERN_H_
+#define LANTERN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t lantern_status;
+
+enum {
+  LANTERN_OK = 0,
+  LANTERN_E_NULL = -1,          /* a required pointer is NULL */
+  LANTERN_E_SHAPE = -2,         /* a size is out of the supported range (see each call) */
+  LANTERN_E_PARAM = -3,         /* a scalar parameter is invalid (T <= 0, delta < 0, NaN ...) */
+  LANTERN_E_WORKSPACE = -4,     /* workspace missing, too small or misaligned */
+  LANTERN_E_CUDA = -5,          /* a CUDA runtime call failed (no device, launch error) */
+  LANTERN_E_ALIGN = -6,         /* a pointer is not 16-byte aligned */
+  LANTERN_E_UNIMPLEMENTED = -7  /* valid request this build does not cover (T == 0) */
+};
+
+/* storage type of logits */
+enum { LANTERN_F32 = 0, LANTERN_BF16 = 1 };
+
+/* bits of out_status[b] */
+enum {
+  LANTERN_ST_BAD_TOKEN = 1,     /* a draft token outside [0, V) */
+  LANTERN_ST_BAD_PARENT = 2,    /* a parent index outside [-1, own index) */
+  LANTERN_ST_BAD_UNIFORM = 4,   /* a uniform outside [0, 1) */
+  LANTERN_ST_NONFINITE = 8,     /* NaN / +inf logit, or a row with no finite logit, on the walked path */
+  LANTERN_ST_DEGENERATE = 16,   /* a residual of zero total weight (rounding only) */
+  LANTERN_ST_BAD_TABLE = 32,    /* a neighbour entry outside [0, V) was met (it carries no mass) */
+  LANTERN_ST_INTERNAL = 64      /* an on-chip copy did not complete within its wait limit */
+};
+
+/* Human-readable name of a return code (static storage). */
+const char* lantern_status_string(lantern_status s);
+
+/* ------------------------------------------------------------------------------------------
+ * Neighbour table.  Algorithm 2, block "Precompute B_k for all tokens" (Appendix D.2), with
+ * the l2 latent distance of Section 5.1.
+ *
+ * For every code i: squared l2 distance to every code j, accumulated in fp32 in dimension
+ * order as acc = fma(a_d - b_d, a_d - b_d, acc); the k smallest (distance, index) pairs with
+ * i itself forced into slot 0; stored in increasing distance, ties by smaller index.
+ *
+ *   codebook   [V, D] row-major fp32, finite values
+ *   V, D, k    1 <= k <= V <= 32768, 1 <= D <= 4096, k <= 4097
+ *   idx        out [V, k] int32; idx[i,0] == i
+ *   dist       out [V, k] fp32 squared distances, dist[i,0] == 0; may be NULL
+ *   workspace  lantern_build_workspace_bytes(V, D, k) bytes (0 for D <= 32: may then be NULL)
+ * ---------------------------------------------------------------------------------------- */
+size_t lantern_build_workspace_bytes(int V, int D, int k);
+
+lantern_status lantern_build_neighbors(const float* codebook, int V, int D, int k, int32_t* idx, float* dist,
+                                       void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
+ * One verification step.  Algorithm 1, verification loop and the bonus-token line after it,
+ * with the acceptance rule and residual of Section 4.3 and A_{k,delta} built as in
+ * Algorithm 2's second block.
+ *
+ * Per sequence b the drafts form a tree of N nodes (a chain when tree_parents is NULL).
+ * Context row 0 is the root; row i+1 is the context that follows node i.  Node i is tested
+ * in the context of its parent with
+ *     q = softmax((l_u + s (l_c - l_u)) / T)   of that row's target logits (guidance scales of
+ *                                              Appendix B.2; l_c alone when has_uncond == 0)
+ *     p = softmax(draft row / T)
+ * and is accepted iff  r_i * p(x~) < sum_{x in A_{k,delta}(x~)} q(x).  Children of one context
+ * are tried in node order; a rejection replaces q by the normalised residual
+ * [q_{k,delta}(.|D = x~) - p]_+ and removes x~ from p before the next sibling.  The walk
+ * follows accepted nodes; where every child is rejected the next token is drawn from the
+ * last residual, and where the walk reaches a node without children it is drawn from that
+ * row's q, both by inverse CDF at uniforms[b, N].
+ *
+ *   target_logits  [C, B, N+1, V], C = 2 (conditional, unconditional) if has_uncond else 1
+ *   draft_logits   [B, N+1, V] (already guided); rows of contexts without children are not read;
+ *                  may be NULL when N == 0
+ *   dtype          LANTERN_F32 or LANTERN_BF16, for both logit tensors; bases 16-byte aligned
+ *   cfg_scale      s, read only if has_uncond
+ *   T              temperature > 0
+ *   draft_tokens   [B, N] int32 in [0, V)
+ *   tree_parents   [B, N] int32, -1 = child of the root, else an index < own index; NULL = chain
+ *   neighbor_idx   [V, k] int32 as written by lantern_build_neighbors (slot 0 = the token itself)
+ *   k, delta       1 <= k <= V; delta >= 0 (delta = 0 or k = 1 gives standard speculative sampling)
+ *   uniforms       [B, N+1] fp32 in [0, 1): entry i tests node i, entry N is the final draw
+ *   B, N, V        B >= 0; 0 <= N <= 1024; V a multiple of 8, 8 <= V <= 16384, and small enough
+ *                  that C+1 logit rows plus V floats fit in shared memory (fp32 logits with
+ *                  has_uncond: V <= 8192)
+ *   out_accept_len  [B] number of accepted nodes
+ *   out_next_token  [B] resampled or bonus token (-1 with a fault bit in out_status)
+ *   out_accept_path [B, N] node ids of the accepted path in order, -1 padded; may be NULL
+ *   out_status      [B] LANTERN_ST_* bits; may be NULL
+ *   out_node_qa, out_node_px  [B, N] fp32: sum_A q and p(x~) as used in each node's test;
+ *   out_node_m                [B, N] int32: |A_{k,delta}(x~)| - 1.  Every node whose parent
+ *                  context has a child is evaluated up to and including the first accepted
+ *                  sibling; other nodes get NaN / -1.  Each may be NULL.
+ *   workspace       lantern_verify_workspace_bytes(B, N) bytes, 256-byte aligned
+ * ---------------------------------------------------------------------------------------- */
+size_t lantern_verify_workspace_bytes(int B, int N);
+
+lantern_status lantern_verify(const void* target_logits, const void* draft_logits, int dtype, float cfg_scale,
+                              int has_uncond, float T, const int32_t* draft_tokens, const int32_t* tree_parents,
+                              const int32_t* neighbor_idx, int k, float delta, const float* uniforms, int B,
+                              int N, int V, int32_t* out_accept_len, int32_t* out_next_token,
+                              int32_t* out_accept_path, int32_t* out_status, float* out_node_qa,
+                              float* out_node_px, int32_t* out_node_m, void* workspace, size_t workspace_bytes,
+                              void* cuda_stream);
+
+/* Number of kernels (and memsets) one lantern_verify call enqueues; for launch accounting. */
+int lantern_verify_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LANTERN_H_ */

@@ -43,13 +43,16 @@ def _p(a: Optional[np.ndarray]):
     return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
 
 
-def build_neighbors(codebook: np.ndarray, k: int):
-    """B_k for every code (Algorithm 2, precompute block). Returns idx [V,k] int32, dist [V,k] fp32."""
+def build_neighbors(codebook: np.ndarray, k: int, rows: Optional[np.ndarray] = None):
+    """B_k for every code, or for the codes listed in `rows` (Algorithm 2, precompute block).
+    Returns idx [n, k] int32, dist [n, k] fp32 with n = V or len(rows)."""
     cb = np.ascontiguousarray(codebook, dtype=np.float32)
     V, D = cb.shape
-    idx = np.empty((V, k), dtype=np.int32)
-    dist = np.empty((V, k), dtype=np.float32)
-    rc = _load().oracle_build_neighbors(_p(cb), V, D, int(k), _p(idx), _p(dist))
+    rw = None if rows is None else np.ascontiguousarray(rows, dtype=np.int32)
+    n = V if rw is None else rw.shape[0]
+    idx = np.empty((n, k), dtype=np.int32)
+    dist = np.empty((n, k), dtype=np.float32)
+    rc = _load().oracle_build_neighbors_rows(_p(cb), V, D, int(k), _p(rw), n, _p(idx), _p(dist))
     if rc != 0:
         raise ValueError(f"oracle_build_neighbors: bad arguments ({rc})")
     return idx, dist

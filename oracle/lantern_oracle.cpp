@@ -131,13 +131,19 @@ extern "C" {
 // Algorithm 2, first block: for every code, its k nearest codes (itself included), stored
 // in increasing distance.  R1 fixes the key.  Returns 0, or -1 on bad arguments.
 // ---------------------------------------------------------------------------------------
-int oracle_build_neighbors(const float* codebook, int V, int D, int k, int32_t* idx, float* dist) {
+// `rows` (nrows entries) selects which codes to compute; row r of idx / dist then belongs to
+// code rows[r].  rows == nullptr computes all V codes in order.
+int oracle_build_neighbors_rows(const float* codebook, int V, int D, int k, const int32_t* rows, int nrows,
+                                int32_t* idx, float* dist) {
   if (!codebook || !idx || V < 1 || D < 1 || k < 1 || k > V) return -1;
+  if (!rows) nrows = V;
   for (size_t e = 0; e < static_cast<size_t>(V) * D; ++e)
     if (!std::isfinite(codebook[e])) return -2;  // distances would not be ordered
   std::vector<float> key(V);
   std::vector<int32_t> order(V);
-  for (int i = 0; i < V; ++i) {
+  for (int r = 0; r < nrows; ++r) {
+    const int i = rows ? rows[r] : r;
+    if (i < 0 || i >= V) return -1;
     const float* a = codebook + static_cast<size_t>(i) * D;
     for (int j = 0; j < V; ++j) {
       const float* b = codebook + static_cast<size_t>(j) * D;
@@ -155,15 +161,19 @@ int oracle_build_neighbors(const float* codebook, int V, int D, int k, int32_t* 
       if (key[x] != key[y]) return key[x] < key[y];
       return x < y;
     });
-    int32_t* row = idx + static_cast<size_t>(i) * k;
+    int32_t* row = idx + static_cast<size_t>(r) * k;
     row[0] = i;
     for (int j = 1; j < k; ++j) row[j] = order[j - 1];
     if (dist) {
-      float* drow = dist + static_cast<size_t>(i) * k;
+      float* drow = dist + static_cast<size_t>(r) * k;
       for (int j = 0; j < k; ++j) drow[j] = key[row[j]];
     }
   }
   return 0;
+}
+
+int oracle_build_neighbors(const float* codebook, int V, int D, int k, int32_t* idx, float* dist) {
+  return oracle_build_neighbors_rows(codebook, V, D, k, nullptr, V, idx, dist);
 }
 
 // Number of rows whose neighbour order under double-precision distances differs from the
@@ -357,6 +367,7 @@ int oracle_verify(const void* target_logits, const void* draft_logits, int dtype
       }
 
       int accepted = -1;
+      bool degenerate = false;
       for (int c : kids[cur]) {
         const int32_t xt = draft_tokens[static_cast<size_t>(b) * N + c];
         const double r = uniforms[static_cast<size_t>(b) * R + c];
@@ -395,11 +406,14 @@ int oracle_verify(const void* target_logits, const void* draft_logits, int dtype
           W += w[x];
         }
         if (tr_w) tr_w[b] = W;
-        if (W > 0.0) {
-          for (int x = 0; x < V; ++x) q[x] = w[x] / W;
-        } else {
-          status |= ST_DEGENERATE;  // cannot occur in exact arithmetic; keep the current target
+        if (!(W > 0.0)) {
+          // Cannot occur in exact arithmetic (a rejection leaves at least p(x~) - sum_A q of
+          // residual mass); if rounding produces it, the step ends here with no token.
+          status |= ST_DEGENERATE;
+          degenerate = true;
+          break;
         }
+        for (int x = 0; x < V; ++x) q[x] = w[x] / W;
         // R6: the rejected token leaves the drafter distribution
         p[xt] = 0.0;
         double S = 0.0;
@@ -410,6 +424,7 @@ int oracle_verify(const void* target_logits, const void* draft_logits, int dtype
           std::fill(p.begin(), p.end(), 0.0);
         }
       }
+      if (degenerate) break;  // next_token stays -1
       if (accepted >= 0) {
         if (path) path[accept_len] = accepted;
         ++accept_len;

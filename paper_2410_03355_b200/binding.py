@@ -1,0 +1,169 @@
+"""ctypes binding of liblantern.so: argument marshalling only.
+
+Functions mirror the C entry points of include/lantern.h.  Tensors must live on a CUDA device;
+there is no CPU path: a missing library or a CPU tensor raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import dataclasses
+import os
+from typing import Optional
+
+import torch
+
+F32, BF16 = 0, 1
+ST_BAD_TOKEN, ST_BAD_PARENT, ST_BAD_UNIFORM, ST_NONFINITE, ST_DEGENERATE, ST_BAD_TABLE, ST_INTERNAL = \
+    1, 2, 4, 8, 16, 32, 64
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "liblantern.so")
+_lib = None
+
+
+class LanternError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (code {code})")
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library():
+    """Load liblantern.so (built in-tree by paper_2410_03355_b200.build). Fails loudly if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise FileNotFoundError(
+            f"{_LIB_PATH} not found: build it with `python -m paper_2410_03355_b200.build` "
+            "(there is no fallback implementation)")
+    lib = ctypes.CDLL(_LIB_PATH)
+    vp, i32, f32, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    lib.lantern_status_string.restype = ctypes.c_char_p
+    lib.lantern_status_string.argtypes = [i32]
+    lib.lantern_build_workspace_bytes.restype = sz
+    lib.lantern_build_workspace_bytes.argtypes = [i32, i32, i32]
+    lib.lantern_build_neighbors.restype = i32
+    lib.lantern_build_neighbors.argtypes = [vp, i32, i32, i32, vp, vp, vp, sz, vp]
+    lib.lantern_verify_workspace_bytes.restype = sz
+    lib.lantern_verify_workspace_bytes.argtypes = [i32, i32]
+    lib.lantern_verify_launch_count.restype = i32
+    lib.lantern_verify_launch_count.argtypes = []
+    lib.lantern_verify.restype = i32
+    lib.lantern_verify.argtypes = [vp, vp, i32, f32, i32, f32, vp, vp, vp, i32, f32, vp, i32, i32, i32,
+                                   vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    _lib = lib
+    return lib
+
+
+def status_string(code: int) -> str:
+    return load_library().lantern_status_string(int(code)).decode()
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None, name: str = "tensor"):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor (the library has no CPU path)")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"{name} must have dtype {dtype}, got {t.dtype}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def build_workspace_bytes(V: int, D: int, k: int) -> int:
+    return int(load_library().lantern_build_workspace_bytes(V, D, k))
+
+
+def build_neighbors(codebook: torch.Tensor, k: int, *, with_dist: bool = True,
+                    workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """lantern_build_neighbors: [V, D] fp32 codebook -> (idx [V, k] int32, dist [V, k] fp32 or None)."""
+    lib = load_library()
+    V, D = codebook.shape
+    with torch.cuda.device(codebook.device):
+        idx = torch.empty((V, k), dtype=torch.int32, device=codebook.device)
+        dist = torch.empty((V, k), dtype=torch.float32, device=codebook.device) if with_dist else None
+        need = build_workspace_bytes(V, D, k)
+        if workspace is None and need:
+            workspace = torch.empty(need, dtype=torch.uint8, device=codebook.device)
+        rc = lib.lantern_build_neighbors(_ptr(codebook, torch.float32, "codebook"), V, D, int(k), _ptr(idx),
+                                         _ptr(dist), _ptr(workspace), workspace.numel() if workspace is not None else 0,
+                                         _stream_ptr(stream))
+    if rc != 0:
+        raise LanternError(rc, "lantern_build_neighbors")
+    return idx, dist
+
+
+def verify_workspace_bytes(B: int, N: int) -> int:
+    return int(load_library().lantern_verify_workspace_bytes(B, N))
+
+
+@dataclasses.dataclass
+class VerifyOutputs:
+    accept_len: torch.Tensor            # [B] int32
+    next_token: torch.Tensor            # [B] int32
+    accept_path: Optional[torch.Tensor]  # [B, N] int32
+    status: Optional[torch.Tensor]      # [B] int32
+    node_qa: Optional[torch.Tensor]     # [B, N] fp32
+    node_px: Optional[torch.Tensor]     # [B, N] fp32
+    node_m: Optional[torch.Tensor]      # [B, N] int32
+
+
+def verify(target_logits: torch.Tensor, draft_logits: Optional[torch.Tensor], cfg_scale: float, T: float,
+           draft_tokens: Optional[torch.Tensor], tree_parents: Optional[torch.Tensor], neighbor_idx: torch.Tensor,
+           delta: float, uniforms: torch.Tensor, *, out: Optional[VerifyOutputs] = None, trace: bool = False,
+           workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None) -> VerifyOutputs:
+    """lantern_verify on torch tensors.
+
+    target_logits [C, B, N+1, V] (C = 2: conditional, unconditional; C = 1: no guidance), fp32 or bf16;
+    draft_logits [B, N+1, V]; draft_tokens / tree_parents [B, N] int32 (tree_parents None = chain);
+    neighbor_idx [V, k] int32; uniforms [B, N+1] fp32.  Outputs are allocated unless `out` is given.
+    """
+    lib = load_library()
+    C, B, R, V = target_logits.shape
+    N = R - 1
+    if C not in (1, 2):
+        raise ValueError("target_logits must have 1 or 2 guidance branches")
+    if target_logits.dtype == torch.bfloat16:
+        dtype = BF16
+    elif target_logits.dtype == torch.float32:
+        dtype = F32
+    else:
+        raise ValueError("logits must be float32 or bfloat16")
+    dev = target_logits.device
+    k = neighbor_idx.shape[1]
+    if neighbor_idx.shape[0] != V:
+        raise ValueError("neighbor_idx must have V rows")
+    with torch.cuda.device(dev):
+        if out is None:
+            i32 = dict(dtype=torch.int32, device=dev)
+            out = VerifyOutputs(
+                accept_len=torch.empty(B, **i32), next_token=torch.empty(B, **i32),
+                accept_path=torch.empty((B, N), **i32), status=torch.empty(B, **i32),
+                node_qa=torch.empty((B, N), dtype=torch.float32, device=dev) if trace else None,
+                node_px=torch.empty((B, N), dtype=torch.float32, device=dev) if trace else None,
+                node_m=torch.empty((B, N), **i32) if trace else None)
+        need = verify_workspace_bytes(B, N)
+        if workspace is None:
+            workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+        rc = lib.lantern_verify(
+            _ptr(target_logits, None, "target_logits"), _ptr(draft_logits, target_logits.dtype, "draft_logits"),
+            dtype, float(cfg_scale), int(C == 2), float(T), _ptr(draft_tokens, torch.int32, "draft_tokens"),
+            _ptr(tree_parents, torch.int32, "tree_parents"), _ptr(neighbor_idx, torch.int32, "neighbor_idx"),
+            int(k), float(delta), _ptr(uniforms, torch.float32, "uniforms"), B, N, V,
+            _ptr(out.accept_len, torch.int32), _ptr(out.next_token, torch.int32),
+            _ptr(out.accept_path, torch.int32), _ptr(out.status, torch.int32), _ptr(out.node_qa, torch.float32),
+            _ptr(out.node_px, torch.float32), _ptr(out.node_m, torch.int32), _ptr(workspace),
+            workspace.numel(), _stream_ptr(stream))
+    if rc != 0:
+        raise LanternError(rc, "lantern_verify")
+    return out

@@ -1,0 +1,98 @@
+// Device-side helpers shared by the LANTERN kernels: accurate exponential, warp/block
+// reductions and scans, mbarrier + bulk-copy (TMA) wrappers for sm_100a.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace lantern {
+
+constexpr int kWarp = 32;
+constexpr unsigned kFull = 0xffffffffu;
+
+// ---------------------------------------------------------------------------------------
+// exp(t) for t <= 0 (softmax numerators) with about 2.5e-7 relative error.
+// 2^(t*log2e) is evaluated by the hardware ex2 unit on x = fl(t*L_hi); the rounding error
+// of that product and the low part of log2(e) are folded back in to first order:
+// 2^(x+e) = 2^x * (1 + e ln2 + ...).  NaN propagates; t = -inf gives 0.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ float exp_nonpos(float t) {
+  const float L_hi = 1.44269502162933349609375f;     // fl32(log2 e)
+  const float L_lo = 1.925963033500011e-08f;         // log2 e - L_hi
+  const float LN2 = 0.693147182464599609375f;
+  t = (t < -104.0f) ? -104.0f : t;                   // keeps NaN, maps -inf to a flushed-to-zero result
+  float x = t * L_hi;
+  float e = __fmaf_rn(t, L_hi, -x);
+  e = __fmaf_rn(t, L_lo, e);
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return __fmaf_rn(y, e * LN2, y);
+}
+
+// ---------------------------------------------------------------------------------------
+// warp primitives
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(kFull, v, o));
+  return v;
+}
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+  return v;
+}
+__device__ __forceinline__ double warp_incl_scan(double v, int lane) {
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    double t = __shfl_up_sync(kFull, v, o);
+    if (lane >= o) v += t;
+  }
+  return v;
+}
+
+// ---------------------------------------------------------------------------------------
+// shared-memory barrier (mbarrier) and bulk asynchronous copy global -> shared
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_addr(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_mbar_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
+               : "memory");
+}
+// One bulk copy of `bytes` (multiple of 16, both addresses 16-byte aligned) that reports its
+// completion to `bar`.  No multicast: the destination is this CTA's own shared memory.
+__device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_addr(dst_smem)),
+               "l"(src_gmem), "r"(bytes), "r"(smem_addr(bar))
+               : "memory");
+}
+// Bounded wait for phase `parity` of `bar`.  Returns false if the limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t max_tries = (1u << 22)) {
+  const uint32_t a = smem_addr(bar);
+  for (uint32_t i = 0; i < max_tries; ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(a), "r"(parity)
+        : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+
+}  // namespace lantern

@@ -1,0 +1,956 @@
+// LANTERN relaxed verification step on sm_100a: plan -> fused context pass -> walk -> bonus.
+//
+// One "context" is a row of logits that has at least one drafted child.  The fused pass is
+// a persistent kernel, one CTA per SM: a bulk asynchronous copy (TMA, completion on an
+// mbarrier) brings the context's two target rows and its drafter row into shared memory
+// while the CTA is still working on the previous context; the rows are then read ONCE into
+// registers, guidance-combined, turned into softmax numerators, and every child of the
+// context is tested on chip:
+//     A_{k,delta}(x~)  : gather of the target numerators at the token's neighbour row and a
+//                        block-wide prefix scan with the strict bound (Algorithm 2, 2nd block)
+//     accept test      : r * p(x~) < sum_A q                     (Section 4.3, final rule)
+//     on rejection     : residual [q_{k,delta}(.|D=x~) - p]_+ over all V tokens, its total,
+//                        and either the next sibling's test on the renormalised residual or
+//                        the inverse-CDF draw of the replacement token   (Section 4.3, Alg. 1)
+// Each context leaves a 16-byte record; a tiny walk kernel follows the records from the root
+// (Algorithm 1's loop), and a last kernel draws the bonus token where the walk ended on a
+// context without children (Algorithm 1, line after the loop).
+//
+// Precision: processed logits are fp32 (difference, fused multiply-add, division, each
+// rounded once); exponentials are fp32 with ~2.5e-7 relative error; every sum over more
+// than eight terms and every threshold comparison is done in double precision.
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+
+#include "lantern.h"
+#include "lantern_device.cuh"
+
+namespace lantern {
+
+constexpr int NT = 1024;        // threads per CTA of the context / bonus kernels
+constexpr int NW = NT / 32;
+constexpr int LOG_NT = 10;
+constexpr int MAX_N = 1024;
+
+struct Counters {               // first 256 bytes of the workspace, zeroed per call
+  int work_next;                // next work item to hand out
+  int n_heavy;                  // contexts with >= 2 children (handed out first)
+  int n_light;                  // contexts with exactly 1 child
+  int n_bonus;                  // sequences whose walk ended on a childless context
+};
+
+struct Record {                 // result of one context
+  int accepted;                 // accepted child node, or -1 if every child was rejected
+  int token;                    // replacement token if every child was rejected
+  int status;                   // LANTERN_ST_* bits found in this context
+  int pad;
+};
+
+struct VerifyParams {
+  const void* target;
+  const void* draft;
+  const int32_t* tokens;
+  const int32_t* parents;
+  const int32_t* nbr;
+  const float* uniforms;
+  int32_t* out_len;
+  int32_t* out_tok;
+  int32_t* out_path;
+  int32_t* out_status;
+  float* out_qa;
+  float* out_px;
+  int32_t* out_m;
+  // workspace pieces
+  Counters* counters;
+  int32_t* work_heavy;
+  int32_t* work_light;
+  int32_t* child_start;         // [B, R+1]
+  int32_t* child_nodes;         // [B, N]
+  Record* records;              // [B, R]
+  int32_t* seq_status;          // [B]
+  int32_t* bonus_seq;           // [B]
+  int32_t* bonus_ctx;           // [B]
+  int B, N, R, V, k;
+  float cfg_scale, T, delta;
+};
+
+// ---------------------------------------------------------------------------------------
+// layout of a row held by a CTA: thread t owns, for chunk c, the eight consecutive tokens
+// [(c*NT + t)*8, +8).  In shared memory the numerators E are stored so that both 16-byte
+// halves of a thread's chunk are bank-conflict free: physical float index of token x below.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ int phys(int x) {
+  const int g = x >> 3;
+  const int c = g >> LOG_NT;
+  const int t = g & (NT - 1);
+  const int h = (x >> 2) & 1;
+  return ((((c << 1) | h) << LOG_NT) + t) << 2 | (x & 3);
+}
+
+struct BlockScratch {
+  double wt[2 * NW];            // per-(chunk, warp) totals
+  double wbase[2 * NW];         // their exclusive prefix
+  double sp[NW];
+  double total;
+  double total2;
+  double sm;
+  float fm[2 * NW];
+  float px;
+  int first;
+  int win;
+  int tok;
+  int item;
+  int bad;
+};
+
+// max of two values over the block
+__device__ __forceinline__ void block_max2(float& a, float& b, BlockScratch& S, int lane, int warp) {
+  a = warp_max(a);
+  b = warp_max(b);
+  if (lane == 0) {
+    S.fm[warp] = a;
+    S.fm[NW + warp] = b;
+  }
+  __syncthreads();
+  a = warp_max(S.fm[lane]);
+  b = warp_max(S.fm[NW + lane]);
+  __syncthreads();
+}
+
+// sum of two doubles over the block
+__device__ __forceinline__ void block_sum2(double& a, double& b, BlockScratch& S, int lane, int warp) {
+  a = warp_sum(a);
+  b = warp_sum(b);
+  if (lane == 0) {
+    S.wt[warp] = a;
+    S.wt[NW + warp] = b;
+  }
+  __syncthreads();
+  a = warp_sum(S.wt[lane]);
+  b = warp_sum(S.wt[NW + lane]);
+  __syncthreads();
+}
+
+__device__ __forceinline__ float sum8(const float* v) {
+  return ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
+}
+
+// Exclusive prefix (over the order chunk-major, then thread) of per-chunk sums cs[c], the
+// grand total in S.total, and the block sum of `extra` in S.total2.
+template <int CH>
+__device__ __forceinline__ void block_scan_chunks(const double (&cs)[CH], double (&excl)[CH], double extra,
+                                                  BlockScratch& S, int lane, int warp) {
+  double incl[CH];
+#pragma unroll
+  for (int c = 0; c < CH; ++c) {
+    incl[c] = warp_incl_scan(cs[c], lane);
+    if (lane == 31) S.wt[c * NW + warp] = incl[c];
+  }
+  extra = warp_sum(extra);
+  if (lane == 0) S.sp[warp] = extra;
+  __syncthreads();
+  if (warp == 0) {
+    double carry = 0.0;
+#pragma unroll
+    for (int c = 0; c < CH; ++c) {
+      const double t = S.wt[c * NW + lane];
+      const double in = warp_incl_scan(t, lane);
+      S.wbase[c * NW + lane] = carry + in - t;
+      carry += __shfl_sync(kFull, in, 31);
+    }
+    const double e = warp_sum(S.sp[lane]);
+    if (lane == 0) {
+      S.total = carry;
+      S.total2 = e;
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int c = 0; c < CH; ++c) excl[c] = S.wbase[c * NW + warp] + incl[c] - cs[c];
+}
+
+// Inverse CDF over the weights w (registers, layout above): smallest token whose inclusive
+// cumulative weight exceeds target; if rounding leaves none, the largest token of positive
+// weight; -1 if there is no positive weight.  Must be called by the whole block.
+template <int CH>
+__device__ __forceinline__ int block_draw(const float (&w)[CH * 8], const double (&cs)[CH], const double (&excl)[CH],
+                                          double target, int V, BlockScratch& S, int tid) {
+  if (tid == 0) {
+    S.win = 0x7fffffff;
+    S.tok = -1;
+  }
+  __syncthreads();
+  int cand = 0x7fffffff;
+#pragma unroll
+  for (int c = CH - 1; c >= 0; --c)
+    if (excl[c] + cs[c] > target) cand = c * NT + tid;
+  const int wmin = __reduce_min_sync(kFull, cand);
+  if ((tid & 31) == 0 && wmin != 0x7fffffff) atomicMin(&S.win, wmin);
+  __syncthreads();
+  const int win = S.win;
+  if (win == 0x7fffffff) {
+    int last = -1;
+#pragma unroll
+    for (int c = 0; c < CH; ++c)
+#pragma unroll
+      for (int e = 0; e < 8; ++e)
+        if (w[c * 8 + e] > 0.0f) last = (c * NT + tid) * 8 + e;
+    if (last >= V) last = -1;
+    if (last >= 0) atomicMax(&S.tok, last);
+  } else if ((win & (NT - 1)) == tid) {
+    const int wc = win >> LOG_NT;
+    int tok = -1, lastpos = -1;
+#pragma unroll
+    for (int c = 0; c < CH; ++c) {
+      if (c == wc) {
+        double cum = excl[c];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const float wv = w[c * 8 + e];
+          cum += static_cast<double>(wv);
+          if (wv > 0.0f) lastpos = e;
+          if (tok < 0 && cum > target) tok = e;
+        }
+      }
+    }
+    if (tok < 0) tok = lastpos;
+    S.tok = win * 8 + tok;
+  }
+  __syncthreads();
+  return S.tok;
+}
+
+// Read one context's rows from shared-memory staging into registers as processed logits.
+template <int CH, bool BF16, bool UNC, bool WITH_DRAFT>
+__device__ __forceinline__ void load_rows(const unsigned char* stage, int rowbytes, int V, float s, float T,
+                                          float (&zq)[CH * 8], float (&zp)[CH * 8], int tid) {
+  const unsigned char* rc = stage;
+  const unsigned char* ru = stage + rowbytes;
+  const unsigned char* rd = stage + (UNC ? 2 : 1) * rowbytes;
+  const float ninf = __int_as_float(0xff800000);
+#pragma unroll
+  for (int c = 0; c < CH; ++c) {
+    const int g = c * NT + tid;
+    if (g * 8 < V) {
+      float lc[8], lu[8], ld[8];
+      if (BF16) {
+        const uint4 a = *reinterpret_cast<const uint4*>(rc + g * 16);
+        const uint32_t aw[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          lc[2 * i] = __uint_as_float(aw[i] << 16);
+          lc[2 * i + 1] = __uint_as_float(aw[i] & 0xffff0000u);
+        }
+        if (UNC) {
+          const uint4 b = *reinterpret_cast<const uint4*>(ru + g * 16);
+          const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            lu[2 * i] = __uint_as_float(bw[i] << 16);
+            lu[2 * i + 1] = __uint_as_float(bw[i] & 0xffff0000u);
+          }
+        }
+        if (WITH_DRAFT) {
+          const uint4 d = *reinterpret_cast<const uint4*>(rd + g * 16);
+          const uint32_t dw[4] = {d.x, d.y, d.z, d.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            ld[2 * i] = __uint_as_float(dw[i] << 16);
+            ld[2 * i + 1] = __uint_as_float(dw[i] & 0xffff0000u);
+          }
+        }
+      } else {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const float4 a = *reinterpret_cast<const float4*>(rc + g * 32 + h * 16);
+          lc[4 * h] = a.x, lc[4 * h + 1] = a.y, lc[4 * h + 2] = a.z, lc[4 * h + 3] = a.w;
+          if (UNC) {
+            const float4 b = *reinterpret_cast<const float4*>(ru + g * 32 + h * 16);
+            lu[4 * h] = b.x, lu[4 * h + 1] = b.y, lu[4 * h + 2] = b.z, lu[4 * h + 3] = b.w;
+          }
+          if (WITH_DRAFT) {
+            const float4 d = *reinterpret_cast<const float4*>(rd + g * 32 + h * 16);
+            ld[4 * h] = d.x, ld[4 * h + 1] = d.y, ld[4 * h + 2] = d.z, ld[4 * h + 3] = d.w;
+          }
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        float l = lc[e];
+        if (UNC) l = __fmaf_rn(s, __fsub_rn(lc[e], lu[e]), lu[e]);   // l_u + s (l_c - l_u)
+        float d = WITH_DRAFT ? ld[e] : 0.0f;
+        if (T != 1.0f) {
+          l = __fdiv_rn(l, T);
+          d = __fdiv_rn(d, T);
+        }
+        zq[c * 8 + e] = l;
+        zp[c * 8 + e] = d;
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        zq[c * 8 + e] = ninf;
+        zp[c * 8 + e] = ninf;
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// kernel 1: plan.  One warp per sequence: validate tokens / parents / uniforms, bucket the
+// nodes by parent context (children in node order), initialise the per-node outputs and
+// append the contexts that have children to the work lists.
+// ---------------------------------------------------------------------------------------
+constexpr int PLAN_WARPS = 4;
+
+__global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyParams P) {
+  extern __shared__ int plan_smem[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int b = blockIdx.x * PLAN_WARPS + warp;
+  if (b >= P.B) return;
+  const int N = P.N, R = P.R;
+  int* cnt = plan_smem + warp * (R + 1);       // cnt[c], c in [0, R]; later the fill cursor
+  for (int i = lane; i <= R; i += 32) cnt[i] = 0;
+  __syncwarp();
+  int status = 0;
+  const float qnan = __int_as_float(0x7fc00000);
+  for (int i = lane; i < N; i += 32) {
+    const size_t o = static_cast<size_t>(b) * N + i;
+    const int tok = P.tokens[o];
+    if (static_cast<unsigned>(tok) >= static_cast<unsigned>(P.V)) status |= LANTERN_ST_BAD_TOKEN;
+    const int par = P.parents ? P.parents[o] : i - 1;
+    if (par < -1 || par >= i) status |= LANTERN_ST_BAD_PARENT;
+    else atomicAdd(&cnt[par + 1], 1);
+    if (P.out_path) P.out_path[o] = -1;
+    if (P.out_qa) P.out_qa[o] = qnan;
+    if (P.out_px) P.out_px[o] = qnan;
+    if (P.out_m) P.out_m[o] = -1;
+  }
+  for (int i = lane; i <= N; i += 32) {
+    const float r = P.uniforms[static_cast<size_t>(b) * R + i];
+    if (!(r >= 0.0f && r < 1.0f)) status |= LANTERN_ST_BAD_UNIFORM;
+  }
+  status = __reduce_or_sync(kFull, status);
+  __syncwarp();
+  int32_t* cstart = P.child_start + static_cast<size_t>(b) * (R + 1);
+  if (lane == 0) P.seq_status[b] = status;
+  if (status) {
+    for (int i = lane; i <= R; i += 32) cstart[i] = 0;
+    return;
+  }
+  // work items (before the counts are turned into cursors)
+  for (int base = 0; base < R; base += 32) {
+    const int c = base + lane;
+    const int n = c < R ? cnt[c] : 0;
+    const unsigned heavy = __ballot_sync(kFull, n >= 2);
+    const unsigned light = __ballot_sync(kFull, n == 1);
+    int hb = 0, lb = 0;
+    if (lane == 0) {
+      if (heavy) hb = atomicAdd(&P.counters->n_heavy, __popc(heavy));
+      if (light) lb = atomicAdd(&P.counters->n_light, __popc(light));
+    }
+    hb = __shfl_sync(kFull, hb, 0);
+    lb = __shfl_sync(kFull, lb, 0);
+    const unsigned below = (1u << lane) - 1u;
+    if (n >= 2) P.work_heavy[hb + __popc(heavy & below)] = b * R + c;
+    if (n == 1) P.work_light[lb + __popc(light & below)] = b * R + c;
+  }
+  __syncwarp();
+  if (lane == 0) {
+    int run = 0;
+    for (int c = 0; c < R; ++c) {
+      const int n = cnt[c];
+      cstart[c] = run;
+      cnt[c] = run;
+      run += n;
+    }
+    cstart[R] = run;
+    int32_t* cn = P.child_nodes + static_cast<size_t>(b) * N;
+    for (int i = 0; i < N; ++i) {
+      const int par = P.parents ? P.parents[static_cast<size_t>(b) * N + i] : i - 1;
+      cn[cnt[par + 1]++] = i;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// kernel 2: fused context pass (see the header of this file).
+// ---------------------------------------------------------------------------------------
+template <bool BF16, bool UNC>
+__device__ __forceinline__ void issue_rows(const VerifyParams& P, int item, unsigned char* stage, int rowbytes,
+                                           uint64_t* bar) {
+  const int nrows = UNC ? 3 : 2;
+  mbar_expect_tx(bar, static_cast<uint32_t>(nrows * rowbytes));
+  const size_t row_off = static_cast<size_t>(item) * rowbytes;
+  const size_t branch = static_cast<size_t>(P.B) * P.R * rowbytes;
+  const unsigned char* src[3];
+  src[0] = static_cast<const unsigned char*>(P.target) + row_off;
+  src[1] = UNC ? static_cast<const unsigned char*>(P.target) + branch + row_off
+               : static_cast<const unsigned char*>(P.draft) + row_off;
+  src[2] = static_cast<const unsigned char*>(P.draft) + row_off;
+  for (int r = 0; r < nrows; ++r)
+    for (int off = 0; off < rowbytes; off += 16384) {
+      const int n = min(16384, rowbytes - off);
+      bulk_load(stage + r * rowbytes + off, src[r] + off, static_cast<uint32_t>(n), bar);
+    }
+}
+
+template <int CH, bool BF16, bool UNC>
+__global__ void __launch_bounds__(NT, 1) lantern_context_kernel(VerifyParams P) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  __shared__ BlockScratch S;
+  __shared__ __align__(8) uint64_t bar;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int V = P.V, N = P.N, R = P.R, k = P.k;
+  const int rowbytes = V * (BF16 ? 2 : 4);
+  unsigned char* stage = smem;
+  float* E = reinterpret_cast<float*>(smem + (UNC ? 3 : 2) * rowbytes);
+
+  const int n_heavy = P.counters->n_heavy;
+  const int total = n_heavy + P.counters->n_light;
+
+  auto item_of = [&](int w) { return w < n_heavy ? P.work_heavy[w] : P.work_light[w - n_heavy]; };
+
+  if (tid == 0) {
+    mbar_init(&bar, 1);
+    fence_mbar_init();
+    fence_proxy_async();
+    const int w = atomicAdd(&P.counters->work_next, 1);
+    int item = -1;
+    if (w < total) {
+      item = item_of(w);
+      issue_rows<BF16, UNC>(P, item, stage, rowbytes, &bar);
+    }
+    S.item = item;
+  }
+  __syncthreads();
+  uint32_t parity = 0;
+
+  for (;;) {
+    const int item = S.item;
+    if (item < 0) break;
+    const int b = item / R, c = item - b * R;
+    const int32_t* cstart = P.child_start + static_cast<size_t>(b) * (R + 1);
+    const int cs_ = cstart[c], ce_ = cstart[c + 1];
+    const int32_t* cnodes = P.child_nodes + static_cast<size_t>(b) * N;
+    const int32_t* toks = P.tokens + static_cast<size_t>(b) * N;
+
+    // first child's neighbour row: issued before the wait so its latency hides behind it
+    int node = cnodes[cs_];
+    int xt = toks[node];
+    int nreg = (tid + 1 < k) ? __ldg(P.nbr + static_cast<size_t>(xt) * k + tid + 1) : -1;
+
+    // every thread must take the same branch: agree on whether the rows have landed
+    const bool arrived = __syncthreads_and(mbar_wait(&bar, parity)) != 0;
+    if (!arrived) {
+      // The copy did not land within the limit: report it, give the copy in flight one more
+      // bounded chance to finish before this CTA's shared memory is released, and stop.
+      if (tid == 0) {
+        Record rec = {-1, -1, LANTERN_ST_INTERNAL, 0};
+        P.records[item] = rec;
+      }
+      mbar_wait(&bar, parity);
+      break;
+    }
+    parity ^= 1u;
+
+    float a[CH * 8], ep[CH * 8];
+    load_rows<CH, BF16, UNC, true>(stage, rowbytes, V, P.cfg_scale, P.T, a, ep, tid);
+    float mq = a[0], mp = ep[0];
+#pragma unroll
+    for (int i = 1; i < CH * 8; ++i) {
+      mq = fmaxf(mq, a[i]);
+      mp = fmaxf(mp, ep[i]);
+    }
+    block_max2(mq, mp, S, lane, warp);   // barrier inside: every thread has drained the staging rows
+
+    // staging is free: hand out the next context and start its copy
+    if (tid == 0) {
+      const int w = atomicAdd(&P.counters->work_next, 1);
+      int nxt = -1;
+      if (w < total) {
+        nxt = item_of(w);
+        fence_proxy_async();
+        issue_rows<BF16, UNC>(P, nxt, stage, rowbytes, &bar);
+      }
+      S.item = nxt;   // read at the top of the next iteration, after many barriers
+    }
+
+    // softmax numerators and their totals
+    double zq_sum, zp_sum;
+    {
+      float pq[CH], pp[CH];
+#pragma unroll
+      for (int cc = 0; cc < CH; ++cc) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          a[cc * 8 + e] = exp_nonpos(a[cc * 8 + e] - mq);
+          ep[cc * 8 + e] = exp_nonpos(ep[cc * 8 + e] - mp);
+        }
+        pq[cc] = sum8(&a[cc * 8]);
+        pp[cc] = sum8(&ep[cc * 8]);
+        const int g = cc * NT + tid;
+        if (g * 8 < V) {
+          float4* dst = reinterpret_cast<float4*>(E);
+          dst[(((cc << 1) | 0) << LOG_NT) + tid] = make_float4(a[cc * 8], a[cc * 8 + 1], a[cc * 8 + 2], a[cc * 8 + 3]);
+          dst[(((cc << 1) | 1) << LOG_NT) + tid] =
+              make_float4(a[cc * 8 + 4], a[cc * 8 + 5], a[cc * 8 + 6], a[cc * 8 + 7]);
+        }
+      }
+      zq_sum = pq[0];
+      zp_sum = pp[0];
+#pragma unroll
+      for (int cc = 1; cc < CH; ++cc) {
+        zq_sum += pq[cc];
+        zp_sum += pp[cc];
+      }
+    }
+    block_sum2(zq_sum, zp_sum, S, lane, warp);   // barriers inside also publish E
+
+    int status = 0;
+    int accepted = -1, token = -1;
+    if (!(zq_sum > 0.0 && zq_sum < 1e300 && zp_sum > 0.0 && zp_sum < 1e300)) {
+      status |= LANTERN_ST_NONFINITE;
+    } else {
+      double qscale = 1.0 / zq_sum;     // q'(x) = E(x) * qscale
+      double pscale = 1.0 / zp_sum;     // p'(x) = ep(x) * pscale
+      const double delta = static_cast<double>(P.delta);
+
+      for (int ci = cs_; ci < ce_; ++ci) {
+        const float r = P.uniforms[static_cast<size_t>(b) * R + node];
+        const int32_t* nrow = P.nbr + static_cast<size_t>(xt) * k;
+        const float e_xt = E[phys(xt)];   // read while E is stable (before any flagging below)
+        // owner of x~ publishes its drafter numerator
+        {
+          const int g = xt >> 3;
+          if ((g & (NT - 1)) == tid) {
+            const int li = ((g >> LOG_NT) << 3) | (xt & 7);
+            float v = 0.0f;
+#pragma unroll
+            for (int i = 0; i < CH * 8; ++i)
+              if (i == li) v = ep[i];
+            S.px = v;
+          }
+        }
+        // ---- A_{k,delta}(x~): gather + prefix scan with the strict bound ----
+        const double thr = delta * (1.0 / qscale);   // compare unnormalised sums
+        double carry = 0.0, sm = 0.0;
+        int m = k - 1;
+        bool cut = false;
+        for (int base = 0; base < k - 1 && !cut; base += NT) {
+          const int j = base + tid + 1;
+          const bool valid = j < k;
+          const int n = (base == 0) ? nreg : (valid ? __ldg(nrow + j) : -1);
+          float v = 0.0f;
+          if (valid) {
+            if (static_cast<unsigned>(n) < static_cast<unsigned>(V)) v = E[phys(n)];
+            else status |= LANTERN_ST_BAD_TABLE;
+          }
+          const double incl = warp_incl_scan(static_cast<double>(v), lane);
+          if (lane == 31) S.wt[warp] = incl;
+          if (tid == 0) S.first = 0x7fffffff;
+          __syncthreads();
+          if (warp == 0) {
+            const double t = S.wt[lane];
+            const double in = warp_incl_scan(t, lane);
+            S.wbase[lane] = in - t;
+            if (lane == 31) S.total = in;
+          }
+          __syncthreads();
+          const double Sj = carry + S.wbase[warp] + incl;
+          const bool fail = valid && !(Sj < thr);
+          const unsigned bal = __ballot_sync(kFull, fail);
+          if (bal && lane == __ffs(bal) - 1) atomicMin(&S.first, j);
+          __syncthreads();
+          const int first = S.first;
+          if (first != 0x7fffffff) {
+            m = first - 1;
+            if (j == m) S.sm = Sj;
+            __syncthreads();
+            sm = (m == base) ? carry : S.sm;
+            cut = true;
+          } else {
+            carry += S.total;
+            sm = carry;
+            __syncthreads();
+          }
+        }
+        if (k == 1) __syncthreads();   // publish S.px when the scan loop did not run
+        const double qa = (static_cast<double>(e_xt) + sm) * qscale;
+        const double px = static_cast<double>(S.px) * pscale;
+        const bool accept = static_cast<double>(r) * px < qa;   // Section 4.3: min(1, sum_A q / p(x~))
+        if (tid == 0) {
+          const size_t o = static_cast<size_t>(b) * N + node;
+          if (P.out_qa) P.out_qa[o] = static_cast<float>(qa);
+          if (P.out_px) P.out_px[o] = static_cast<float>(px);
+          if (P.out_m) P.out_m[o] = m;
+        }
+        if (accept) {
+          accepted = node;
+          break;
+        }
+        // ---- rejected: residual [q_{k,delta}(.|D = x~) - p]_+ ----
+        // members of A (x~ included) leave no residual mass: flag them with a negative sign
+        for (int j = tid + 1; j <= m; j += NT) {
+          const int n = (j <= NT) ? nreg : __ldg(nrow + j);
+          if (static_cast<unsigned>(n) < static_cast<unsigned>(V)) {
+            const int q_ = phys(n);
+            E[q_] = -fabsf(E[q_]);
+          }
+        }
+        if (tid == 0) E[phys(xt)] = -fabsf(E[phys(xt)]);
+        {   // x~ leaves the drafter distribution for the following siblings
+          const int g = xt >> 3;
+          if ((g & (NT - 1)) == tid) {
+            const int li = ((g >> LOG_NT) << 3) | (xt & 7);
+#pragma unroll
+            for (int i = 0; i < CH * 8; ++i)
+              if (i == li) ep[i] = 0.0f;
+          }
+        }
+        const bool last = (ci + 1 == ce_);
+        if (!last) {   // next sibling's neighbour row, in flight during the residual pass
+          node = cnodes[ci + 1];
+          xt = toks[node];
+          nreg = (tid + 1 < k) ? __ldg(P.nbr + static_cast<size_t>(xt) * k + tid + 1) : -1;
+        }
+        __syncthreads();
+        const float ratio = static_cast<float>(pscale / qscale);   // w = E - ratio * ep, in units of E
+        double cs[CH], excl[CH];
+        float psum = 0.0f;
+#pragma unroll
+        for (int cc = 0; cc < CH; ++cc) {
+          const int g = cc * NT + tid;
+          if (g * 8 < V) {
+            const float4* src = reinterpret_cast<const float4*>(E);
+            const float4 lo = src[(((cc << 1) | 0) << LOG_NT) + tid];
+            const float4 hi = src[(((cc << 1) | 1) << LOG_NT) + tid];
+            const float e8[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+#pragma unroll
+            for (int e = 0; e < 8; ++e) a[cc * 8 + e] = fmaxf(0.0f, __fmaf_rn(-ratio, ep[cc * 8 + e], e8[e]));
+          } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) a[cc * 8 + e] = 0.0f;
+          }
+          cs[cc] = static_cast<double>(sum8(&a[cc * 8]));
+          psum += sum8(&ep[cc * 8]);
+        }
+        block_scan_chunks<CH>(cs, excl, static_cast<double>(psum), S, lane, warp);
+        const double W = S.total, Sp = S.total2;
+        if (!(W > 0.0)) {
+          status |= LANTERN_ST_DEGENERATE;
+          break;
+        }
+        if (last) {
+          const double u = static_cast<double>(P.uniforms[static_cast<size_t>(b) * R + N]);
+          token = block_draw<CH>(a, cs, excl, u * W, V, S, tid);
+        } else {
+#pragma unroll
+          for (int cc = 0; cc < CH; ++cc) {
+            const int g = cc * NT + tid;
+            if (g * 8 < V) {
+              float4* dst = reinterpret_cast<float4*>(E);
+              dst[(((cc << 1) | 0) << LOG_NT) + tid] =
+                  make_float4(a[cc * 8], a[cc * 8 + 1], a[cc * 8 + 2], a[cc * 8 + 3]);
+              dst[(((cc << 1) | 1) << LOG_NT) + tid] =
+                  make_float4(a[cc * 8 + 4], a[cc * 8 + 5], a[cc * 8 + 6], a[cc * 8 + 7]);
+            }
+          }
+          qscale = 1.0 / W;
+          pscale = Sp > 0.0 ? 1.0 / Sp : 0.0;
+          __syncthreads();
+        }
+      }
+    }
+    status = __syncthreads_or(status);
+    if (tid == 0) {
+      Record rec = {accepted, token, status, 0};
+      P.records[item] = rec;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// kernel 3: walk (Algorithm 1's loop over the records; one thread per sequence)
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) lantern_walk_kernel(VerifyParams P) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= P.B) return;
+  const int N = P.N, R = P.R;
+  int status = P.seq_status[b];
+  int len = 0, next = -1;
+  if (status == 0) {
+    const int32_t* cstart = P.child_start + static_cast<size_t>(b) * (R + 1);
+    int cur = 0;
+    for (int step = 0; step <= N; ++step) {
+      if (cstart[cur + 1] == cstart[cur]) {   // no drafts left on this path: bonus token from q
+        const int slot = atomicAdd(&P.counters->n_bonus, 1);
+        P.bonus_seq[slot] = b;
+        P.bonus_ctx[slot] = cur;
+        break;
+      }
+      const Record rec = P.records[static_cast<size_t>(b) * R + cur];
+      status |= rec.status;
+      if (rec.status & (LANTERN_ST_NONFINITE | LANTERN_ST_DEGENERATE | LANTERN_ST_INTERNAL)) break;
+      if (rec.accepted >= 0) {
+        if (P.out_path) P.out_path[static_cast<size_t>(b) * N + len] = rec.accepted;
+        ++len;
+        cur = rec.accepted + 1;
+        continue;
+      }
+      next = rec.token;
+      break;
+    }
+  }
+  P.out_len[b] = len;
+  P.out_tok[b] = next;
+  if (P.out_status) P.out_status[b] = status;
+}
+
+// ---------------------------------------------------------------------------------------
+// kernel 4: bonus token ~ q at the context where the walk ran out of drafts
+// (Algorithm 1, line after the verification loop)
+// ---------------------------------------------------------------------------------------
+template <int CH, bool BF16, bool UNC>
+__global__ void __launch_bounds__(NT, 1) lantern_bonus_kernel(VerifyParams P) {
+  __shared__ BlockScratch S;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int V = P.V, R = P.R, N = P.N;
+  const int rowbytes = V * (BF16 ? 2 : 4);
+  const int count = P.counters->n_bonus;
+  for (int i = blockIdx.x; i < count; i += gridDim.x) {
+    const int b = P.bonus_seq[i], ctx = P.bonus_ctx[i];
+    const size_t row_off = (static_cast<size_t>(b) * R + ctx) * rowbytes;
+    const size_t branch = static_cast<size_t>(P.B) * R * rowbytes;
+    const unsigned char* rc = static_cast<const unsigned char*>(P.target) + row_off;
+    const unsigned char* ru = rc + branch;
+    float a[CH * 8];
+    const float ninf = __int_as_float(0xff800000);
+#pragma unroll
+    for (int c = 0; c < CH; ++c) {
+      const int g = c * NT + tid;
+      float lc[8], lu[8];
+      if (g * 8 < V) {
+        if (BF16) {
+          const uint4 x = __ldg(reinterpret_cast<const uint4*>(rc + g * 16));
+          const uint32_t xw[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            lc[2 * j] = __uint_as_float(xw[j] << 16);
+            lc[2 * j + 1] = __uint_as_float(xw[j] & 0xffff0000u);
+          }
+          if (UNC) {
+            const uint4 y = __ldg(reinterpret_cast<const uint4*>(ru + g * 16));
+            const uint32_t yw[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              lu[2 * j] = __uint_as_float(yw[j] << 16);
+              lu[2 * j + 1] = __uint_as_float(yw[j] & 0xffff0000u);
+            }
+          }
+        } else {
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const float4 x = __ldg(reinterpret_cast<const float4*>(rc + g * 32 + h * 16));
+            lc[4 * h] = x.x, lc[4 * h + 1] = x.y, lc[4 * h + 2] = x.z, lc[4 * h + 3] = x.w;
+            if (UNC) {
+              const float4 y = __ldg(reinterpret_cast<const float4*>(ru + g * 32 + h * 16));
+              lu[4 * h] = y.x, lu[4 * h + 1] = y.y, lu[4 * h + 2] = y.z, lu[4 * h + 3] = y.w;
+            }
+          }
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          float l = lc[e];
+          if (UNC) l = __fmaf_rn(P.cfg_scale, __fsub_rn(lc[e], lu[e]), lu[e]);
+          if (P.T != 1.0f) l = __fdiv_rn(l, P.T);
+          a[c * 8 + e] = l;
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) a[c * 8 + e] = ninf;
+      }
+    }
+    float mq = a[0], dummy = 0.0f;
+#pragma unroll
+    for (int j = 1; j < CH * 8; ++j) mq = fmaxf(mq, a[j]);
+    block_max2(mq, dummy, S, lane, warp);
+    double cs[CH], excl[CH];
+#pragma unroll
+    for (int c = 0; c < CH; ++c) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) a[c * 8 + e] = exp_nonpos(a[c * 8 + e] - mq);
+      cs[c] = static_cast<double>(sum8(&a[c * 8]));
+    }
+    block_scan_chunks<CH>(cs, excl, 0.0, S, lane, warp);
+    const double Z = S.total;
+    int tok = -1, st = 0;
+    if (Z > 0.0 && Z < 1e300) {
+      const double u = static_cast<double>(P.uniforms[static_cast<size_t>(b) * R + N]);
+      tok = block_draw<CH>(a, cs, excl, u * Z, V, S, tid);
+    } else {
+      st = LANTERN_ST_NONFINITE;
+    }
+    if (tid == 0) {
+      P.out_tok[b] = tok;
+      if (st && P.out_status) P.out_status[b] |= st;
+    }
+    __syncthreads();
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct WsLayout {
+  size_t counters, heavy, light, cstart, cnodes, records, seqst, bseq, bctx, total;
+};
+
+static WsLayout ws_layout(int B, int N) {
+  const size_t R = static_cast<size_t>(N) + 1, b = static_cast<size_t>(B);
+  WsLayout L;
+  size_t o = 0;
+  L.counters = o; o += 256;
+  L.heavy = o;    o += align_up(b * R * 4, 256);
+  L.light = o;    o += align_up(b * R * 4, 256);
+  L.cstart = o;   o += align_up(b * (R + 1) * 4, 256);
+  L.cnodes = o;   o += align_up(b * N * 4 + 4, 256);
+  L.records = o;  o += align_up(b * R * sizeof(Record), 256);
+  L.seqst = o;    o += align_up(b * 4, 256);
+  L.bseq = o;     o += align_up(b * 4, 256);
+  L.bctx = o;     o += align_up(b * 4, 256);
+  L.total = o;
+  return L;
+}
+
+template <int CH, bool BF16, bool UNC>
+static cudaError_t launch_verify(const VerifyParams& P, int grid_ctx, int grid_bonus, size_t smem_bytes,
+                                 cudaStream_t st) {
+  auto kc = lantern_context_kernel<CH, BF16, UNC>;
+  cudaError_t e = cudaFuncSetAttribute(kc, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+  if (e != cudaSuccess) return e;
+  kc<<<grid_ctx, NT, smem_bytes, st>>>(P);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  lantern_walk_kernel<<<(P.B + 127) / 128, 128, 0, st>>>(P);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  lantern_bonus_kernel<CH, BF16, UNC><<<grid_bonus, NT, 0, st>>>(P);
+  return cudaGetLastError();
+}
+
+}  // namespace lantern
+
+using namespace lantern;
+
+extern "C" size_t lantern_verify_workspace_bytes(int B, int N) {
+  if (B < 0 || N < 0 || N > MAX_N) return 0;
+  return ws_layout(B > 0 ? B : 1, N).total;
+}
+
+extern "C" int lantern_verify_launch_count(void) { return 5; }
+
+extern "C" lantern_status lantern_verify(const void* target_logits, const void* draft_logits, int dtype,
+                                         float cfg_scale, int has_uncond, float T, const int32_t* draft_tokens,
+                                         const int32_t* tree_parents, const int32_t* neighbor_idx, int k,
+                                         float delta, const float* uniforms, int B, int N, int V,
+                                         int32_t* out_accept_len, int32_t* out_next_token,
+                                         int32_t* out_accept_path, int32_t* out_status, float* out_node_qa,
+                                         float* out_node_px, int32_t* out_node_m, void* workspace,
+                                         size_t workspace_bytes, void* cuda_stream) {
+  if (dtype != LANTERN_F32 && dtype != LANTERN_BF16) return LANTERN_E_PARAM;
+  if (B < 0 || N < 0 || N > MAX_N || V < 8 || V > 16384 || (V % 8) != 0 || k < 1 || k > V) return LANTERN_E_SHAPE;
+  if (static_cast<long long>(B) * (N + 1) >= (1ll << 31)) return LANTERN_E_SHAPE;
+  if (!(T >= 0.0f) || !(delta >= 0.0f) || !isfinite(T) || !isfinite(delta)) return LANTERN_E_PARAM;
+  if (has_uncond && !isfinite(cfg_scale)) return LANTERN_E_PARAM;
+  if (T == 0.0f) return LANTERN_E_UNIMPLEMENTED;   // greedy decoding is not part of this build
+  const int esize = dtype == LANTERN_BF16 ? 2 : 4;
+  const int nrows = has_uncond ? 3 : 2;
+  const int CH = V > NT * 8 ? 2 : 1;
+  const size_t smem_bytes = static_cast<size_t>(nrows) * V * esize + static_cast<size_t>(CH) * NT * 8 * 4;
+  if (smem_bytes > 220 * 1024) return LANTERN_E_SHAPE;
+  if (B == 0) return LANTERN_OK;
+  if (!target_logits || !neighbor_idx || !uniforms || !out_accept_len || !out_next_token) return LANTERN_E_NULL;
+  if (N > 0 && (!draft_logits || !draft_tokens)) return LANTERN_E_NULL;
+  if ((reinterpret_cast<uintptr_t>(target_logits) & 15) || (reinterpret_cast<uintptr_t>(draft_logits) & 15))
+    return LANTERN_E_ALIGN;
+  const WsLayout L = ws_layout(B, N);
+  if (!workspace || workspace_bytes < L.total || (reinterpret_cast<uintptr_t>(workspace) & 255))
+    return LANTERN_E_WORKSPACE;
+
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  VerifyParams P;
+  P.target = target_logits;
+  P.draft = draft_logits;
+  P.tokens = draft_tokens;
+  P.parents = tree_parents;
+  P.nbr = neighbor_idx;
+  P.uniforms = uniforms;
+  P.out_len = out_accept_len;
+  P.out_tok = out_next_token;
+  P.out_path = out_accept_path;
+  P.out_status = out_status;
+  P.out_qa = out_node_qa;
+  P.out_px = out_node_px;
+  P.out_m = out_node_m;
+  P.counters = reinterpret_cast<Counters*>(ws + L.counters);
+  P.work_heavy = reinterpret_cast<int32_t*>(ws + L.heavy);
+  P.work_light = reinterpret_cast<int32_t*>(ws + L.light);
+  P.child_start = reinterpret_cast<int32_t*>(ws + L.cstart);
+  P.child_nodes = reinterpret_cast<int32_t*>(ws + L.cnodes);
+  P.records = reinterpret_cast<Record*>(ws + L.records);
+  P.seq_status = reinterpret_cast<int32_t*>(ws + L.seqst);
+  P.bonus_seq = reinterpret_cast<int32_t*>(ws + L.bseq);
+  P.bonus_ctx = reinterpret_cast<int32_t*>(ws + L.bctx);
+  P.B = B;
+  P.N = N;
+  P.R = N + 1;
+  P.V = V;
+  P.k = k;
+  P.cfg_scale = cfg_scale;
+  P.T = T;
+  P.delta = delta;
+
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return LANTERN_E_CUDA;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return LANTERN_E_CUDA;
+  if (sms < 1) return LANTERN_E_CUDA;
+
+  if (cudaMemsetAsync(P.counters, 0, 256, st) != cudaSuccess) return LANTERN_E_CUDA;
+  const size_t plan_smem = static_cast<size_t>(PLAN_WARPS) * (N + 2) * sizeof(int);
+  lantern_plan_kernel<<<(B + PLAN_WARPS - 1) / PLAN_WARPS, PLAN_WARPS * 32, plan_smem, st>>>(P);
+  if (cudaGetLastError() != cudaSuccess) return LANTERN_E_CUDA;
+
+  const long long items = static_cast<long long>(B) * (N + 1);
+  const int grid_ctx = static_cast<int>(items < sms ? items : sms);
+  const int grid_bonus = B < sms ? B : sms;
+  cudaError_t e;
+  const bool bf = dtype == LANTERN_BF16, un = has_uncond != 0;
+#define LANTERN_DISPATCH(CHV)                                                                        \
+  (bf ? (un ? launch_verify<CHV, true, true>(P, grid_ctx, grid_bonus, smem_bytes, st)                \
+            : launch_verify<CHV, true, false>(P, grid_ctx, grid_bonus, smem_bytes, st))              \
+      : (un ? launch_verify<CHV, false, true>(P, grid_ctx, grid_bonus, smem_bytes, st)               \
+            : launch_verify<CHV, false, false>(P, grid_ctx, grid_bonus, smem_bytes, st)))
+  e = CH == 2 ? LANTERN_DISPATCH(2) : LANTERN_DISPATCH(1);
+#undef LANTERN_DISPATCH
+  return e == cudaSuccess ? LANTERN_OK : LANTERN_E_CUDA;
+}
+
+extern "C" const char* lantern_status_string(lantern_status s) {
+  switch (s) {
+    case LANTERN_OK: return "ok";
+    case LANTERN_E_NULL: return "a required pointer is NULL";
+    case LANTERN_E_SHAPE: return "a size is outside the supported range";
+    case LANTERN_E_PARAM: return "a scalar parameter is invalid";
+    case LANTERN_E_WORKSPACE: return "workspace missing, too small or misaligned";
+    case LANTERN_E_CUDA: return "a CUDA runtime call failed";
+    case LANTERN_E_ALIGN: return "a pointer is not 16-byte aligned";
+    case LANTERN_E_UNIMPLEMENTED: return "not implemented in this build";
+    default: return "unknown status";
+  }
+}

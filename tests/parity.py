@@ -1,0 +1,123 @@
+"""Comparison of the CUDA library with the CPU oracle on one verification call.
+
+Rule: accept lengths, next tokens and accepted paths must be identical, except for sequences
+in which some decision of the oracle lies within WINDOW of its threshold (the accept test
+|r - sum_A q / p(x~)|, the prefix cut |moved mass - delta|, or the final draw's distance to a
+CDF edge).  Such a sequence is counted as "near" and must reproduce exactly under the oracle
+once the corresponding input (that node's uniform, delta, or the final uniform) is nudged
+across the window.  Probabilities must agree to REL.
+"""
+from __future__ import annotations
+
+import dataclasses
+
+import numpy as np
+import torch
+
+import lantern_inputs as li
+import oracle
+import paper_2410_03355_b200 as lt
+
+WINDOW = 1e-6
+REL = 1e-5
+
+
+def to_device(inp: li.VerifyInputs, device="cuda"):
+    def logits(a):
+        t = torch.from_numpy(a)
+        if inp.dtype == li.BF16:
+            t = t.view(torch.int16).view(torch.bfloat16)
+        return t.to(device)
+    return dict(
+        target_logits=logits(inp.target_logits), draft_logits=logits(inp.draft_logits),
+        draft_tokens=torch.from_numpy(inp.draft_tokens).to(device),
+        tree_parents=None if inp.tree_parents is None else torch.from_numpy(inp.tree_parents).to(device),
+        uniforms=torch.from_numpy(inp.uniforms).to(device))
+
+
+def run_gpu(inp: li.VerifyInputs, table_dev: torch.Tensor, delta: float, trace=True) -> lt.VerifyOutputs:
+    d = to_device(inp)
+    out = lt.verify(d["target_logits"], d["draft_logits"], inp.cfg_scale, inp.T, d["draft_tokens"],
+                    d["tree_parents"], table_dev, delta, d["uniforms"], trace=trace)
+    torch.cuda.synchronize()
+    return out
+
+
+def _slice(inp: li.VerifyInputs, b: int) -> li.VerifyInputs:
+    return dataclasses.replace(
+        inp, target_logits=np.ascontiguousarray(inp.target_logits[:, b:b + 1]),
+        draft_logits=np.ascontiguousarray(inp.draft_logits[b:b + 1]),
+        draft_tokens=np.ascontiguousarray(inp.draft_tokens[b:b + 1]),
+        tree_parents=None if inp.tree_parents is None else np.ascontiguousarray(inp.tree_parents[b:b + 1]),
+        uniforms=inp.uniforms[b:b + 1].copy(), B=1)
+
+
+def _explained_by_window(inp, table, delta, b, ora, want) -> bool:
+    """Does the oracle give `want` = (len, token, path) once a near-threshold input is nudged?"""
+    one = _slice(inp, b)
+    eps = 4 * WINDOW
+    trials = []
+    near_nodes = [i for i in range(inp.N) if ora.tested[b, i] and ora.margin[b, i] < WINDOW]
+    for i in near_nodes:
+        for s in (-eps, eps):
+            u = one.uniforms.copy()
+            u[0, i] = np.float32(min(max(u[0, i] + s, 0.0), 1.0 - 2.0 ** -24))
+            trials.append((u, delta))
+    if near_nodes:
+        trials += [(one.uniforms, delta - eps), (one.uniforms, delta + eps)]
+    if ora.draw_margin[b] < WINDOW:
+        for s in (-eps, eps):
+            u = one.uniforms.copy()
+            u[0, inp.N] = np.float32(min(max(u[0, inp.N] + s, 0.0), 1.0 - 2.0 ** -24))
+            trials.append((u, delta))
+    for u, d in trials:
+        r = oracle.verify_inputs(dataclasses.replace(one, uniforms=u), table, max(d, 0.0))
+        if (r.accept_len[0], r.next_token[0]) == want[:2] and np.array_equal(r.accept_path[0], want[2]):
+            return True
+    return False
+
+
+def compare(inp: li.VerifyInputs, table: np.ndarray, delta: float, gpu: lt.VerifyOutputs, ora=None):
+    """Returns dict(n_seq, near, mismatch_outside, prob_bad, ...); asserts nothing itself."""
+    if ora is None:
+        ora = oracle.verify_inputs(inp, table, delta)
+    g_len = gpu.accept_len.cpu().numpy()
+    g_tok = gpu.next_token.cpu().numpy()
+    g_path = gpu.accept_path.cpu().numpy()
+    g_st = gpu.status.cpu().numpy()
+    near = outside = 0
+    bad = []
+    for b in range(inp.B):
+        same = (g_len[b] == ora.accept_len[b] and g_tok[b] == ora.next_token[b]
+                and np.array_equal(g_path[b], ora.accept_path[b]))
+        if same:
+            continue
+        if _explained_by_window(inp, table, delta, b, ora, (g_len[b], g_tok[b], g_path[b])):
+            near += 1
+        else:
+            outside += 1
+            bad.append(b)
+    res = dict(n_seq=inp.B, near=near, mismatch_outside=outside, bad=bad,
+               status_equal=bool(np.array_equal(g_st, ora.status)), accept_mean=float(ora.accept_len.mean()))
+    if gpu.node_qa is not None:
+        qa, px, m = gpu.node_qa.cpu().numpy(), gpu.node_px.cpu().numpy(), gpu.node_m.cpu().numpy()
+        t = ora.tested.astype(bool) & (ora.status[:, None] == 0)
+        far = t & (ora.margin >= WINDOW)
+        # A different cut changes sum_A q legitimately, so probabilities are compared where the cut agrees
+        # (which it must, away from the window).
+        res["m_mismatch_outside"] = int((m[far] != ora.m[far]).sum())
+        agree = t & (m == ora.m)
+        rel_qa = np.abs(qa[agree] - ora.qa[agree]) / np.maximum(ora.qa[agree], 1e-30)
+        rel_px = np.abs(px[t] - ora.px[t]) / np.maximum(ora.px[t], 1e-30)
+        res["qa_rel_max"] = float(rel_qa.max()) if rel_qa.size else 0.0
+        res["px_rel_max"] = float(rel_px.max()) if rel_px.size else 0.0
+        res["nodes_tested"] = int(t.sum())
+    return res
+
+
+def assert_parity(res):
+    assert res["mismatch_outside"] == 0, res
+    assert res["status_equal"], res
+    if "qa_rel_max" in res:
+        assert res["m_mismatch_outside"] == 0, res
+        assert res["qa_rel_max"] < REL and res["px_rel_max"] < REL, res

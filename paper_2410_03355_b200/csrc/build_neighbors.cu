@@ -90,7 +90,8 @@ __global__ void __launch_bounds__(256) lantern_distance_tile_kernel(const float*
 __global__ void __launch_bounds__(BT) lantern_knn_row_kernel(BuildParams P, int P2 /* pow2 >= k-1 */) {
   extern __shared__ __align__(16) unsigned char dsm[];
   uint32_t* keys = reinterpret_cast<uint32_t*>(dsm);                                  // [V]
-  unsigned long long* list = reinterpret_cast<unsigned long long*>(dsm + static_cast<size_t>(P.V) * 4);  // [P2]
+  unsigned long long* list =
+      reinterpret_cast<unsigned long long*>(dsm + ((static_cast<size_t>(P.V) * 4 + 15) & ~size_t(15)));  // [P2]
   __shared__ int hist[256];
   __shared__ int wcnt[BW];
   __shared__ float ai[SMALL_D];
@@ -294,7 +295,7 @@ extern "C" lantern_status lantern_build_neighbors(const float* codebook, int V, 
     return LANTERN_E_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const int P2 = k > 1 ? next_pow2(k - 1 < 2 ? 2 : k - 1) : 2;
-  const size_t smem = static_cast<size_t>(V) * 4 + static_cast<size_t>(P2) * 8;
+  const size_t smem = ((static_cast<size_t>(V) * 4 + 15) & ~size_t(15)) + static_cast<size_t>(P2) * 8;
   if (smem > 220 * 1024) return LANTERN_E_SHAPE;
   if (cudaFuncSetAttribute(lantern_knn_row_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) !=
       cudaSuccess)

@@ -664,7 +664,9 @@ __global__ void __launch_bounds__(NT, 1) lantern_context_kernel(VerifyParams P) 
         }
       }
     }
-    status = __syncthreads_or(status);
+    // NONFINITE / DEGENERATE are set by every thread alike; a bad table entry is seen by one thread
+    status = (status & ~LANTERN_ST_BAD_TABLE) |
+             (__syncthreads_or(status & LANTERN_ST_BAD_TABLE) ? LANTERN_ST_BAD_TABLE : 0);
     if (tid == 0) {
       Record rec = {accepted, token, status, 0};
       P.records[item] = rec;

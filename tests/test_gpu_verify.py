@@ -78,7 +78,7 @@ def test_trees(depth, N):
         for delta in (0.0, 0.05, 0.3):
             res = check(inp, host, dev, delta, min_tested=24)
             n_sib += res["nodes_tested"]
-    assert n_sib > 24 * 4 * 3 * 2          # sibling rounds were exercised
+    assert n_sib > 24 * 4 * 3 * 1.5        # sibling rounds were exercised
 
 
 def test_chain_equals_explicit_tree():

@@ -1,0 +1,393 @@
+#!/usr/bin/env python
+"""Benchmark of the LANTERN relaxed-verification step (metric: verified draft positions per second).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload batch_chain|stress|...] [--impl reference]
+
+A step is one `verify` call over one batch of synthetic input: every drafted position of every
+sequence is tested (guidance combine, softmax of target and drafter, A_{k,delta} aggregation,
+relaxed accept test, residual resampling, walk, bonus draw).  The default workload is the
+V = 16384, k = 1000, delta = 0.4 chain configuration with its 32 images x 256 positions
+flattened into one call of 8192 sequences x 7 drafts (6.4 GB of bf16 logits, far larger than
+L2, so consecutive steps cannot be served from cache).  The neighbour table is built once
+before the timed region, as in the method, and its build time is reported separately.
+
+With N > 1 (under torch.distributed.run) every rank verifies its own batch of the same
+shape: the path has no exchange step, so this is weak scaling with no collective on the
+data path; the ranks only meet at the timing barriers.
+
+`--impl reference` times the CPU oracle (oracle/, as it stands, one thread) on a bounded
+sample of the same workload and prints the same JSON line with "impl": "reference".
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "relaxed_verify_positions_per_s"
+UNIT = "positions/s"
+
+# the paper's guidance/neighbourhood settings per workload; B is the flattened call size
+WORKLOADS = {
+    "batch_chain": dict(config="batch_chain", B=32 * 256, note="32 images x 256 positions, chain of 7 drafts"),
+    "stress": dict(config="stress", B=128, note="128 sequences x 60-node depth-6 trees"),
+    "px512_tree": dict(config="px512_tree", B=8 * 64, note="8 images x 64 positions, 60-node trees"),
+    "single_image": dict(config="single_image", B=256, note="1 image x 256 positions, 60-node trees"),
+    "tiny": dict(config="tiny", B=64, note="64 steps of the tiny chain configuration"),
+}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+def algorithmic_bytes(cfg: dict, B: int, parents) -> int:
+    """Bytes the method must move per call: for each context with at least one child, two target
+    rows and one drafter row (one target row without guidance), plus one neighbour row of 4k
+    bytes per drafted node.  Bonus rows, tokens, uniforms and outputs (< 0.1 %) are left out."""
+    import lantern_inputs as li
+    esize = 2 if cfg["dtype"] == li.BF16 else 4
+    rows = 3 if cfg["has_uncond"] else 2
+    N, V, k = cfg["N"], cfg["V"], cfg["k"]
+    if parents is None:
+        n_ctx = B * N
+    else:
+        par = parents.cpu().numpy()
+        n_ctx = sum(len(set(par[b].tolist())) for b in range(B))
+    return n_ctx * rows * V * esize + B * N * 4 * k
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_sample_rate(host_inp, table_host, delta, budget_s=20.0):
+    """Oracle throughput (drafted positions verified per second) on as many leading sequences of
+    `host_inp` as fit in about `budget_s` seconds; returns (rate, n_sequences, seconds)."""
+    import dataclasses
+
+    import oracle
+    done, t_used, pos = 0, 0.0, 0
+    chunk = 8
+    while done < host_inp.B and t_used < budget_s:
+        n = min(chunk, host_inp.B - done)
+        sl = slice(done, done + n)
+        part = dataclasses.replace(
+            host_inp, target_logits=np.ascontiguousarray(host_inp.target_logits[:, sl]),
+            draft_logits=np.ascontiguousarray(host_inp.draft_logits[sl]),
+            draft_tokens=np.ascontiguousarray(host_inp.draft_tokens[sl]),
+            tree_parents=None if host_inp.tree_parents is None else np.ascontiguousarray(host_inp.tree_parents[sl]),
+            uniforms=np.ascontiguousarray(host_inp.uniforms[sl]), B=n)
+        t0 = time.perf_counter()
+        oracle.verify_inputs(part, table_host, delta)
+        t_used += time.perf_counter() - t0
+        done += n
+        pos += n * host_inp.N
+        chunk = min(chunk * 2, 256)
+    return pos / t_used, done, t_used
+
+
+def run_reference(args, rank, world):
+    """The reference arm: the CPU oracle as it stands, timed on host cores on a bounded sample."""
+    if rank != 0:
+        return
+    import lantern_inputs as li
+    import oracle
+    w = WORKLOADS[args.workload]
+    cfg = li.CONFIGS[w["config"]]
+    # bounded sample: a few sequences per step so that the run ends within minutes
+    nseq = {"batch_chain": 64, "stress": 4, "px512_tree": 4, "single_image": 4, "tiny": 64}[args.workload]
+    cb = li.config_codebook(w["config"])
+    steps_t = []
+    table_cache = {}   # the table is an input of the step: only the rows the sample's drafts touch are built
+
+    def table_for(inp):
+        need = np.unique(inp.draft_tokens)
+        miss = np.array([t for t in need if t not in table_cache], dtype=np.int32)
+        if miss.size:
+            idx, _ = oracle.build_neighbors(cb, cfg["k"], rows=miss)
+            for r, t in enumerate(miss):
+                table_cache[int(t)] = idx[r]
+        tab = np.zeros((cfg["V"], cfg["k"]), np.int32)
+        tab[:, 0] = np.arange(cfg["V"])
+        for t in need:
+            tab[t] = table_cache[int(t)]
+        return tab
+
+    for step in range(args.warmup + args.steps):
+        inp = li.config_verify_inputs(w["config"], step=step, B=nseq)
+        tab = table_for(inp)
+        t1 = time.perf_counter()
+        oracle.verify_inputs(inp, tab, cfg["delta"])
+        dt = time.perf_counter() - t1
+        if step >= args.warmup:
+            steps_t.append(dt)
+    total = sum(steps_t)
+    value = nseq * cfg["N"] * len(steps_t) / total
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(steps_t),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "V": cfg["V"], "k": cfg["k"], "delta": cfg["delta"], "N": cfg["N"],
+                   "sequences_per_step": nseq},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+                         "sample": f"{nseq} sequences x {cfg['N']} drafts per step of the {args.workload} workload "
+                                   f"(bounded sample; neighbour rows built by the oracle outside the timed region)"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="batch_chain", choices=sorted(WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--batch", type=int, default=0, help="override the number of sequences per call")
+    ap.add_argument("--rho", type=float, default=0.0, help="correlation of conditional and unconditional rows")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+
+    import torch
+
+    import lantern_inputs as li
+    import lantern_inputs.device as lid
+    import paper_2410_03355_b200 as lt
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    lt.load_library()
+
+    w = WORKLOADS[args.workload]
+    cfg = li.CONFIGS[w["config"]]
+    B = args.batch or w["B"]
+    N, V, k, delta = cfg["N"], cfg["V"], cfg["k"], cfg["delta"]
+
+    # ---- one-time neighbour table (timed separately) ----
+    cb = torch.from_numpy(li.config_codebook(w["config"])).cuda()
+    bws = torch.empty(max(lt.build_workspace_bytes(V, cfg["D"], k), 16), dtype=torch.uint8, device="cuda")
+    lt.build_neighbors(cb, k, with_dist=False, workspace=bws)      # warm-up
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    table, _ = lt.build_neighbors(cb, k, with_dist=False, workspace=bws)
+    e1.record()
+    torch.cuda.synchronize()
+    build_ms = e0.elapsed_time(e1)
+    del bws
+
+    # ---- inputs resident in HBM ----
+    d = lid.config_verify_inputs_device(w["config"], B=B, seed=li.BASE_SEED + 17 * rank, rho=args.rho)
+    torch.cuda.synchronize()
+    alg_bytes = algorithmic_bytes(cfg, B, d["tree_parents"])
+    ws = torch.empty(lt.verify_workspace_bytes(B, N), dtype=torch.uint8, device="cuda")
+    i32 = dict(dtype=torch.int32, device="cuda")
+    out = lt.VerifyOutputs(accept_len=torch.empty(B, **i32), next_token=torch.empty(B, **i32),
+                           accept_path=torch.empty((B, N), **i32), status=torch.empty(B, **i32),
+                           node_qa=None, node_px=None, node_m=None)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        lt.verify(d["target_logits"], d["draft_logits"], d["cfg_scale"], d["T"], d["draft_tokens"], d["tree_parents"],
+                  table, delta, d["uniforms"], out=out, workspace=ws, stream=stream)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+
+    # per-step events around the fused kernel (dominant kernel of the roofline)
+    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for a, b_ in kev:       # torch creates the CUDA event on first record
+        a.record()
+        b_.record()
+    torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t_start, t_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    for a, b_ in kev:
+        lt.profile_events(a, b_)
+        step()
+    t_stop.record()
+    torch.cuda.synchronize()
+    lt.profile_events(None, None)
+    if dist is not None:
+        dist.barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = t_start.elapsed_time(t_stop)
+    fused_ms = float(np.mean([a.elapsed_time(b_) for a, b_ in kev]))
+    if dist is not None:
+        t = torch.tensor([ms_total, fused_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total, fused_ms = float(t[0]), float(t[1])
+    ms_per_step = ms_total / args.steps
+    value = world * B * N / (ms_per_step * 1e-3)
+
+    status_bad = int((out.status != 0).sum().item())
+    accept_mean = float(out.accept_len.float().mean().item())
+
+    # ---- end to end: host buffers in, host results out, through the public API ----
+    e2e = None
+    if not args.no_e2e:
+        host = {}
+        for name in ("target_logits", "draft_logits", "draft_tokens", "tree_parents", "uniforms"):
+            t = d[name]
+            host[name] = None if t is None else torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t)
+        h_len = torch.empty(B, dtype=torch.int32, pin_memory=True)
+        h_tok = torch.empty(B, dtype=torch.int32, pin_memory=True)
+        h2d = sum(t.numel() * t.element_size() for t in host.values() if t is not None)
+        d2h = 2 * B * 4
+
+        def e2e_step():
+            for name, t in host.items():
+                if t is not None:
+                    d[name].copy_(t, non_blocking=True)
+            step()
+            h_len.copy_(out.accept_len, non_blocking=True)
+            h_tok.copy_(out.next_token, non_blocking=True)
+
+        e2e_step()
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        b_.record()
+        torch.cuda.synchronize()
+        ms_e2e = a.elapsed_time(b_) / args.e2e_steps
+        if dist is not None:
+            t = torch.tensor([ms_e2e], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t[0])
+        e2e = {"value": world * B * N / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+               "d2h_bytes_per_step": int(d2h), "ms_per_step": ms_e2e, "steps": args.e2e_steps}
+        del host
+
+    # ---- CPU baseline: the oracle on a bounded sample of the same inputs (rank 0, N = 1) ----
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        n_s = min(B, 2048)
+        host_inp = lid.to_host(d, rows=np.arange(n_s))
+        rate, n_done, secs = oracle_sample_rate(host_inp, table.cpu().numpy(), delta)
+        cpu = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": f"first {n_done} sequences ({n_done * N} drafted positions) of this call, {secs:.1f} s"}
+
+    if rank == 0:
+        peak, peak_kind = load_peaks()
+        achieved = alg_bytes / (fused_ms * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": args.workload, "note": w["note"], "sequences_per_call": B, "drafts_per_sequence": N,
+                       "V": V, "k": k, "delta": delta, "cfg_scale": cfg["cfg_scale"], "T": cfg["T"],
+                       "logits": "bf16" if cfg["dtype"] == li.BF16 else "f32", "rho": args.rho,
+                       "l2_policy": "inputs larger than L2 (%.2f GB of logits per call)" %
+                                    ((d["target_logits"].numel() + d["draft_logits"].numel()) *
+                                     d["target_logits"].element_size() / 1e9),
+                       "parallelism": "replicas" if world > 1 else "single"},
+            "roofline": {"bound": "hbm", "kernel": "lantern_context_kernel", "achieved": achieved, "peak": peak,
+                         "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                         "algorithmic_bytes_per_launch": int(alg_bytes), "kernel_ms": fused_ms},
+            "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": 4 * args.steps, "clocks": clocks,
+            "neighbor_build": {"ms": build_ms, "V": V, "D": cfg["D"], "k": k,
+                               "pairs_per_s": V * V / (build_ms * 1e-3)},
+            "outputs": {"mean_accept_len": accept_mean, "sequences_with_status_bits": status_bad},
+        }
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

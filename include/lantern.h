@@ -137,6 +137,13 @@ lantern_status lantern_verify(const void* target_logits, const void* draft_logit
 /* Number of kernels (and memsets) one lantern_verify call enqueues; for launch accounting. */
 int lantern_verify_launch_count(void);
 
+/* Measurement hook (not part of the method): when both arguments are non-NULL cudaEvent_t
+ * handles, every later lantern_verify call made by the calling host thread records
+ * `before_fused` on its stream right before the fused context kernel and `after_fused` right
+ * after it, so that a benchmark can time that kernel alone with CUDA events.  Pass two NULLs
+ * to switch it off.  The events are owned by the caller. */
+lantern_status lantern_verify_profile_events(void* before_fused, void* after_fused);
+
 #ifdef __cplusplus
 }
 #endif

@@ -52,6 +52,8 @@ def load_library():
     lib.lantern_verify_workspace_bytes.argtypes = [i32, i32]
     lib.lantern_verify_launch_count.restype = i32
     lib.lantern_verify_launch_count.argtypes = []
+    lib.lantern_verify_profile_events.restype = i32
+    lib.lantern_verify_profile_events.argtypes = [vp, vp]
     lib.lantern_verify.restype = i32
     lib.lantern_verify.argtypes = [vp, vp, i32, f32, i32, f32, vp, vp, vp, i32, f32, vp, i32, i32, i32,
                                    vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -167,3 +169,21 @@ def verify(target_logits: torch.Tensor, draft_logits: Optional[torch.Tensor], cf
     if rc != 0:
         raise LanternError(rc, "lantern_verify")
     return out
+
+
+def verify_launch_count() -> int:
+    """Stream operations (4 kernels + 1 memset) enqueued by one verify() call."""
+    return int(load_library().lantern_verify_launch_count())
+
+
+def profile_events(before: Optional[torch.cuda.Event], after: Optional[torch.cuda.Event]) -> None:
+    """lantern_verify_profile_events: record `before` / `after` around the fused context kernel of every
+    later verify() call of this thread (both None switches it off).  Events need enable_timing=True and
+    must have been recorded once (torch creates the CUDA event lazily)."""
+    lib = load_library()
+    if before is None or after is None:
+        rc = lib.lantern_verify_profile_events(None, None)
+    else:
+        rc = lib.lantern_verify_profile_events(ctypes.c_void_p(before.cuda_event), ctypes.c_void_p(after.cuda_event))
+    if rc != 0:
+        raise LanternError(rc, "lantern_verify_profile_events")

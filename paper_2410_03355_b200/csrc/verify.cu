@@ -829,15 +829,19 @@ static WsLayout ws_layout(int B, int N) {
   return L;
 }
 
+static thread_local cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
+
 template <int CH, bool BF16, bool UNC>
 static cudaError_t launch_verify(const VerifyParams& P, int grid_ctx, int grid_bonus, size_t smem_bytes,
                                  cudaStream_t st) {
   auto kc = lantern_context_kernel<CH, BF16, UNC>;
   cudaError_t e = cudaFuncSetAttribute(kc, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
   if (e != cudaSuccess) return e;
+  if (g_ev_before && g_ev_after) cudaEventRecord(g_ev_before, st);
   kc<<<grid_ctx, NT, smem_bytes, st>>>(P);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
+  if (g_ev_before && g_ev_after) cudaEventRecord(g_ev_after, st);
   lantern_walk_kernel<<<(P.B + 127) / 128, 128, 0, st>>>(P);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
@@ -855,6 +859,13 @@ extern "C" size_t lantern_verify_workspace_bytes(int B, int N) {
 }
 
 extern "C" int lantern_verify_launch_count(void) { return 5; }
+
+extern "C" lantern_status lantern_verify_profile_events(void* before_fused, void* after_fused) {
+  if ((before_fused == nullptr) != (after_fused == nullptr)) return LANTERN_E_NULL;
+  g_ev_before = static_cast<cudaEvent_t>(before_fused);
+  g_ev_after = static_cast<cudaEvent_t>(after_fused);
+  return LANTERN_OK;
+}
 
 extern "C" lantern_status lantern_verify(const void* target_logits, const void* draft_logits, int dtype,
                                          float cfg_scale, int has_uncond, float T, const int32_t* draft_tokens,

@@ -134,6 +134,46 @@ lantern_status lantern_verify(const void* target_logits, const void* draft_logit
                               float* out_node_px, int32_t* out_node_m, void* workspace, size_t workspace_bytes,
                               void* cuda_stream);
 
+/* ------------------------------------------------------------------------------------------
+ * lantern_verify without a caller-supplied workspace.  (The paper has no counterpart: this
+ * entry point exists for integration reasons only and computes exactly what lantern_verify
+ * computes.)
+ *
+ * Who needs it: code that may not allocate device memory at the point where it verifies
+ * drafts -- a serving loop whose HBM was handed out in full at start-up (KV cache, activation
+ * arenas) so that a cudaMalloc would fail or fragment it, a plug-in that runs under an
+ * allocator it does not own, or a latency-critical step that cannot afford the device-wide
+ * synchronisation a cudaMalloc / cudaFree implies.  Such callers still own the inputs and
+ * outputs; only the scratch that lantern_verify asks for is taken off their hands.
+ *
+ * The scratch lives in a fixed array inside the library's device image,
+ * LANTERN_STATIC_WORKSPACE_BYTES (4 MiB) large: every GPU on which the library is loaded
+ * holds those 4 MiB until the process exits.  The call makes no cudaMalloc / cudaFree and
+ * calls nothing that allocates.
+ *
+ *   - Sizes: lantern_verify_workspace_bytes(B, N) must not exceed
+ *     LANTERN_STATIC_WORKSPACE_BYTES (e.g. B = 8192, N = 7 or B = 1024, N = 60 fit);
+ *     otherwise the call returns LANTERN_E_WORKSPACE and does nothing.  All other argument
+ *     rules and return codes are those of lantern_verify.
+ *   - First call on a device: the library looks up the device address of its array (once per
+ *     device, with that device current, no allocation).  Make that first call outside any
+ *     stream capture.
+ *   - The array is shared by every call on that device and keeps the previous call's contents;
+ *     the call itself resets the few words that must start at zero.  Two such calls that may
+ *     run on the GPU at the same time (different streams, different host threads) would write
+ *     the same scratch and corrupt each other: serialise them, or use lantern_verify with
+ *     separate workspaces.
+ * ---------------------------------------------------------------------------------------- */
+#define LANTERN_STATIC_WORKSPACE_BYTES (4u << 20)
+
+lantern_status lantern_verify_static(const void* target_logits, const void* draft_logits, int dtype,
+                                     float cfg_scale, int has_uncond, float T, const int32_t* draft_tokens,
+                                     const int32_t* tree_parents, const int32_t* neighbor_idx, int k, float delta,
+                                     const float* uniforms, int B, int N, int V, int32_t* out_accept_len,
+                                     int32_t* out_next_token, int32_t* out_accept_path, int32_t* out_status,
+                                     float* out_node_qa, float* out_node_px, int32_t* out_node_m,
+                                     void* cuda_stream);
+
 /* Number of kernels (and memsets) one lantern_verify call enqueues; for launch accounting. */
 int lantern_verify_launch_count(void);
 

@@ -52,6 +52,9 @@ def load_library():
     lib.lantern_verify_workspace_bytes.argtypes = [i32, i32]
     lib.lantern_verify_launch_count.restype = i32
     lib.lantern_verify_launch_count.argtypes = []
+    lib.lantern_verify_static.restype = i32
+    lib.lantern_verify_static.argtypes = [vp, vp, i32, f32, i32, f32, vp, vp, vp, i32, f32, vp, i32, i32, i32,
+                                          vp, vp, vp, vp, vp, vp, vp, vp]
     lib.lantern_verify_profile_events.restype = i32
     lib.lantern_verify_profile_events.argtypes = [vp, vp]
     lib.lantern_verify.restype = i32
@@ -187,3 +190,44 @@ def profile_events(before: Optional[torch.cuda.Event], after: Optional[torch.cud
         rc = lib.lantern_verify_profile_events(ctypes.c_void_p(before.cuda_event), ctypes.c_void_p(after.cuda_event))
     if rc != 0:
         raise LanternError(rc, "lantern_verify_profile_events")
+
+
+STATIC_WORKSPACE_BYTES = 4 << 20
+
+
+def verify_static(target_logits: torch.Tensor, draft_logits: Optional[torch.Tensor], cfg_scale: float, T: float,
+                  draft_tokens: Optional[torch.Tensor], tree_parents: Optional[torch.Tensor],
+                  neighbor_idx: torch.Tensor, delta: float, uniforms: torch.Tensor, *, out: VerifyOutputs,
+                  stream: Optional[torch.cuda.Stream] = None) -> VerifyOutputs:
+    """lantern_verify_static: verify() for callers that must not allocate device memory.
+
+    The library's scratch comes from a fixed 4 MiB array inside its device image, so nothing is
+    allocated here either: the caller passes every output tensor in `out` (allocated whenever it was
+    still allowed to).  The call is refused (LanternError, code -4) if verify_workspace_bytes(B, N)
+    exceeds STATIC_WORKSPACE_BYTES.  Calls on one device share the array: do not let two of them run
+    on the GPU at the same time.  Make the first call on a device outside stream capture."""
+    lib = load_library()
+    C, B, R, V = target_logits.shape
+    N = R - 1
+    if C not in (1, 2):
+        raise ValueError("target_logits must have 1 or 2 guidance branches")
+    if target_logits.dtype == torch.bfloat16:
+        dtype = BF16
+    elif target_logits.dtype == torch.float32:
+        dtype = F32
+    else:
+        raise ValueError("logits must be float32 or bfloat16")
+    if neighbor_idx.shape[0] != V:
+        raise ValueError("neighbor_idx must have V rows")
+    with torch.cuda.device(target_logits.device):
+        rc = lib.lantern_verify_static(
+            _ptr(target_logits, None, "target_logits"), _ptr(draft_logits, target_logits.dtype, "draft_logits"),
+            dtype, float(cfg_scale), int(C == 2), float(T), _ptr(draft_tokens, torch.int32, "draft_tokens"),
+            _ptr(tree_parents, torch.int32, "tree_parents"), _ptr(neighbor_idx, torch.int32, "neighbor_idx"),
+            int(neighbor_idx.shape[1]), float(delta), _ptr(uniforms, torch.float32, "uniforms"), B, N, V,
+            _ptr(out.accept_len, torch.int32), _ptr(out.next_token, torch.int32),
+            _ptr(out.accept_path, torch.int32), _ptr(out.status, torch.int32), _ptr(out.node_qa, torch.float32),
+            _ptr(out.node_px, torch.float32), _ptr(out.node_m, torch.int32), _stream_ptr(stream))
+    if rc != 0:
+        raise LanternError(rc, "lantern_verify_static")
+    return out

@@ -954,6 +954,50 @@ extern "C" lantern_status lantern_verify(const void* target_logits, const void* 
   return e == cudaSuccess ? LANTERN_OK : LANTERN_E_CUDA;
 }
 
+// ---------------------------------------------------------------------------------------
+// lantern_verify_static: same computation, scratch taken from a fixed array in the device
+// image instead of a caller workspace (for callers that must not allocate device memory).
+// ---------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_workspace[LANTERN_STATIC_WORKSPACE_BYTES];
+
+// In host code `g_static_workspace` is only a handle for the symbol, never an address a kernel
+// could use; the device address is asked for once per device and remembered here.
+static void* g_static_workspace_ptr[64] = {};
+
+static lantern_status static_workspace_address(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return LANTERN_E_CUDA;
+  void* p = __atomic_load_n(&g_static_workspace_ptr[dev], __ATOMIC_ACQUIRE);
+  if (!p) {
+    if (cudaGetSymbolAddress(&p, g_static_workspace) != cudaSuccess || !p) return LANTERN_E_CUDA;
+    __atomic_store_n(&g_static_workspace_ptr[dev], p, __ATOMIC_RELEASE);   // same value whoever wins
+  }
+  *out = p;
+  return LANTERN_OK;
+}
+
+extern "C" lantern_status lantern_verify_static(const void* target_logits, const void* draft_logits, int dtype,
+                                                float cfg_scale, int has_uncond, float T,
+                                                const int32_t* draft_tokens, const int32_t* tree_parents,
+                                                const int32_t* neighbor_idx, int k, float delta,
+                                                const float* uniforms, int B, int N, int V,
+                                                int32_t* out_accept_len, int32_t* out_next_token,
+                                                int32_t* out_accept_path, int32_t* out_status, float* out_node_qa,
+                                                float* out_node_px, int32_t* out_node_m, void* cuda_stream) {
+  if (B < 0 || N < 0 || N > MAX_N) return LANTERN_E_SHAPE;
+  // the fixed array bounds the call size: refuse anything whose scratch would not fit
+  if (B > 0 && ws_layout(B, N).total > static_cast<size_t>(LANTERN_STATIC_WORKSPACE_BYTES)) return LANTERN_E_WORKSPACE;
+  void* ws = nullptr;
+  const lantern_status rc = static_workspace_address(&ws);
+  if (rc != LANTERN_OK) return rc;
+  // lantern_verify zeroes the counters at the head of the scratch on the stream before its first
+  // kernel, so whatever the previous call left in the array does not matter.
+  return lantern_verify(target_logits, draft_logits, dtype, cfg_scale, has_uncond, T, draft_tokens, tree_parents,
+                        neighbor_idx, k, delta, uniforms, B, N, V, out_accept_len, out_next_token, out_accept_path,
+                        out_status, out_node_qa, out_node_px, out_node_m, ws, LANTERN_STATIC_WORKSPACE_BYTES,
+                        cuda_stream);
+}
+
 extern "C" const char* lantern_status_string(lantern_status s) {
   switch (s) {
     case LANTERN_OK: return "ok";

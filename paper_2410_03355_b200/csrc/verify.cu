@@ -34,16 +34,35 @@ constexpr int LOG_NT = 10;
 constexpr int MAX_N = 1024;
 
 struct Counters {               // first 256 bytes of the workspace, zeroed per call
-  int work_next;                // next work item to hand out
+  int work_next;                // dynamic part of the work counter
   int n_heavy;                  // contexts with >= 2 children (handed out first)
   int n_light;                  // contexts with exactly 1 child
   int n_bonus;                  // sequences whose walk ended on a childless context
 };
 
 struct Record {                 // result of one context
-  int accepted;                 // accepted child node, or -1 if every child was rejected
+  int accepted;                 // accepted child node; -1 if every child was rejected; kLeaf if it has none
   int token;                    // replacement token if every child was rejected
   int status;                   // LANTERN_ST_* bits found in this context
+  int pad;
+};
+constexpr int kLeaf = -2;
+
+struct ChildInfo {              // one drafted node, stored in the order its parent context tries it
+  int node;                     // node index within the sequence
+  int token;                    // x~
+  float r;                      // its acceptance uniform
+  int pad;
+};
+
+struct WorkItem {               // one context with children: everything its CTA needs, in one 32-byte load
+  int item;                     // b * R + c  (row index of the context); -1 = none
+  int cbase;                    // index of its first child in the ChildInfo array
+  int nchild;
+  int node0;                    // first child, inlined
+  int tok0;
+  float r0;
+  float u_final;                // the sequence's uniform for the final draw
   int pad;
 };
 
@@ -63,10 +82,8 @@ struct VerifyParams {
   int32_t* out_m;
   // workspace pieces
   Counters* counters;
-  int32_t* work_heavy;
-  int32_t* work_light;
-  int32_t* child_start;         // [B, R+1]
-  int32_t* child_nodes;         // [B, N]
+  WorkItem* work;               // [B*N]: heavy items from the front, light items from the back
+  ChildInfo* children;          // [B, N]
   Record* records;              // [B, R]
   int32_t* seq_status;          // [B]
   int32_t* bonus_seq;           // [B]
@@ -299,8 +316,8 @@ __device__ __forceinline__ void load_rows(const unsigned char* stage, int rowbyt
 
 // ---------------------------------------------------------------------------------------
 // kernel 1: plan.  One warp per sequence: validate tokens / parents / uniforms, bucket the
-// nodes by parent context (children in node order), initialise the per-node outputs and
-// append the contexts that have children to the work lists.
+// nodes by parent context (children in node order), initialise the per-node outputs, mark
+// childless contexts, and append one self-contained work item per context with children.
 // ---------------------------------------------------------------------------------------
 constexpr int PLAN_WARPS = 4;
 
@@ -310,7 +327,8 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
   const int b = blockIdx.x * PLAN_WARPS + warp;
   if (b >= P.B) return;
   const int N = P.N, R = P.R;
-  int* cnt = plan_smem + warp * (R + 1);       // cnt[c], c in [0, R]; later the fill cursor
+  int* cnt = plan_smem + warp * 2 * (R + 1);   // cnt[c]: number of children of context c
+  int* cur = cnt + (R + 1);                    // fill cursor, ends as the end offset of context c
   for (int i = lane; i <= R; i += 32) cnt[i] = 0;
   __syncwarp();
   int status = 0;
@@ -333,13 +351,26 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
   }
   status = __reduce_or_sync(kFull, status);
   __syncwarp();
-  int32_t* cstart = P.child_start + static_cast<size_t>(b) * (R + 1);
   if (lane == 0) P.seq_status[b] = status;
-  if (status) {
-    for (int i = lane; i <= R; i += 32) cstart[i] = 0;
-    return;
+  if (status) return;   // the walk reports the fault; no work is queued for this sequence
+
+  ChildInfo* kids = P.children + static_cast<size_t>(b) * N;
+  if (lane == 0) {      // children of each context, in node order
+    int run = 0;
+    for (int c = 0; c < R; ++c) {
+      cur[c] = run;
+      run += cnt[c];
+    }
+    for (int i = 0; i < N; ++i) {
+      const size_t o = static_cast<size_t>(b) * N + i;
+      const int par = P.parents ? P.parents[o] : i - 1;
+      ChildInfo ci = {i, P.tokens[o], P.uniforms[static_cast<size_t>(b) * R + i], 0};
+      kids[cur[par + 1]++] = ci;
+    }
   }
-  // work items (before the counts are turned into cursors)
+  __syncwarp();         // lane 0's writes to cur[] and kids[] are visible to the warp
+  const float u_final = P.uniforms[static_cast<size_t>(b) * R + N];
+  const int cap = P.B * N;
   for (int base = 0; base < R; base += 32) {
     const int c = base + lane;
     const int n = c < R ? cnt[c] : 0;
@@ -353,23 +384,17 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
     hb = __shfl_sync(kFull, hb, 0);
     lb = __shfl_sync(kFull, lb, 0);
     const unsigned below = (1u << lane) - 1u;
-    if (n >= 2) P.work_heavy[hb + __popc(heavy & below)] = b * R + c;
-    if (n == 1) P.work_light[lb + __popc(light & below)] = b * R + c;
-  }
-  __syncwarp();
-  if (lane == 0) {
-    int run = 0;
-    for (int c = 0; c < R; ++c) {
-      const int n = cnt[c];
-      cstart[c] = run;
-      cnt[c] = run;
-      run += n;
-    }
-    cstart[R] = run;
-    int32_t* cn = P.child_nodes + static_cast<size_t>(b) * N;
-    for (int i = 0; i < N; ++i) {
-      const int par = P.parents ? P.parents[static_cast<size_t>(b) * N + i] : i - 1;
-      cn[cnt[par + 1]++] = i;
+    if (c < R) {
+      if (n == 0) {
+        Record leaf = {kLeaf, -1, 0, 0};
+        P.records[static_cast<size_t>(b) * R + c] = leaf;
+      } else {
+        const int start = cur[c] - n;
+        const ChildInfo f = kids[start];
+        WorkItem w = {b * R + c, b * N + start, n, f.node, f.token, f.r, u_final, 0};
+        const int slot = n >= 2 ? hb + __popc(heavy & below) : cap - 1 - (lb + __popc(light & below));
+        P.work[slot] = w;
+      }
     }
   }
 }
@@ -410,36 +435,56 @@ __global__ void __launch_bounds__(NT, 1) lantern_context_kernel(VerifyParams P) 
 
   const int n_heavy = P.counters->n_heavy;
   const int total = n_heavy + P.counters->n_light;
+  const int cap = P.B * N;
+  const int G = gridDim.x;
 
-  auto item_of = [&](int w) { return w < n_heavy ? P.work_heavy[w] : P.work_light[w - n_heavy]; };
-
+  // Work distribution.  Items 0..3G-1 are dealt statically (CTA x takes x, x+G, x+2G); from
+  // then on a global counter hands them out.  Thread 0 keeps a three-deep pipeline so that no
+  // global round trip sits on the critical path: while context i is processed, the rows of
+  // i+1 are in flight, the descriptor of i+2 is being loaded and the index of i+3 is being
+  // fetched from the counter.
+  auto load_item = [&](int w) -> WorkItem {
+    WorkItem it;
+    it.item = -1;
+    if (w < total) {
+      const int slot = w < n_heavy ? w : cap - 1 - (w - n_heavy);
+      const int4 lo = __ldg(reinterpret_cast<const int4*>(P.work + slot));
+      const int4 hi = __ldg(reinterpret_cast<const int4*>(P.work + slot) + 1);
+      it.item = lo.x, it.cbase = lo.y, it.nchild = lo.z, it.node0 = lo.w;
+      it.tok0 = hi.x, it.r0 = __int_as_float(hi.y), it.u_final = __int_as_float(hi.z), it.pad = 0;
+    }
+    return it;
+  };
+  __shared__ WorkItem s_work[2];
+  WorkItem it_next;            // thread 0: descriptor of the context after the current one
+  int w_next2 = 0;             // thread 0: index of the context after that
+  it_next.item = -1;
   if (tid == 0) {
     mbar_init(&bar, 1);
     fence_mbar_init();
     fence_proxy_async();
-    const int w = atomicAdd(&P.counters->work_next, 1);
-    int item = -1;
-    if (w < total) {
-      item = item_of(w);
-      issue_rows<BF16, UNC>(P, item, stage, rowbytes, &bar);
-    }
-    S.item = item;
+    const WorkItem first = load_item(blockIdx.x);
+    it_next = load_item(blockIdx.x + G);
+    w_next2 = blockIdx.x + 2 * G;
+    if (first.item >= 0) issue_rows<BF16, UNC>(P, first.item, stage, rowbytes, &bar);
+    s_work[0] = first;
   }
   __syncthreads();
   uint32_t parity = 0;
+  int slot_cur = 0;
 
   for (;;) {
-    const int item = S.item;
+    const WorkItem cur = s_work[slot_cur];
+    const int item = cur.item;
     if (item < 0) break;
-    const int b = item / R, c = item - b * R;
-    const int32_t* cstart = P.child_start + static_cast<size_t>(b) * (R + 1);
-    const int cs_ = cstart[c], ce_ = cstart[c + 1];
-    const int32_t* cnodes = P.child_nodes + static_cast<size_t>(b) * N;
-    const int32_t* toks = P.tokens + static_cast<size_t>(b) * N;
+    const int b = item / R;
+    const ChildInfo* kids = P.children + cur.cbase;
+    const int cs_ = 0, ce_ = cur.nchild;
 
     // first child's neighbour row: issued before the wait so its latency hides behind it
-    int node = cnodes[cs_];
-    int xt = toks[node];
+    int node = cur.node0;
+    int xt = cur.tok0;
+    float r = cur.r0;
     int nreg = (tid + 1 < k) ? __ldg(P.nbr + static_cast<size_t>(xt) * k + tid + 1) : -1;
 
     // every thread must take the same branch: agree on whether the rows have landed
@@ -466,16 +511,16 @@ __global__ void __launch_bounds__(NT, 1) lantern_context_kernel(VerifyParams P) 
     }
     block_max2(mq, mp, S, lane, warp);   // barrier inside: every thread has drained the staging rows
 
-    // staging is free: hand out the next context and start its copy
+    // staging is free: start the copy of the next context's rows, publish its descriptor for the
+    // next iteration, and move the look-ahead pipeline one step
     if (tid == 0) {
-      const int w = atomicAdd(&P.counters->work_next, 1);
-      int nxt = -1;
-      if (w < total) {
-        nxt = item_of(w);
+      if (it_next.item >= 0) {
         fence_proxy_async();
-        issue_rows<BF16, UNC>(P, nxt, stage, rowbytes, &bar);
+        issue_rows<BF16, UNC>(P, it_next.item, stage, rowbytes, &bar);
       }
-      S.item = nxt;   // read at the top of the next iteration, after many barriers
+      s_work[slot_cur ^ 1] = it_next;
+      it_next = load_item(w_next2);
+      w_next2 = 3 * G + atomicAdd(&P.counters->work_next, 1);
     }
 
     // softmax numerators and their totals
@@ -519,8 +564,13 @@ __global__ void __launch_bounds__(NT, 1) lantern_context_kernel(VerifyParams P) 
       const double delta = static_cast<double>(P.delta);
 
       for (int ci = cs_; ci < ce_; ++ci) {
-        const float r = P.uniforms[static_cast<size_t>(b) * R + node];
         const int32_t* nrow = P.nbr + static_cast<size_t>(xt) * k;
+        // the next sibling's description, wanted only after a rejection: in flight meanwhile
+        ChildInfo sib = {0, 0, 0.0f, 0};
+        if (ci + 1 < ce_) {
+          const int4 v = __ldg(reinterpret_cast<const int4*>(kids + ci + 1));
+          sib.node = v.x, sib.token = v.y, sib.r = __int_as_float(v.z);
+        }
         const float e_xt = E[phys(xt)];   // read while E is stable (before any flagging below)
         // owner of x~ publishes its drafter numerator
         {
@@ -612,8 +662,9 @@ __global__ void __launch_bounds__(NT, 1) lantern_context_kernel(VerifyParams P) 
         }
         const bool last = (ci + 1 == ce_);
         if (!last) {   // next sibling's neighbour row, in flight during the residual pass
-          node = cnodes[ci + 1];
-          xt = toks[node];
+          node = sib.node;
+          xt = sib.token;
+          r = sib.r;
           nreg = (tid + 1 < k) ? __ldg(P.nbr + static_cast<size_t>(xt) * k + tid + 1) : -1;
         }
         __syncthreads();
@@ -644,8 +695,7 @@ __global__ void __launch_bounds__(NT, 1) lantern_context_kernel(VerifyParams P) 
           break;
         }
         if (last) {
-          const double u = static_cast<double>(P.uniforms[static_cast<size_t>(b) * R + N]);
-          token = block_draw<CH>(a, cs, excl, u * W, V, S, tid);
+          token = block_draw<CH>(a, cs, excl, static_cast<double>(cur.u_final) * W, V, S, tid);
         } else {
 #pragma unroll
           for (int cc = 0; cc < CH; ++cc) {
@@ -671,6 +721,7 @@ __global__ void __launch_bounds__(NT, 1) lantern_context_kernel(VerifyParams P) 
       Record rec = {accepted, token, status, 0};
       P.records[item] = rec;
     }
+    slot_cur ^= 1;
   }
 }
 
@@ -684,16 +735,15 @@ __global__ void __launch_bounds__(128) lantern_walk_kernel(VerifyParams P) {
   int status = P.seq_status[b];
   int len = 0, next = -1;
   if (status == 0) {
-    const int32_t* cstart = P.child_start + static_cast<size_t>(b) * (R + 1);
     int cur = 0;
     for (int step = 0; step <= N; ++step) {
-      if (cstart[cur + 1] == cstart[cur]) {   // no drafts left on this path: bonus token from q
+      const Record rec = P.records[static_cast<size_t>(b) * R + cur];
+      if (rec.accepted == kLeaf) {   // no drafts left on this path: bonus token from q
         const int slot = atomicAdd(&P.counters->n_bonus, 1);
         P.bonus_seq[slot] = b;
         P.bonus_ctx[slot] = cur;
         break;
       }
-      const Record rec = P.records[static_cast<size_t>(b) * R + cur];
       status |= rec.status;
       if (rec.status & (LANTERN_ST_NONFINITE | LANTERN_ST_DEGENERATE | LANTERN_ST_INTERNAL)) break;
       if (rec.accepted >= 0) {
@@ -809,7 +859,7 @@ __global__ void __launch_bounds__(NT, 1) lantern_bonus_kernel(VerifyParams P) {
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WsLayout {
-  size_t counters, heavy, light, cstart, cnodes, records, seqst, bseq, bctx, total;
+  size_t counters, work, children, records, seqst, bseq, bctx, total;
 };
 
 static WsLayout ws_layout(int B, int N) {
@@ -817,10 +867,8 @@ static WsLayout ws_layout(int B, int N) {
   WsLayout L;
   size_t o = 0;
   L.counters = o; o += 256;
-  L.heavy = o;    o += align_up(b * R * 4, 256);
-  L.light = o;    o += align_up(b * R * 4, 256);
-  L.cstart = o;   o += align_up(b * (R + 1) * 4, 256);
-  L.cnodes = o;   o += align_up(b * N * 4 + 4, 256);
+  L.work = o;     o += align_up(b * (N > 0 ? N : 1) * sizeof(WorkItem), 256);
+  L.children = o; o += align_up(b * (N > 0 ? N : 1) * sizeof(ChildInfo), 256);
   L.records = o;  o += align_up(b * R * sizeof(Record), 256);
   L.seqst = o;    o += align_up(b * 4, 256);
   L.bseq = o;     o += align_up(b * 4, 256);
@@ -912,10 +960,8 @@ extern "C" lantern_status lantern_verify(const void* target_logits, const void* 
   P.out_px = out_node_px;
   P.out_m = out_node_m;
   P.counters = reinterpret_cast<Counters*>(ws + L.counters);
-  P.work_heavy = reinterpret_cast<int32_t*>(ws + L.heavy);
-  P.work_light = reinterpret_cast<int32_t*>(ws + L.light);
-  P.child_start = reinterpret_cast<int32_t*>(ws + L.cstart);
-  P.child_nodes = reinterpret_cast<int32_t*>(ws + L.cnodes);
+  P.work = reinterpret_cast<WorkItem*>(ws + L.work);
+  P.children = reinterpret_cast<ChildInfo*>(ws + L.children);
   P.records = reinterpret_cast<Record*>(ws + L.records);
   P.seq_status = reinterpret_cast<int32_t*>(ws + L.seqst);
   P.bonus_seq = reinterpret_cast<int32_t*>(ws + L.bseq);
@@ -935,11 +981,11 @@ extern "C" lantern_status lantern_verify(const void* target_logits, const void* 
   if (sms < 1) return LANTERN_E_CUDA;
 
   if (cudaMemsetAsync(P.counters, 0, 256, st) != cudaSuccess) return LANTERN_E_CUDA;
-  const size_t plan_smem = static_cast<size_t>(PLAN_WARPS) * (N + 2) * sizeof(int);
+  const size_t plan_smem = static_cast<size_t>(PLAN_WARPS) * 2 * (N + 2) * sizeof(int);
   lantern_plan_kernel<<<(B + PLAN_WARPS - 1) / PLAN_WARPS, PLAN_WARPS * 32, plan_smem, st>>>(P);
   if (cudaGetLastError() != cudaSuccess) return LANTERN_E_CUDA;
 
-  const long long items = static_cast<long long>(B) * (N + 1);
+  const long long items = static_cast<long long>(B) * (N > 0 ? N : 1);   // upper bound of contexts with children
   const int grid_ctx = static_cast<int>(items < sms ? items : sms);
   const int grid_bonus = B < sms ? B : sms;
   cudaError_t e;

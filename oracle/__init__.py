@@ -104,6 +104,7 @@ class VerifyResult:
     margin: np.ndarray          # [B, N] float64: distance of the node's decisions to flipping
     w: np.ndarray               # [B] float64: total weight of the last residual
     draw_margin: np.ndarray     # [B] float64
+    qa_mag: np.ndarray          # [B, N] float64: magnitude of the terms qa was formed from (>= qa)
 
 
 def verify(target_logits: np.ndarray, draft_logits: np.ndarray, dtype: int, cfg_scale: float, has_uncond: int,
@@ -129,12 +130,12 @@ def verify(target_logits: np.ndarray, draft_logits: np.ndarray, dtype: int, cfg_
         accept_path=np.full((B, N), -1, np.int32), status=np.zeros(B, np.int32),
         tested=np.zeros((B, N), np.uint8), qa=np.zeros((B, N)), px=np.zeros((B, N)),
         m=np.full((B, N), -1, np.int32), margin=np.full((B, N), np.inf), w=np.zeros(B),
-        draw_margin=np.full(B, np.inf))
+        draw_margin=np.full(B, np.inf), qa_mag=np.zeros((B, N)))
     rc = _load().oracle_verify(
         _p(tl), _p(dl), int(dtype), ctypes.c_float(cfg_scale), int(has_uncond), ctypes.c_float(T), _p(tok),
         _p(par), _p(nb), int(k), ctypes.c_float(delta), _p(un), B, N, V, _p(res.accept_len),
         _p(res.next_token), _p(res.accept_path), _p(res.status), _p(res.tested), _p(res.qa), _p(res.px),
-        _p(res.m), _p(res.margin), _p(res.w), _p(res.draw_margin))
+        _p(res.m), _p(res.margin), _p(res.w), _p(res.draw_margin), _p(res.qa_mag))
     if rc != 0:
         raise ValueError(f"oracle_verify: bad arguments ({rc})")
     return res

@@ -274,6 +274,10 @@ int oracle_a_set(const double* q, int V, const int32_t* nbr_row, int k, double d
 //   tr_px      current drafter probability of x~
 //   tr_m       |A_{k,delta}(x~)| - 1
 //   tr_margin  min(|r - qa/px|, cut margin)      (distance of the node's decisions to flipping)
+//   tr_qa_mag  magnitude of the terms qa was formed from: equal to qa for the first child of a
+//              context; after sibling rejections the target is a difference (q' - p')/W, and this
+//              is the sum over A of the minuend-plus-subtrahend magnitudes carried through the
+//              rounds.  A diagnostic for setting a floating-point tolerance, not part of the method.
 // per sequence [B]:
 //   tr_w       total weight of the last residual (0 if none)
 //   tr_draw_margin  margin of the final inverse-CDF draw
@@ -284,7 +288,7 @@ int oracle_verify(const void* target_logits, const void* draft_logits, int dtype
                   const int32_t* neighbor_idx, int k, float delta_f, const float* uniforms, int B, int N,
                   int V, int32_t* out_accept_len, int32_t* out_next_token, int32_t* out_accept_path,
                   int32_t* out_status, uint8_t* tr_tested, double* tr_qa, double* tr_px, int32_t* tr_m,
-                  double* tr_margin, double* tr_w, double* tr_draw_margin) {
+                  double* tr_margin, double* tr_w, double* tr_draw_margin, double* tr_qa_mag) {
   if (B < 0 || N < 0 || V < 1 || k < 1 || k > V) return -2;
   if (!(T > 0.0f) || !(delta_f >= 0.0f)) return -3;
   if (B == 0) return 0;
@@ -298,7 +302,7 @@ int oracle_verify(const void* target_logits, const void* draft_logits, int dtype
   const size_t branch = static_cast<size_t>(B) * R * rowsz;  // elements per guidance branch
 
   std::vector<float> z(V);
-  std::vector<double> q, p, w(V);
+  std::vector<double> q, p, w(V), mag(V);
   std::vector<std::vector<int>> kids(R);
 
   for (int b = 0; b < B; ++b) {
@@ -312,6 +316,7 @@ int oracle_verify(const void* target_logits, const void* draft_logits, int dtype
       if (tr_px) tr_px[o] = 0.0;
       if (tr_m) tr_m[o] = -1;
       if (tr_margin) tr_margin[o] = std::numeric_limits<double>::infinity();
+      if (tr_qa_mag) tr_qa_mag[o] = 0.0;
     }
     if (tr_w) tr_w[b] = 0.0;
     if (tr_draw_margin) tr_draw_margin[b] = std::numeric_limits<double>::infinity();
@@ -368,6 +373,7 @@ int oracle_verify(const void* target_logits, const void* draft_logits, int dtype
 
       int accepted = -1;
       bool degenerate = false;
+      if (tr_qa_mag) mag.assign(q.begin(), q.end());
       for (int c : kids[cur]) {
         const int32_t xt = draft_tokens[static_cast<size_t>(b) * N + c];
         const double r = uniforms[static_cast<size_t>(b) * R + c];
@@ -384,6 +390,12 @@ int oracle_verify(const void* target_logits, const void* draft_logits, int dtype
         if (tr_qa) tr_qa[o] = qa;
         if (tr_px) tr_px[o] = px;
         if (tr_m) tr_m[o] = m;
+        if (tr_qa_mag) {
+          double g = mag[xt];
+          for (int j = 1; j <= m; ++j)
+            if (nrow[j] >= 0 && nrow[j] < V) g += mag[nrow[j]];
+          tr_qa_mag[o] = g;
+        }
         if (tr_margin) {
           double am = px > 0.0 ? std::fabs(r - qa / px) : std::numeric_limits<double>::infinity();
           tr_margin[o] = std::min(am, k > 1 ? cut_margin : std::numeric_limits<double>::infinity());
@@ -413,6 +425,8 @@ int oracle_verify(const void* target_logits, const void* draft_logits, int dtype
           degenerate = true;
           break;
         }
+        if (tr_qa_mag)
+          for (int x = 0; x < V; ++x) mag[x] = w[x] > 0.0 ? (mag[x] + p[x]) / W : 0.0;
         for (int x = 0; x < V; ++x) q[x] = w[x] / W;
         // R6: the rejected token leaves the drafter distribution
         p[xt] = 0.0;

@@ -238,82 +238,6 @@ __device__ __forceinline__ int block_draw(const float (&w)[CH * 8], const double
   return S.tok;
 }
 
-// Read one context's rows from shared-memory staging into registers as processed logits.
-template <int CH, bool BF16, bool UNC, bool WITH_DRAFT>
-__device__ __forceinline__ void load_rows(const unsigned char* stage, int rowbytes, int V, float s, float T,
-                                          float (&zq)[CH * 8], float (&zp)[CH * 8], int tid) {
-  const unsigned char* rc = stage;
-  const unsigned char* ru = stage + rowbytes;
-  const unsigned char* rd = stage + (UNC ? 2 : 1) * rowbytes;
-  const float ninf = __int_as_float(0xff800000);
-#pragma unroll
-  for (int c = 0; c < CH; ++c) {
-    const int g = c * NT + tid;
-    if (g * 8 < V) {
-      float lc[8], lu[8], ld[8];
-      if (BF16) {
-        const uint4 a = *reinterpret_cast<const uint4*>(rc + g * 16);
-        const uint32_t aw[4] = {a.x, a.y, a.z, a.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          lc[2 * i] = __uint_as_float(aw[i] << 16);
-          lc[2 * i + 1] = __uint_as_float(aw[i] & 0xffff0000u);
-        }
-        if (UNC) {
-          const uint4 b = *reinterpret_cast<const uint4*>(ru + g * 16);
-          const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            lu[2 * i] = __uint_as_float(bw[i] << 16);
-            lu[2 * i + 1] = __uint_as_float(bw[i] & 0xffff0000u);
-          }
-        }
-        if (WITH_DRAFT) {
-          const uint4 d = *reinterpret_cast<const uint4*>(rd + g * 16);
-          const uint32_t dw[4] = {d.x, d.y, d.z, d.w};
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            ld[2 * i] = __uint_as_float(dw[i] << 16);
-            ld[2 * i + 1] = __uint_as_float(dw[i] & 0xffff0000u);
-          }
-        }
-      } else {
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const float4 a = *reinterpret_cast<const float4*>(rc + g * 32 + h * 16);
-          lc[4 * h] = a.x, lc[4 * h + 1] = a.y, lc[4 * h + 2] = a.z, lc[4 * h + 3] = a.w;
-          if (UNC) {
-            const float4 b = *reinterpret_cast<const float4*>(ru + g * 32 + h * 16);
-            lu[4 * h] = b.x, lu[4 * h + 1] = b.y, lu[4 * h + 2] = b.z, lu[4 * h + 3] = b.w;
-          }
-          if (WITH_DRAFT) {
-            const float4 d = *reinterpret_cast<const float4*>(rd + g * 32 + h * 16);
-            ld[4 * h] = d.x, ld[4 * h + 1] = d.y, ld[4 * h + 2] = d.z, ld[4 * h + 3] = d.w;
-          }
-        }
-      }
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        float l = lc[e];
-        if (UNC) l = __fmaf_rn(s, __fsub_rn(lc[e], lu[e]), lu[e]);   // l_u + s (l_c - l_u)
-        float d = WITH_DRAFT ? ld[e] : 0.0f;
-        if (T != 1.0f) {
-          l = __fdiv_rn(l, T);
-          d = __fdiv_rn(d, T);
-        }
-        zq[c * 8 + e] = l;
-        zp[c * 8 + e] = d;
-      }
-    } else {
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        zq[c * 8 + e] = ninf;
-        zp[c * 8 + e] = ninf;
-      }
-    }
-  }
-}
-
 // ---------------------------------------------------------------------------------------
 // kernel 1: plan.  One warp per sequence: validate tokens / parents / uniforms, bucket the
 // nodes by parent context (children in node order), initialise the per-node outputs, mark
@@ -399,331 +323,12 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
   }
 }
 
-// ---------------------------------------------------------------------------------------
-// kernel 2: fused context pass (see the header of this file).
-// ---------------------------------------------------------------------------------------
-template <bool BF16, bool UNC>
-__device__ __forceinline__ void issue_rows(const VerifyParams& P, int item, unsigned char* stage, int rowbytes,
-                                           uint64_t* bar) {
-  const int nrows = UNC ? 3 : 2;
-  mbar_expect_tx(bar, static_cast<uint32_t>(nrows * rowbytes));
-  const size_t row_off = static_cast<size_t>(item) * rowbytes;
-  const size_t branch = static_cast<size_t>(P.B) * P.R * rowbytes;
-  const unsigned char* src[3];
-  src[0] = static_cast<const unsigned char*>(P.target) + row_off;
-  src[1] = UNC ? static_cast<const unsigned char*>(P.target) + branch + row_off
-               : static_cast<const unsigned char*>(P.draft) + row_off;
-  src[2] = static_cast<const unsigned char*>(P.draft) + row_off;
-  for (int r = 0; r < nrows; ++r)
-    for (int off = 0; off < rowbytes; off += 16384) {
-      const int n = min(16384, rowbytes - off);
-      bulk_load(stage + r * rowbytes + off, src[r] + off, static_cast<uint32_t>(n), bar);
-    }
-}
+}  // namespace lantern
 
-template <int CH, bool BF16, bool UNC>
-__global__ void __launch_bounds__(NT, 1) lantern_context_kernel(VerifyParams P) {
-  extern __shared__ __align__(128) unsigned char smem[];
-  __shared__ BlockScratch S;
-  __shared__ __align__(8) uint64_t bar;
+// kernel 2: the fused context pass
+#include "verify_context.cuh"
 
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int V = P.V, N = P.N, R = P.R, k = P.k;
-  const int rowbytes = V * (BF16 ? 2 : 4);
-  unsigned char* stage = smem;
-  float* E = reinterpret_cast<float*>(smem + (UNC ? 3 : 2) * rowbytes);
-
-  const int n_heavy = P.counters->n_heavy;
-  const int total = n_heavy + P.counters->n_light;
-  const int cap = P.B * N;
-  const int G = gridDim.x;
-
-  // Work distribution.  Items 0..3G-1 are dealt statically (CTA x takes x, x+G, x+2G); from
-  // then on a global counter hands them out.  Thread 0 keeps a three-deep pipeline so that no
-  // global round trip sits on the critical path: while context i is processed, the rows of
-  // i+1 are in flight, the descriptor of i+2 is being loaded and the index of i+3 is being
-  // fetched from the counter.
-  auto load_item = [&](int w) -> WorkItem {
-    WorkItem it;
-    it.item = -1;
-    if (w < total) {
-      const int slot = w < n_heavy ? w : cap - 1 - (w - n_heavy);
-      const int4 lo = __ldg(reinterpret_cast<const int4*>(P.work + slot));
-      const int4 hi = __ldg(reinterpret_cast<const int4*>(P.work + slot) + 1);
-      it.item = lo.x, it.cbase = lo.y, it.nchild = lo.z, it.node0 = lo.w;
-      it.tok0 = hi.x, it.r0 = __int_as_float(hi.y), it.u_final = __int_as_float(hi.z), it.pad = 0;
-    }
-    return it;
-  };
-  __shared__ WorkItem s_work[2];
-  WorkItem it_next;            // thread 0: descriptor of the context after the current one
-  int w_next2 = 0;             // thread 0: index of the context after that
-  it_next.item = -1;
-  if (tid == 0) {
-    mbar_init(&bar, 1);
-    fence_mbar_init();
-    fence_proxy_async();
-    const WorkItem first = load_item(blockIdx.x);
-    it_next = load_item(blockIdx.x + G);
-    w_next2 = blockIdx.x + 2 * G;
-    if (first.item >= 0) issue_rows<BF16, UNC>(P, first.item, stage, rowbytes, &bar);
-    s_work[0] = first;
-  }
-  __syncthreads();
-  uint32_t parity = 0;
-  int slot_cur = 0;
-
-  for (;;) {
-    const WorkItem cur = s_work[slot_cur];
-    const int item = cur.item;
-    if (item < 0) break;
-    const int b = item / R;
-    const ChildInfo* kids = P.children + cur.cbase;
-    const int cs_ = 0, ce_ = cur.nchild;
-
-    // first child's neighbour row: issued before the wait so its latency hides behind it
-    int node = cur.node0;
-    int xt = cur.tok0;
-    float r = cur.r0;
-    int nreg = (tid + 1 < k) ? __ldg(P.nbr + static_cast<size_t>(xt) * k + tid + 1) : -1;
-
-    // every thread must take the same branch: agree on whether the rows have landed
-    const bool arrived = __syncthreads_and(mbar_wait(&bar, parity)) != 0;
-    if (!arrived) {
-      // The copy did not land within the limit: report it, give the copy in flight one more
-      // bounded chance to finish before this CTA's shared memory is released, and stop.
-      if (tid == 0) {
-        Record rec = {-1, -1, LANTERN_ST_INTERNAL, 0};
-        P.records[item] = rec;
-      }
-      mbar_wait(&bar, parity);
-      break;
-    }
-    parity ^= 1u;
-
-    float a[CH * 8], ep[CH * 8];
-    load_rows<CH, BF16, UNC, true>(stage, rowbytes, V, P.cfg_scale, P.T, a, ep, tid);
-    float mq = a[0], mp = ep[0];
-#pragma unroll
-    for (int i = 1; i < CH * 8; ++i) {
-      mq = fmaxf(mq, a[i]);
-      mp = fmaxf(mp, ep[i]);
-    }
-    block_max2(mq, mp, S, lane, warp);   // barrier inside: every thread has drained the staging rows
-
-    // staging is free: start the copy of the next context's rows, publish its descriptor for the
-    // next iteration, and move the look-ahead pipeline one step
-    if (tid == 0) {
-      if (it_next.item >= 0) {
-        fence_proxy_async();
-        issue_rows<BF16, UNC>(P, it_next.item, stage, rowbytes, &bar);
-      }
-      s_work[slot_cur ^ 1] = it_next;
-      it_next = load_item(w_next2);
-      w_next2 = 3 * G + atomicAdd(&P.counters->work_next, 1);
-    }
-
-    // softmax numerators and their totals
-    double zq_sum, zp_sum;
-    {
-      float pq[CH], pp[CH];
-#pragma unroll
-      for (int cc = 0; cc < CH; ++cc) {
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          a[cc * 8 + e] = exp_nonpos(a[cc * 8 + e] - mq);
-          ep[cc * 8 + e] = exp_nonpos(ep[cc * 8 + e] - mp);
-        }
-        pq[cc] = sum8(&a[cc * 8]);
-        pp[cc] = sum8(&ep[cc * 8]);
-        const int g = cc * NT + tid;
-        if (g * 8 < V) {
-          float4* dst = reinterpret_cast<float4*>(E);
-          dst[(((cc << 1) | 0) << LOG_NT) + tid] = make_float4(a[cc * 8], a[cc * 8 + 1], a[cc * 8 + 2], a[cc * 8 + 3]);
-          dst[(((cc << 1) | 1) << LOG_NT) + tid] =
-              make_float4(a[cc * 8 + 4], a[cc * 8 + 5], a[cc * 8 + 6], a[cc * 8 + 7]);
-        }
-      }
-      zq_sum = pq[0];
-      zp_sum = pp[0];
-#pragma unroll
-      for (int cc = 1; cc < CH; ++cc) {
-        zq_sum += pq[cc];
-        zp_sum += pp[cc];
-      }
-    }
-    block_sum2(zq_sum, zp_sum, S, lane, warp);   // barriers inside also publish E
-
-    int status = 0;
-    int accepted = -1, token = -1;
-    if (!(zq_sum > 0.0 && zq_sum < 1e300 && zp_sum > 0.0 && zp_sum < 1e300)) {
-      status |= LANTERN_ST_NONFINITE;
-    } else {
-      double qscale = 1.0 / zq_sum;     // q'(x) = E(x) * qscale
-      double pscale = 1.0 / zp_sum;     // p'(x) = ep(x) * pscale
-      const double delta = static_cast<double>(P.delta);
-
-      for (int ci = cs_; ci < ce_; ++ci) {
-        const int32_t* nrow = P.nbr + static_cast<size_t>(xt) * k;
-        // the next sibling's description, wanted only after a rejection: in flight meanwhile
-        ChildInfo sib = {0, 0, 0.0f, 0};
-        if (ci + 1 < ce_) {
-          const int4 v = __ldg(reinterpret_cast<const int4*>(kids + ci + 1));
-          sib.node = v.x, sib.token = v.y, sib.r = __int_as_float(v.z);
-        }
-        const float e_xt = E[phys(xt)];   // read while E is stable (before any flagging below)
-        // owner of x~ publishes its drafter numerator
-        {
-          const int g = xt >> 3;
-          if ((g & (NT - 1)) == tid) {
-            const int li = ((g >> LOG_NT) << 3) | (xt & 7);
-            float v = 0.0f;
-#pragma unroll
-            for (int i = 0; i < CH * 8; ++i)
-              if (i == li) v = ep[i];
-            S.px = v;
-          }
-        }
-        // ---- A_{k,delta}(x~): gather + prefix scan with the strict bound ----
-        const double thr = delta * (1.0 / qscale);   // compare unnormalised sums
-        double carry = 0.0, sm = 0.0;
-        int m = k - 1;
-        bool cut = false;
-        for (int base = 0; base < k - 1 && !cut; base += NT) {
-          const int j = base + tid + 1;
-          const bool valid = j < k;
-          const int n = (base == 0) ? nreg : (valid ? __ldg(nrow + j) : -1);
-          float v = 0.0f;
-          if (valid) {
-            if (static_cast<unsigned>(n) < static_cast<unsigned>(V)) v = E[phys(n)];
-            else status |= LANTERN_ST_BAD_TABLE;
-          }
-          const double incl = warp_incl_scan(static_cast<double>(v), lane);
-          if (lane == 31) S.wt[warp] = incl;
-          if (tid == 0) S.first = 0x7fffffff;
-          __syncthreads();
-          if (warp == 0) {
-            const double t = S.wt[lane];
-            const double in = warp_incl_scan(t, lane);
-            S.wbase[lane] = in - t;
-            if (lane == 31) S.total = in;
-          }
-          __syncthreads();
-          const double Sj = carry + S.wbase[warp] + incl;
-          const bool fail = valid && !(Sj < thr);
-          const unsigned bal = __ballot_sync(kFull, fail);
-          if (bal && lane == __ffs(bal) - 1) atomicMin(&S.first, j);
-          __syncthreads();
-          const int first = S.first;
-          if (first != 0x7fffffff) {
-            m = first - 1;
-            if (j == m) S.sm = Sj;
-            __syncthreads();
-            sm = (m == base) ? carry : S.sm;
-            cut = true;
-          } else {
-            carry += S.total;
-            sm = carry;
-            __syncthreads();
-          }
-        }
-        if (k == 1) __syncthreads();   // publish S.px when the scan loop did not run
-        const double qa = (static_cast<double>(e_xt) + sm) * qscale;
-        const double px = static_cast<double>(S.px) * pscale;
-        const bool accept = static_cast<double>(r) * px < qa;   // Section 4.3: min(1, sum_A q / p(x~))
-        if (tid == 0) {
-          const size_t o = static_cast<size_t>(b) * N + node;
-          if (P.out_qa) P.out_qa[o] = static_cast<float>(qa);
-          if (P.out_px) P.out_px[o] = static_cast<float>(px);
-          if (P.out_m) P.out_m[o] = m;
-        }
-        if (accept) {
-          accepted = node;
-          break;
-        }
-        // ---- rejected: residual [q_{k,delta}(.|D = x~) - p]_+ ----
-        // members of A (x~ included) leave no residual mass: flag them with a negative sign
-        for (int j = tid + 1; j <= m; j += NT) {
-          const int n = (j <= NT) ? nreg : __ldg(nrow + j);
-          if (static_cast<unsigned>(n) < static_cast<unsigned>(V)) {
-            const int q_ = phys(n);
-            E[q_] = -fabsf(E[q_]);
-          }
-        }
-        if (tid == 0) E[phys(xt)] = -fabsf(E[phys(xt)]);
-        {   // x~ leaves the drafter distribution for the following siblings
-          const int g = xt >> 3;
-          if ((g & (NT - 1)) == tid) {
-            const int li = ((g >> LOG_NT) << 3) | (xt & 7);
-#pragma unroll
-            for (int i = 0; i < CH * 8; ++i)
-              if (i == li) ep[i] = 0.0f;
-          }
-        }
-        const bool last = (ci + 1 == ce_);
-        if (!last) {   // next sibling's neighbour row, in flight during the residual pass
-          node = sib.node;
-          xt = sib.token;
-          r = sib.r;
-          nreg = (tid + 1 < k) ? __ldg(P.nbr + static_cast<size_t>(xt) * k + tid + 1) : -1;
-        }
-        __syncthreads();
-        const float ratio = static_cast<float>(pscale / qscale);   // w = E - ratio * ep, in units of E
-        double cs[CH], excl[CH];
-        float psum = 0.0f;
-#pragma unroll
-        for (int cc = 0; cc < CH; ++cc) {
-          const int g = cc * NT + tid;
-          if (g * 8 < V) {
-            const float4* src = reinterpret_cast<const float4*>(E);
-            const float4 lo = src[(((cc << 1) | 0) << LOG_NT) + tid];
-            const float4 hi = src[(((cc << 1) | 1) << LOG_NT) + tid];
-            const float e8[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
-#pragma unroll
-            for (int e = 0; e < 8; ++e) a[cc * 8 + e] = fmaxf(0.0f, __fmaf_rn(-ratio, ep[cc * 8 + e], e8[e]));
-          } else {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) a[cc * 8 + e] = 0.0f;
-          }
-          cs[cc] = static_cast<double>(sum8(&a[cc * 8]));
-          psum += sum8(&ep[cc * 8]);
-        }
-        block_scan_chunks<CH>(cs, excl, static_cast<double>(psum), S, lane, warp);
-        const double W = S.total, Sp = S.total2;
-        if (!(W > 0.0)) {
-          status |= LANTERN_ST_DEGENERATE;
-          break;
-        }
-        if (last) {
-          token = block_draw<CH>(a, cs, excl, static_cast<double>(cur.u_final) * W, V, S, tid);
-        } else {
-#pragma unroll
-          for (int cc = 0; cc < CH; ++cc) {
-            const int g = cc * NT + tid;
-            if (g * 8 < V) {
-              float4* dst = reinterpret_cast<float4*>(E);
-              dst[(((cc << 1) | 0) << LOG_NT) + tid] =
-                  make_float4(a[cc * 8], a[cc * 8 + 1], a[cc * 8 + 2], a[cc * 8 + 3]);
-              dst[(((cc << 1) | 1) << LOG_NT) + tid] =
-                  make_float4(a[cc * 8 + 4], a[cc * 8 + 5], a[cc * 8 + 6], a[cc * 8 + 7]);
-            }
-          }
-          qscale = 1.0 / W;
-          pscale = Sp > 0.0 ? 1.0 / Sp : 0.0;
-          __syncthreads();
-        }
-      }
-    }
-    // NONFINITE / DEGENERATE are set by every thread alike; a bad table entry is seen by one thread
-    status = (status & ~LANTERN_ST_BAD_TABLE) |
-             (__syncthreads_or(status & LANTERN_ST_BAD_TABLE) ? LANTERN_ST_BAD_TABLE : 0);
-    if (tid == 0) {
-      Record rec = {accepted, token, status, 0};
-      P.records[item] = rec;
-    }
-    slot_cur ^= 1;
-  }
-}
+namespace lantern {
 
 // ---------------------------------------------------------------------------------------
 // kernel 3: walk (Algorithm 1's loop over the records; one thread per sequence)
@@ -879,21 +484,22 @@ static WsLayout ws_layout(int B, int N) {
 
 static thread_local cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
 
-template <int CH, bool BF16, bool UNC>
+template <int CHC, bool BF16, bool UNC>
 static cudaError_t launch_verify(const VerifyParams& P, int grid_ctx, int grid_bonus, size_t smem_bytes,
                                  cudaStream_t st) {
-  auto kc = lantern_context_kernel<CH, BF16, UNC>;
+  constexpr int CHB = CHC == 4 ? 2 : 1;   // the bonus kernel runs 1024 threads per row
+  auto kc = lantern_context_kernel<CHC, BF16, UNC>;
   cudaError_t e = cudaFuncSetAttribute(kc, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
   if (e != cudaSuccess) return e;
   if (g_ev_before && g_ev_after) cudaEventRecord(g_ev_before, st);
-  kc<<<grid_ctx, NT, smem_bytes, st>>>(P);
+  kc<<<grid_ctx, CNT, smem_bytes, st>>>(P);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (g_ev_before && g_ev_after) cudaEventRecord(g_ev_after, st);
   lantern_walk_kernel<<<(P.B + 127) / 128, 128, 0, st>>>(P);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  lantern_bonus_kernel<CH, BF16, UNC><<<grid_bonus, NT, 0, st>>>(P);
+  lantern_bonus_kernel<CHB, BF16, UNC><<<grid_bonus, NT, 0, st>>>(P);
   return cudaGetLastError();
 }
 
@@ -931,8 +537,8 @@ extern "C" lantern_status lantern_verify(const void* target_logits, const void* 
   if (T == 0.0f) return LANTERN_E_UNIMPLEMENTED;   // greedy decoding is not part of this build
   const int esize = dtype == LANTERN_BF16 ? 2 : 4;
   const int nrows = has_uncond ? 3 : 2;
-  const int CH = V > NT * 8 ? 2 : 1;
-  const size_t smem_bytes = static_cast<size_t>(nrows) * V * esize + static_cast<size_t>(CH) * NT * 8 * 4;
+  const int CH = V > 2 * CNT * 8 ? 4 : (V > CNT * 8 ? 2 : 1);   // 8-token chunks per thread of the fused kernel
+  const size_t smem_bytes = static_cast<size_t>(nrows) * V * esize + static_cast<size_t>(CH) * CNT * 8 * 4;
   if (smem_bytes > 220 * 1024) return LANTERN_E_SHAPE;
   if (B == 0) return LANTERN_OK;
   if (!target_logits || !neighbor_idx || !uniforms || !out_accept_len || !out_next_token) return LANTERN_E_NULL;
@@ -995,7 +601,7 @@ extern "C" lantern_status lantern_verify(const void* target_logits, const void* 
             : launch_verify<CHV, true, false>(P, grid_ctx, grid_bonus, smem_bytes, st))              \
       : (un ? launch_verify<CHV, false, true>(P, grid_ctx, grid_bonus, smem_bytes, st)               \
             : launch_verify<CHV, false, false>(P, grid_ctx, grid_bonus, smem_bytes, st)))
-  e = CH == 2 ? LANTERN_DISPATCH(2) : LANTERN_DISPATCH(1);
+  e = CH == 4 ? LANTERN_DISPATCH(4) : (CH == 2 ? LANTERN_DISPATCH(2) : LANTERN_DISPATCH(1));
 #undef LANTERN_DISPATCH
   return e == cudaSuccess ? LANTERN_OK : LANTERN_E_CUDA;
 }

@@ -5,7 +5,11 @@ in which some decision of the oracle lies within WINDOW of its threshold (the ac
 |r - sum_A q / p(x~)|, the prefix cut |moved mass - delta|, or the final draw's distance to a
 CDF edge).  Such a sequence is counted as "near" and must reproduce exactly under the oracle
 once the corresponding input (that node's uniform, delta, or the final uniform) is nudged
-across the window.  Probabilities must agree to REL.
+across the window.  Probabilities must agree to REL: p(x~) relative to itself; sum_A q relative
+to the magnitude of the terms it was formed from -- for the first child of a context that is
+sum_A q itself, after sibling rejections the target is a difference (q' - p') / W evaluated in
+fp32, whose rounding error scales with q' + p', not with the difference (the oracle reports
+that magnitude as qa_mag).
 """
 from __future__ import annotations
 
@@ -107,7 +111,7 @@ def compare(inp: li.VerifyInputs, table: np.ndarray, delta: float, gpu: lt.Verif
         # (which it must, away from the window).
         res["m_mismatch_outside"] = int((m[far] != ora.m[far]).sum())
         agree = t & (m == ora.m)
-        rel_qa = np.abs(qa[agree] - ora.qa[agree]) / np.maximum(ora.qa[agree], 1e-30)
+        rel_qa = np.abs(qa[agree] - ora.qa[agree]) / np.maximum(ora.qa_mag[agree], 1e-30)
         rel_px = np.abs(px[t] - ora.px[t]) / np.maximum(ora.px[t], 1e-30)
         res["qa_rel_max"] = float(rel_qa.max()) if rel_qa.size else 0.0
         res["px_rel_max"] = float(rel_px.max()) if rel_px.size else 0.0

@@ -17,7 +17,8 @@ ST_BAD_TOKEN, ST_BAD_PARENT, ST_BAD_UNIFORM, ST_NONFINITE, ST_DEGENERATE, ST_BAD
     1, 2, 4, 8, 16, 32, 64
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "liblantern.so")
+# LANTERN_LIBRARY may point at another build of the same library (e.g. an instrumented one)
+_LIB_PATH = os.environ.get("LANTERN_LIBRARY", os.path.join(_HERE, "liblantern.so"))
 _lib = None
 
 

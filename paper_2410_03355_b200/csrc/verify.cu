@@ -492,7 +492,7 @@ static cudaError_t launch_verify(const VerifyParams& P, int grid_ctx, int grid_b
   cudaError_t e = cudaFuncSetAttribute(kc, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
   if (e != cudaSuccess) return e;
   if (g_ev_before && g_ev_after) cudaEventRecord(g_ev_before, st);
-  kc<<<grid_ctx, CNT, smem_bytes, st>>>(P);
+  kc<<<grid_ctx, CTX_THREADS, smem_bytes, st>>>(P);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (g_ev_before && g_ev_after) cudaEventRecord(g_ev_after, st);
@@ -538,7 +538,9 @@ extern "C" lantern_status lantern_verify(const void* target_logits, const void* 
   const int esize = dtype == LANTERN_BF16 ? 2 : 4;
   const int nrows = has_uncond ? 3 : 2;
   const int CH = V > 2 * CNT * 8 ? 4 : (V > CNT * 8 ? 2 : 1);   // 8-token chunks per thread of the fused kernel
-  const size_t smem_bytes = static_cast<size_t>(nrows) * V * esize + static_cast<size_t>(CH) * CNT * 8 * 4;
+  // two staging areas of (C+1) rows each; the numerators are kept over the rows they came from
+  const size_t smem_bytes = 2 * ((static_cast<size_t>(3) * V * esize + 127) & ~static_cast<size_t>(127));
+  (void)nrows;
   if (smem_bytes > 220 * 1024) return LANTERN_E_SHAPE;
   if (B == 0) return LANTERN_OK;
   if (!target_logits || !neighbor_idx || !uniforms || !out_accept_len || !out_next_token) return LANTERN_E_NULL;

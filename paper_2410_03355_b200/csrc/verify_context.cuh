@@ -1,9 +1,12 @@
 // Fused context pass of the LANTERN verification step (included by verify.cu).
 //
-// Persistent kernel, one CTA of 512 threads per SM.  A bulk asynchronous copy (TMA, completion
-// on an mbarrier, no multicast) brings the next context's rows into a staging area as soon as
-// every warp has drained the current rows into registers (signalled through a second
-// mbarrier, so no block-wide barrier is needed for the hand-over).
+// Persistent kernel, one CTA per SM: 16 consumer warps and one producer warp, two staging areas
+// in shared memory.  The producer hands out contexts and issues bulk asynchronous copies (TMA,
+// completion on an mbarrier, no multicast) that bring the NEXT context's rows into one area for
+// the whole time the consumers work on the current context in the other, so HBM streams
+// continuously and no consumer ever waits on a global round trip of the work queue.  The current context's softmax numerators E are stored over its
+// own raw rows once those have been read into registers: every thread overwrites only bytes
+// that it alone has read, so this needs no barrier and no third buffer.
 //
 // Each warp streams its slice of the rows on its own: guidance combine, the warp's own maximum,
 // numerators 2^((z - max_w) log2 e) through the hardware ex2 unit, partial sums.  One block
@@ -26,15 +29,15 @@ constexpr int CNW = CNT / 32;   // warps per CTA
 constexpr int LOG_CNT = 9;
 constexpr int kNone = 0x7fffffff;
 
-// thread t owns, for chunk c, the eight consecutive tokens [(c*CNT + t)*8, +8); in shared memory
-// the two 16-byte halves of a chunk live in separate planes so that 16-byte accesses of a warp are
-// bank-conflict free.  Physical float index of token x:
-__device__ __forceinline__ int cphys(int x) {
-  const int g = x >> 3;
-  const int c = g >> LOG_CNT;
-  const int t = g & (CNT - 1);
-  const int h = (x >> 2) & 1;
-  return ((((c << 1) | h) << LOG_CNT) + t) << 2 | (x & 3);
+// Thread t owns, for chunk c, the eight consecutive tokens [(c*CNT + t)*8, +8), i.e. 16-byte group
+// g = c*CNT + t of a bf16 row.  E is laid over the context's own raw rows: with bf16 logits the low
+// four numerators of group g replace group g of the first row and the high four replace group g of
+// the second row; with fp32 logits the eight numerators replace the group's own 32 bytes of the
+// first row.  Float index of token x inside the staging area:
+template <bool BF16>
+__device__ __forceinline__ int ephys(int x, int row_floats) {
+  if (BF16) return ((x >> 2) & 1) * row_floats + ((x >> 3) << 2) + (x & 3);
+  return x;
 }
 __device__ __forceinline__ int cowner_thread(int x) { return (x >> 3) & (CNT - 1); }
 
@@ -46,7 +49,6 @@ struct CtxShared {
   double hist[32];              // drafter/target scale ratio of each earlier rejection round of this context
   int acc_valid;                // acc_e / acc_p are usable for the current child
   float mlq[CNW], mlp[CNW];     // per-warp shift constants fl(max_w * log2 e)
-  float px_bulk;                // drafter numerator of x~ as held by its owner (0 once rejected), global units
   int first[CNW];               // a warp's first failing neighbour slot
   int cand[CNW];
   int tok;
@@ -58,6 +60,16 @@ __device__ __forceinline__ float ex2_approx(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+
+// 2^(z log2(e) - shift) for one value, to about 1.5e-7: the exponent is formed in double precision,
+// split into an fp32 head for the ex2 unit and a tail that is applied to first order.
+__device__ __forceinline__ double exp2_single(float z, float shift) {
+  const double x = static_cast<double>(z) * 1.4426950408889634074 - static_cast<double>(shift);
+  const float xh = static_cast<float>(x);
+  const float xl = static_cast<float>(x - static_cast<double>(xh));
+  const float y = ex2_approx(xh);
+  return static_cast<double>(__fmaf_rn(y, xl * 0.693147182464599609375f, y));
 }
 
 template <bool BF16, bool UNC>
@@ -72,11 +84,13 @@ __device__ __forceinline__ void ctx_issue_rows(const VerifyParams& P, int item, 
   src[1] = UNC ? static_cast<const unsigned char*>(P.target) + branch + row_off
                : static_cast<const unsigned char*>(P.draft) + row_off;
   src[2] = static_cast<const unsigned char*>(P.draft) + row_off;
-  for (int r = 0; r < nrows; ++r)
+  for (int r = 0; r < nrows; ++r) {
+    const int dst_row = (r == nrows - 1) ? 2 : r;   // the drafter row always goes to row slot 2
     for (int off = 0; off < rowbytes; off += 16384) {
       const int n = min(16384, rowbytes - off);
-      bulk_load(stage + r * rowbytes + off, src[r] + off, static_cast<uint32_t>(n), bar);
+      bulk_load(stage + dst_row * rowbytes + off, src[r] + off, static_cast<uint32_t>(n), bar);
     }
+  }
 }
 
 // one logit of a row in global memory, widened to fp32
@@ -86,76 +100,137 @@ __device__ __forceinline__ float ctx_raw_logit(const void* base, size_t elem) {
   return __ldg(static_cast<const float*>(base) + elem);
 }
 
+constexpr int CTX_THREADS = CNT + 32;   // 16 consumer warps and one producer warp
+
+// barrier among the 512 consumer threads only (the producer warp never joins it)
+__device__ __forceinline__ void cbar() { asm volatile("bar.sync 1, %0;" ::"n"(CNT) : "memory"); }
+// the same barrier, returning the AND of every consumer thread's predicate
+__device__ __forceinline__ bool cbar_and(bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 p, %1, 0;\n\t"
+      "bar.red.and.pred q, 1, %2, p;\n\t"
+      "selp.u32 %0, 1, 0, q;\n\t}"
+      : "=r"(r)
+      : "r"(static_cast<uint32_t>(pred)), "n"(CNT)
+      : "memory");
+  return r != 0;
+}
+// a load that stays where it is written (issued early on purpose; the value is used much later)
+__device__ __forceinline__ int ld_nc_here(const int32_t* p) {
+  int v;
+  asm volatile("ld.global.nc.s32 %0, [%1];" : "=r"(v) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+
 template <int CH, bool BF16, bool UNC>
-__global__ void __launch_bounds__(CNT, 1) lantern_context_kernel(VerifyParams P) {
+__global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyParams P) {
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ CtxShared S;
-  __shared__ __align__(8) uint64_t bar_full, bar_empty;
+  __shared__ __align__(8) uint64_t bar_full[2], bar_empty[2];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int V = P.V, N = P.N, R = P.R, k = P.k;
   const int rowbytes = V * (BF16 ? 2 : 4);
-  unsigned char* stage = smem;
-  float* E = reinterpret_cast<float*>(smem + (UNC ? 3 : 2) * rowbytes);
+  const int stage_bytes = (3 * rowbytes + 127) & ~127;   // row slots: conditional, unconditional, drafter
+  const int row_floats = rowbytes >> 2;
+  auto EI = [&](int x) { return ephys<BF16>(x, row_floats); };
   const float L_hi = 1.44269502162933349609375f;   // fl32(log2 e)
-  const double LOG2E = 1.4426950408889634074;
   const float ninf = __int_as_float(0xff800000);
 
-  const int n_heavy = P.counters->n_heavy;
-  const int total = n_heavy + P.counters->n_light;
-  const int cap = P.B * N;
-  const int G = gridDim.x;
-
-  // Work distribution.  Items 0..3G-1 are dealt statically (CTA x takes x, x+G, x+2G); from then on
-  // a global counter hands them out.  Thread 0 keeps a three-deep pipeline so that no global round
-  // trip sits on the critical path: while context i is processed, the rows of i+1 are in flight, the
-  // descriptor of i+2 is being loaded and the index of i+3 is being fetched from the counter.
-  auto load_item = [&](int w) -> WorkItem {
-    WorkItem it;
-    it.item = -1;
-    if (w < total) {
-      const int slot = w < n_heavy ? w : cap - 1 - (w - n_heavy);
-      const int4 lo = __ldg(reinterpret_cast<const int4*>(P.work + slot));
-      const int4 hi = __ldg(reinterpret_cast<const int4*>(P.work + slot) + 1);
-      it.item = lo.x, it.cbase = lo.y, it.nchild = lo.z, it.node0 = lo.w;
-      it.tok0 = hi.x, it.r0 = __int_as_float(hi.y), it.u_final = __int_as_float(hi.z), it.pad = 0;
-    }
-    return it;
-  };
-  WorkItem it_next;            // thread 0: descriptor of the context after the current one
-  int w_next2 = 0;             // thread 0: index of the context after that
-  it_next.item = -1;
   if (tid == 0) {
-    mbar_init(&bar_full, 1);
-    mbar_init(&bar_empty, CNW);
+    mbar_init(&bar_full[0], 1);
+    mbar_init(&bar_full[1], 1);
+    mbar_init(&bar_empty[0], CNW);
+    mbar_init(&bar_empty[1], CNW);
     fence_mbar_init();
     fence_proxy_async();
-    const WorkItem first = load_item(blockIdx.x);
-    it_next = load_item(blockIdx.x + G);
-    w_next2 = blockIdx.x + 2 * G;
-    if (first.item >= 0) ctx_issue_rows<BF16, UNC>(P, first.item, stage, rowbytes, &bar_full);
-    S.work[0] = first;
     S.status = 0;
   }
   __syncthreads();
-  uint32_t parity = 0;
-  int slot_cur = 0;
 
-  for (;;) {
+  // ======================= producer warp =======================
+  // One thread hands out work and keeps the copies going.  Items 0..3G-1 are dealt statically (CTA x
+  // takes x, x+G, x+2G); from then on a global counter hands them out.  A three-deep pipeline keeps
+  // every global round trip off the critical path: while the consumers process context i, the rows
+  // of i+1 are in flight, the descriptor of i+2 is being loaded and the index of i+3 is being fetched.
+  if (warp == CNW) {
+    if (lane == 0) {
+      const int n_heavy = P.counters->n_heavy;
+      const int total = n_heavy + P.counters->n_light;
+      const int cap = P.B * N;
+      const int G = gridDim.x;
+      auto load_item = [&](int w) -> WorkItem {
+        WorkItem it;
+        it.item = -1;
+        it.pad = 0;
+        if (w < total) {
+          const int slot = w < n_heavy ? w : cap - 1 - (w - n_heavy);
+          const int4 lo = __ldg(reinterpret_cast<const int4*>(P.work + slot));
+          const int4 hi = __ldg(reinterpret_cast<const int4*>(P.work + slot) + 1);
+          it.item = lo.x, it.cbase = lo.y, it.nchild = lo.z, it.node0 = lo.w;
+          it.tok0 = hi.x, it.r0 = __int_as_float(hi.y), it.u_final = __int_as_float(hi.z);
+        }
+        return it;
+      };
+      WorkItem it_cur = load_item(blockIdx.x);
+      WorkItem it_next = load_item(blockIdx.x + G);
+      int w_next2 = blockIdx.x + 2 * G;
+      for (int i = 0;; ++i) {
+        const int slot = i & 1;
+        // the slot is free once every consumer warp has finished the context that used it
+        if (i >= 2 && !mbar_wait(&bar_empty[slot], ((i >> 1) - 1) & 1)) {
+          it_cur.item = -1;
+          it_cur.pad = LANTERN_ST_INTERNAL;   // a consumer never released the slot: stop handing out work
+        }
+        S.work[slot] = it_cur;                // published by the mbarrier operation below
+        if (it_cur.item < 0) {
+          mbar_arrive(&bar_full[slot]);       // wake the consumers; they see the terminator
+          break;
+        }
+        fence_proxy_async();
+        ctx_issue_rows<BF16, UNC>(P, it_cur.item, smem + slot * stage_bytes, rowbytes, &bar_full[slot]);
+        it_cur = it_next;
+        it_next = load_item(w_next2);
+        w_next2 = 3 * G + atomicAdd(&P.counters->work_next, 1);
+      }
+    }
+    return;
+  }
+
+  // ======================= consumer warps =======================
+  for (int iter = 0;; ++iter) {
+    const int slot_cur = iter & 1;
+    // One warp watches the copy's mbarrier (bounded wait); the consumer barrier then releases everybody
+    // at once and tells every thread alike whether the rows have landed.
+    bool landed = true;
+    if (warp == 0) landed = mbar_wait(&bar_full[slot_cur], (iter >> 1) & 1);
+    const bool arrived = cbar_and(landed);
+    if (!arrived) break;   // the copy did not land within the limit; the walk reports the missing record
     const WorkItem cur = S.work[slot_cur];
     const int item = cur.item;
     if (item < 0) break;
+    unsigned char* stage = smem + slot_cur * stage_bytes;    // this context's rows, later its E
+    float* E = reinterpret_cast<float*>(stage);
     const int b = item / R;
     const ChildInfo* kids = P.children + cur.cbase;
     const int nchild = cur.nchild;
+    // every consumer is past the previous context (its record included): clear the shared status word;
+    // nobody sets it again before the [stats] barrier below
+    if (tid == 0) S.status = 0;
 
-    // first child: its neighbour row (two slots per thread) and, for thread 0, its raw logits
+    // first child: its neighbour row (two slots per thread) and, for thread 0, its raw logits; issued
+    // now, used after the streaming pass
     int node = cur.node0;
     int xt = cur.tok0;
     float r = cur.r0;
     const int j0 = 2 * tid + 1, j1 = 2 * tid + 2;
-    int n0 = (j0 < k) ? __ldg(P.nbr + static_cast<size_t>(xt) * k + j0) : -1;
-    int n1 = (j1 < k) ? __ldg(P.nbr + static_cast<size_t>(xt) * k + j1) : -1;
+    int n0 = (j0 < k) ? ld_nc_here(P.nbr + static_cast<size_t>(xt) * k + j0) : -1;
+    int n1 = (j1 < k) ? ld_nc_here(P.nbr + static_cast<size_t>(xt) * k + j1) : -1;
     float raw_c = 0.0f, raw_u = 0.0f, raw_d = 0.0f;
     if (tid == 0) {
       const size_t e = static_cast<size_t>(item) * V + xt;
@@ -164,45 +239,50 @@ __global__ void __launch_bounds__(CNT, 1) lantern_context_kernel(VerifyParams P)
       raw_d = ctx_raw_logit<BF16>(P.draft, e);
     }
 
-    // every thread must take the same branch: agree on whether the rows have landed
-    const bool arrived = __syncthreads_and(mbar_wait(&bar_full, parity)) != 0;
-    if (!arrived) {
-      // The copy did not land within the limit: report it, give the copy in flight one more bounded
-      // chance to finish before this CTA's shared memory is released, and stop.
-      if (tid == 0) {
-        Record rec = {-1, -1, LANTERN_ST_INTERNAL, 0};
-        P.records[item] = rec;
-      }
-      mbar_wait(&bar_full, parity);
-      break;
-    }
-    // every thread is past the previous context (its record included): clear the shared status word;
-    // nobody sets it again before the [stats] barrier below
-    if (tid == 0) S.status = 0;
-
     // ---------------- streaming pass, warp-local ----------------
-    float a[CH * 8], ep[CH * 8];
+    // staging rows: 0 = conditional target, 1 = unconditional target (if any), 2 = drafter
+    const unsigned char* rc = stage;
+    const unsigned char* ru = stage + rowbytes;
+    unsigned char* rd = stage + 2 * rowbytes;
+    const float Tinv_is_one = P.T == 1.0f;
+    // eight processed drafter logits of 16-byte group g (z_p = l_d / T)
+    auto draft_chunk = [&](int g, float (&out)[8]) {
+      if (BF16) {
+        const uint4 d = *reinterpret_cast<const uint4*>(rd + g * 16);
+        const uint32_t dw[4] = {d.x, d.y, d.z, d.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          out[2 * i] = __uint_as_float(dw[i] << 16);
+          out[2 * i + 1] = __uint_as_float(dw[i] & 0xffff0000u);
+        }
+      } else {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const float4 d = *reinterpret_cast<const float4*>(rd + g * 32 + h * 16);
+          out[4 * h] = d.x, out[4 * h + 1] = d.y, out[4 * h + 2] = d.z, out[4 * h + 3] = d.w;
+        }
+      }
+      if (!Tinv_is_one) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) out[e] = __fdiv_rn(out[e], P.T);
+      }
+    };
+    float a[CH * 8];
+    // --- target: guidance combine, warp maximum, numerators, partial sum; E replaces the raw rows ---
     {
-      const unsigned char* rc = stage;
-      const unsigned char* ru = stage + rowbytes;
-      const unsigned char* rd = stage + (UNC ? 2 : 1) * rowbytes;
-      const float s = P.cfg_scale, T = P.T;
+      const float s = P.cfg_scale;
 #pragma unroll
       for (int c = 0; c < CH; ++c) {
         const int g = c * CNT + tid;
         if (g * 8 < V) {
-          float lc[8], lu[8], ld[8];
+          float lc[8], lu[8];
           if (BF16) {
             const uint4 x = *reinterpret_cast<const uint4*>(rc + g * 16);
             const uint32_t xw[4] = {x.x, x.y, x.z, x.w};
-            const uint4 d = *reinterpret_cast<const uint4*>(rd + g * 16);
-            const uint32_t dw[4] = {d.x, d.y, d.z, d.w};
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
               lc[2 * i] = __uint_as_float(xw[i] << 16);
               lc[2 * i + 1] = __uint_as_float(xw[i] & 0xffff0000u);
-              ld[2 * i] = __uint_as_float(dw[i] << 16);
-              ld[2 * i + 1] = __uint_as_float(dw[i] & 0xffff0000u);
             }
             if (UNC) {
               const uint4 y = *reinterpret_cast<const uint4*>(ru + g * 16);
@@ -218,8 +298,6 @@ __global__ void __launch_bounds__(CNT, 1) lantern_context_kernel(VerifyParams P)
             for (int h = 0; h < 2; ++h) {
               const float4 x = *reinterpret_cast<const float4*>(rc + g * 32 + h * 16);
               lc[4 * h] = x.x, lc[4 * h + 1] = x.y, lc[4 * h + 2] = x.z, lc[4 * h + 3] = x.w;
-              const float4 d = *reinterpret_cast<const float4*>(rd + g * 32 + h * 16);
-              ld[4 * h] = d.x, ld[4 * h + 1] = d.y, ld[4 * h + 2] = d.z, ld[4 * h + 3] = d.w;
               if (UNC) {
                 const float4 y = *reinterpret_cast<const float4*>(ru + g * 32 + h * 16);
                 lu[4 * h] = y.x, lu[4 * h + 1] = y.y, lu[4 * h + 2] = y.z, lu[4 * h + 3] = y.w;
@@ -230,53 +308,59 @@ __global__ void __launch_bounds__(CNT, 1) lantern_context_kernel(VerifyParams P)
           for (int e = 0; e < 8; ++e) {
             float l = lc[e];
             if (UNC) l = __fmaf_rn(s, __fsub_rn(lc[e], lu[e]), lu[e]);   // l_u + s (l_c - l_u)
-            float d = ld[e];
-            if (T != 1.0f) {
-              l = __fdiv_rn(l, T);
-              d = __fdiv_rn(d, T);
-            }
+            if (!Tinv_is_one) l = __fdiv_rn(l, P.T);
             a[c * 8 + e] = l;
-            ep[c * 8 + e] = d;
           }
         } else {
 #pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            a[c * 8 + e] = ninf;
-            ep[c * 8 + e] = ninf;
-          }
+          for (int e = 0; e < 8; ++e) a[c * 8 + e] = ninf;
         }
       }
     }
-    __syncwarp();
-    if (lane == 0) {   // this warp no longer needs the staging rows
-      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(&bar_empty)) : "memory");
-    }
-    float mq = a[0], mp = ep[0];
+    float mq = a[0];
 #pragma unroll
-    for (int i = 1; i < CH * 8; ++i) {
-      mq = fmaxf(mq, a[i]);
-      mp = fmaxf(mp, ep[i]);
-    }
+    for (int i = 1; i < CH * 8; ++i) mq = fmaxf(mq, a[i]);
     // a slice without any finite logit (padding, masked tokens) still needs a finite shift
     mq = fmaxf(warp_max(mq), -1.0e37f);
-    mp = fmaxf(warp_max(mp), -1.0e37f);
-    const float mlq_w = mq * L_hi, mlp_w = mp * L_hi;
-    float tq = 0.0f, tp = 0.0f;
+    const float mlq_w = mq * L_hi;
+    float tq = 0.0f;
 #pragma unroll
     for (int c = 0; c < CH; ++c) {
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        a[c * 8 + e] = ex2_approx(__fmaf_rn(a[c * 8 + e], L_hi, -mlq_w));
-        ep[c * 8 + e] = ex2_approx(__fmaf_rn(ep[c * 8 + e], L_hi, -mlp_w));
-      }
+      for (int e = 0; e < 8; ++e) a[c * 8 + e] = ex2_approx(__fmaf_rn(a[c * 8 + e], L_hi, -mlq_w));
       tq += sum8(&a[c * 8]);
-      tp += sum8(&ep[c * 8]);
       const int g = c * CNT + tid;
       if (g * 8 < V) {
-        float4* dst = reinterpret_cast<float4*>(E);
-        dst[(((c << 1) | 0) << LOG_CNT) + tid] = make_float4(a[c * 8], a[c * 8 + 1], a[c * 8 + 2], a[c * 8 + 3]);
-        dst[(((c << 1) | 1) << LOG_CNT) + tid] = make_float4(a[c * 8 + 4], a[c * 8 + 5], a[c * 8 + 6], a[c * 8 + 7]);
+        *reinterpret_cast<float4*>(E + EI(g * 8)) = make_float4(a[c * 8], a[c * 8 + 1], a[c * 8 + 2], a[c * 8 + 3]);
+        *reinterpret_cast<float4*>(E + EI(g * 8 + 4)) =
+            make_float4(a[c * 8 + 4], a[c * 8 + 5], a[c * 8 + 6], a[c * 8 + 7]);
       }
+    }
+    // --- drafter: warp maximum and partial sum of numerators; the raw row stays in shared memory ---
+#pragma unroll
+    for (int c = 0; c < CH; ++c) {
+      const int g = c * CNT + tid;
+      float d8[8];
+      if (g * 8 < V) {
+        draft_chunk(g, d8);
+      } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) d8[e] = ninf;
+      }
+#pragma unroll
+      for (int e = 0; e < 8; ++e) a[c * 8 + e] = d8[e];
+    }
+    float mp = a[0];
+#pragma unroll
+    for (int i = 1; i < CH * 8; ++i) mp = fmaxf(mp, a[i]);
+    mp = fmaxf(warp_max(mp), -1.0e37f);
+    const float mlp_w = mp * L_hi;
+    float tp = 0.0f;
+#pragma unroll
+    for (int c = 0; c < CH; ++c) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) a[c * 8 + e] = ex2_approx(__fmaf_rn(a[c * 8 + e], L_hi, -mlp_w));
+      tp += sum8(&a[c * 8]);
     }
     {
       const double wq = warp_sum(static_cast<double>(tq));
@@ -289,23 +373,7 @@ __global__ void __launch_bounds__(CNT, 1) lantern_context_kernel(VerifyParams P)
       }
     }
 
-    // thread 0: once every warp has drained the staging rows, start the next context's copy, publish
-    // its descriptor for the next iteration and move the look-ahead pipeline one step
-    if (tid == 0) {
-      const bool drained = mbar_wait(&bar_empty, parity);
-      if (drained && it_next.item >= 0) {
-        fence_proxy_async();
-        ctx_issue_rows<BF16, UNC>(P, it_next.item, stage, rowbytes, &bar_full);
-      } else if (!drained) {
-        it_next.item = -1;          // never overwrite rows that may still be read: stop after this context
-        atomicOr(&S.status, LANTERN_ST_INTERNAL);
-      }
-      S.work[slot_cur ^ 1] = it_next;
-      it_next = load_item(w_next2);
-      w_next2 = 3 * G + atomicAdd(&P.counters->work_next, 1);
-    }
-    parity ^= 1u;
-    __syncthreads();   // [stats] per-warp maxima and sums, and E, are visible
+    cbar();   // [stats] per-warp maxima and sums, and E, are visible
 
     // ---------------- block statistics, computed by every warp for itself ----------------
     float fq_l, fp_l;            // lane l holds the factor that brings warp l's units to global units
@@ -340,8 +408,8 @@ __global__ void __launch_bounds__(CNT, 1) lantern_context_kernel(VerifyParams P)
           zq = __fdiv_rn(zq, P.T);
           zp = __fdiv_rn(zp, P.T);
         }
-        S.acc_e = exp2(static_cast<double>(zq) * LOG2E - static_cast<double>(mlq_g));
-        S.acc_p = exp2(static_cast<double>(zp) * LOG2E - static_cast<double>(mlp_g));
+        S.acc_e = exp2_single(zq, mlq_g);
+        S.acc_p = exp2_single(zp, mlp_g);
         S.acc_valid = 1;
       }
 
@@ -353,16 +421,16 @@ __global__ void __launch_bounds__(CNT, 1) lantern_context_kernel(VerifyParams P)
           const int4 v = __ldg(reinterpret_cast<const int4*>(kids + ci + 1));
           sib.node = v.x, sib.token = v.y, sib.r = __int_as_float(v.z);
         }
-        // owner of x~ publishes its drafter numerator (0 if x~ was rejected before)
-        if (cowner_thread(xt) == tid) {
-          const int li = ((xt >> (3 + LOG_CNT)) << 3) | (xt & 7);
-          float v = 0.0f;
-#pragma unroll
-          for (int i = 0; i < CH * 8; ++i)
-            if (i == li) v = ep[i];
-          S.px_bulk = v * fp_mine;
+        // drafter numerator of x~ from the raw row (-inf, hence 0, once x~ has been rejected), global units
+        float px_bulk;
+        {
+          float dz = BF16 ? __uint_as_float(static_cast<uint32_t>(reinterpret_cast<const unsigned short*>(rd)[xt]) << 16)
+                          : reinterpret_cast<const float*>(rd)[xt];
+          if (!Tinv_is_one) dz = __fdiv_rn(dz, P.T);
+          const int ow = cowner_thread(xt) >> 5;
+          px_bulk = ex2_approx(__fmaf_rn(dz, L_hi, -S.mlp[ow])) * __shfl_sync(kFull, fp_l, ow);
         }
-        const float e_xt_bulk = E[cphys(xt)] * __shfl_sync(kFull, fq_l, cowner_thread(xt) >> 5);
+        const float e_xt_bulk = E[EI(xt)] * __shfl_sync(kFull, fq_l, cowner_thread(xt) >> 5);
 
         // ---- A_{k,delta}(x~): gather + prefix scan with the strict bound ----
         const double thr = delta / qscale;   // the bound in the units of the unnormalised sums
@@ -379,11 +447,11 @@ __global__ void __launch_bounds__(CNT, 1) lantern_context_kernel(VerifyParams P)
           if ((va && !ia) || (vb && !ib)) atomicOr(&S.status, LANTERN_ST_BAD_TABLE);   // carries no mass
           const float fa = __shfl_sync(kFull, fq_l, ia ? cowner_thread(na) >> 5 : 0);
           const float fb = __shfl_sync(kFull, fq_l, ib ? cowner_thread(nb) >> 5 : 0);
-          const double da = ia ? static_cast<double>(E[cphys(na)] * fa) : 0.0;
-          const double db = ib ? static_cast<double>(E[cphys(nb)] * fb) : 0.0;
+          const double da = ia ? static_cast<double>(E[EI(na)] * fa) : 0.0;
+          const double db = ib ? static_cast<double>(E[EI(nb)] * fb) : 0.0;
           const double incl = warp_incl_scan(da + db, lane);
           if (lane == 31) S.wt[warp] = incl;
-          __syncthreads();   // [scan 1]
+          cbar();   // [scan 1]
           double pre, tot;
           {
             const double t = lane < CNW ? S.wt[lane] : 0.0;
@@ -403,7 +471,7 @@ __global__ void __launch_bounds__(CNT, 1) lantern_context_kernel(VerifyParams P)
           } else if (wfirst == kNone && lane == 0) {
             S.first[warp] = kNone;
           }
-          __syncthreads();   // [scan 2]
+          cbar();   // [scan 2]
           const int f_l = lane < CNW ? S.first[lane] : kNone;
           const int gfirst = __reduce_min_sync(kFull, f_l);
           if (gfirst != kNone) {
@@ -416,11 +484,11 @@ __global__ void __launch_bounds__(CNT, 1) lantern_context_kernel(VerifyParams P)
             sm = carry;
           }
         }
-        if (k == 1) __syncthreads();   // publish S.px_bulk / S.acc_* when the scan loop did not run
+        if (k == 1) cbar();   // publish S.acc_* when the scan loop did not run
         // the two single probabilities: thread 0's double-precision values where it has them; a bulk
         // value of exactly zero (token inside an earlier A, or rejected before) stays zero
         const bool acc = S.acc_valid != 0;
-        const float pxb = S.px_bulk;
+        const float pxb = px_bulk;
         const double e_xt = (acc && e_xt_bulk != 0.0f) ? S.acc_e : static_cast<double>(e_xt_bulk);
         const double p_xt = (acc && pxb != 0.0f) ? S.acc_p : static_cast<double>(pxb);
         const double qa = (e_xt + sm) * qscale;
@@ -442,27 +510,25 @@ __global__ void __launch_bounds__(CNT, 1) lantern_context_kernel(VerifyParams P)
           const int ja = base + j0, jb = base + j1;
           if (ja <= m) {
             const int n = base == 0 ? n0 : __ldg(nrow + ja);
-            if (static_cast<unsigned>(n) < static_cast<unsigned>(V)) E[cphys(n)] = -fabsf(E[cphys(n)]);
+            if (static_cast<unsigned>(n) < static_cast<unsigned>(V)) E[EI(n)] = -fabsf(E[EI(n)]);
           }
           if (jb <= m) {
             const int n = base == 0 ? n1 : __ldg(nrow + jb);
-            if (static_cast<unsigned>(n) < static_cast<unsigned>(V)) E[cphys(n)] = -fabsf(E[cphys(n)]);
+            if (static_cast<unsigned>(n) < static_cast<unsigned>(V)) E[EI(n)] = -fabsf(E[EI(n)]);
           }
         }
-        if (tid == 0) E[cphys(xt)] = -fabsf(E[cphys(xt)]);
-        if (cowner_thread(xt) == tid) {   // x~ leaves the drafter distribution for the following siblings
-          const int li = ((xt >> (3 + LOG_CNT)) << 3) | (xt & 7);
-#pragma unroll
-          for (int i = 0; i < CH * 8; ++i)
-            if (i == li) ep[i] = 0.0f;
+        if (tid == 0) E[EI(xt)] = -fabsf(E[EI(xt)]);
+        if (tid == 0) {   // x~ leaves the drafter distribution for the following siblings
+          if (BF16) reinterpret_cast<unsigned short*>(rd)[xt] = 0xff80;   // -inf
+          else reinterpret_cast<float*>(rd)[xt] = ninf;
         }
         const bool last = (ci + 1 == nchild);
         if (!last) {   // next sibling's neighbour row, in flight during the residual pass
           node = sib.node;
           xt = sib.token;
           r = sib.r;
-          n0 = (j0 < k) ? __ldg(P.nbr + static_cast<size_t>(xt) * k + j0) : -1;
-          n1 = (j1 < k) ? __ldg(P.nbr + static_cast<size_t>(xt) * k + j1) : -1;
+          n0 = (j0 < k) ? ld_nc_here(P.nbr + static_cast<size_t>(xt) * k + j0) : -1;
+          n1 = (j1 < k) ? ld_nc_here(P.nbr + static_cast<size_t>(xt) * k + j1) : -1;
           if (tid == 0) {   // its raw logits, for the double-precision replay below
             const size_t e = static_cast<size_t>(item) * V + xt;
             raw_c = ctx_raw_logit<BF16>(P.target, e);
@@ -470,7 +536,7 @@ __global__ void __launch_bounds__(CNT, 1) lantern_context_kernel(VerifyParams P)
             raw_d = ctx_raw_logit<BF16>(P.draft, e);
           }
         }
-        __syncthreads();   // [flags]
+        cbar();   // [flags]
         // w = E - (p'/q' scale ratio) * ep, in this warp's own units of E
         const float ratio = static_cast<float>((pscale * static_cast<double>(fp_mine)) /
                                                (qscale * static_cast<double>(fq_mine)));
@@ -480,19 +546,23 @@ __global__ void __launch_bounds__(CNT, 1) lantern_context_kernel(VerifyParams P)
         for (int c = 0; c < CH; ++c) {
           const int g = c * CNT + tid;
           if (g * 8 < V) {
-            const float4* src = reinterpret_cast<const float4*>(E);
-            const float4 lo = src[(((c << 1) | 0) << LOG_CNT) + tid];
-            const float4 hi = src[(((c << 1) | 1) << LOG_CNT) + tid];
+            const float4 lo = *reinterpret_cast<const float4*>(E + EI(g * 8));
+            const float4 hi = *reinterpret_cast<const float4*>(E + EI(g * 8 + 4));
             const float e8[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+            float ep8[8];
+            draft_chunk(g, ep8);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) a[c * 8 + e] = fmaxf(0.0f, __fmaf_rn(-ratio, ep[c * 8 + e], e8[e]));
+            for (int e = 0; e < 8; ++e) {
+              ep8[e] = ex2_approx(__fmaf_rn(ep8[e], L_hi, -mlp_w));
+              a[c * 8 + e] = fmaxf(0.0f, __fmaf_rn(-ratio, ep8[e], e8[e]));
+            }
+            psum += sum8(ep8);
           } else {
 #pragma unroll
             for (int e = 0; e < 8; ++e) a[c * 8 + e] = 0.0f;
           }
           cs[c] = sum8(&a[c * 8]);
           wsum += cs[c];
-          psum += sum8(&ep[c * 8]);
         }
         const double fqd = static_cast<double>(fq_mine);
         double W, Sp;
@@ -502,9 +572,8 @@ __global__ void __launch_bounds__(CNT, 1) lantern_context_kernel(VerifyParams P)
           for (int c = 0; c < CH; ++c) {
             const int g = c * CNT + tid;
             if (g * 8 < V) {
-              float4* dst = reinterpret_cast<float4*>(E);
-              dst[(((c << 1) | 0) << LOG_CNT) + tid] = make_float4(a[c * 8], a[c * 8 + 1], a[c * 8 + 2], a[c * 8 + 3]);
-              dst[(((c << 1) | 1) << LOG_CNT) + tid] =
+              *reinterpret_cast<float4*>(E + EI(g * 8)) = make_float4(a[c * 8], a[c * 8 + 1], a[c * 8 + 2], a[c * 8 + 3]);
+              *reinterpret_cast<float4*>(E + EI(g * 8 + 4)) =
                   make_float4(a[c * 8 + 4], a[c * 8 + 5], a[c * 8 + 6], a[c * 8 + 7]);
             }
           }
@@ -514,7 +583,7 @@ __global__ void __launch_bounds__(CNT, 1) lantern_context_kernel(VerifyParams P)
             S.wt[warp] = ww;
             S.wt[CNW + warp] = wp;
           }
-          __syncthreads();   // [totals] also publishes the written-back residual
+          cbar();   // [totals] also publishes the written-back residual
           W = warp_sum(lane < CNW ? S.wt[lane] : 0.0);
           Sp = warp_sum(lane < CNW ? S.wt[CNW + lane] : 0.0);
           if (!(W > 0.0)) {
@@ -534,8 +603,8 @@ __global__ void __launch_bounds__(CNT, 1) lantern_context_kernel(VerifyParams P)
                 zq = __fdiv_rn(zq, P.T);
                 zp = __fdiv_rn(zp, P.T);
               }
-              double e = exp2(static_cast<double>(zq) * LOG2E - static_cast<double>(mlq_g));
-              const double pe = exp2(static_cast<double>(zp) * LOG2E - static_cast<double>(mlp_g));
+              double e = exp2_single(zq, mlq_g);
+              const double pe = exp2_single(zp, mlp_g);
               for (int i = 0; i <= ci; ++i) e = fmax(0.0, e - S.hist[i] * pe);
               S.acc_e = e;
               S.acc_p = pe;
@@ -556,7 +625,7 @@ __global__ void __launch_bounds__(CNT, 1) lantern_context_kernel(VerifyParams P)
           incl[c] = warp_incl_scan(csd[c], lane);
           if (lane == 31) S.wt[c * CNW + warp] = incl[c];
         }
-        __syncthreads();   // [draw 1]
+        cbar();   // [draw 1]
         {
           // exclusive prefix over (chunk, warp) in chunk-major order; 32 entries per round
           double carry2 = 0.0;
@@ -588,7 +657,7 @@ __global__ void __launch_bounds__(CNT, 1) lantern_context_kernel(VerifyParams P)
         const int wmin = __reduce_min_sync(kFull, cand);
         if (lane == 0) S.cand[warp] = wmin;
         if (tid == 0) S.tok = -1;
-        __syncthreads();   // [draw 2]
+        cbar();   // [draw 2]
         const int win = __reduce_min_sync(kFull, lane < CNW ? S.cand[lane] : kNone);
         if (win == kNone) {
           // rounding left no slot above the target: the largest token of positive weight
@@ -600,7 +669,7 @@ __global__ void __launch_bounds__(CNT, 1) lantern_context_kernel(VerifyParams P)
               if (a[c * 8 + e] > 0.0f) lastp = (c * CNT + tid) * 8 + e;
           if (lastp >= V) lastp = -1;
           if (lastp >= 0) atomicMax(&S.tok, lastp);
-          __syncthreads();
+          cbar();
           if (tid == 0) {
             Record rec = {-1, S.tok, status | S.status | (S.tok < 0 ? LANTERN_ST_DEGENERATE : 0), 0};
             P.records[item] = rec;
@@ -633,7 +702,9 @@ __global__ void __launch_bounds__(CNT, 1) lantern_context_kernel(VerifyParams P)
       Record rec = {accepted, -1, status | S.status, 0};
       P.records[item] = rec;
     }
-    slot_cur ^= 1;
+    // this context's staging area (rows and E) is no longer needed by this warp
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&bar_empty[slot_cur]);
   }
 }
 

@@ -174,6 +174,10 @@ lantern_status lantern_verify_static(const void* target_logits, const void* draf
                                      float* out_node_qa, float* out_node_px, int32_t* out_node_m,
                                      void* cuda_stream);
 
+/* Revision number of the fused verification kernel; bumped whenever that kernel changes, so that
+ * stored profiler counters can be matched to the code they were taken on. */
+int lantern_kernel_revision(void);
+
 /* Number of kernels (and memsets) one lantern_verify call enqueues; for launch accounting. */
 int lantern_verify_launch_count(void);
 

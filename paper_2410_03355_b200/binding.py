@@ -51,6 +51,8 @@ def load_library():
     lib.lantern_build_neighbors.argtypes = [vp, i32, i32, i32, vp, vp, vp, sz, vp]
     lib.lantern_verify_workspace_bytes.restype = sz
     lib.lantern_verify_workspace_bytes.argtypes = [i32, i32]
+    lib.lantern_kernel_revision.restype = i32
+    lib.lantern_kernel_revision.argtypes = []
     lib.lantern_verify_launch_count.restype = i32
     lib.lantern_verify_launch_count.argtypes = []
     lib.lantern_verify_static.restype = i32
@@ -232,3 +234,8 @@ def verify_static(target_logits: torch.Tensor, draft_logits: Optional[torch.Tens
     if rc != 0:
         raise LanternError(rc, "lantern_verify_static")
     return out
+
+
+def kernel_revision() -> int:
+    """Revision number of the fused verification kernel (matches stored profiler counters to code)."""
+    return int(load_library().lantern_kernel_revision())

@@ -514,6 +514,8 @@ extern "C" size_t lantern_verify_workspace_bytes(int B, int N) {
 
 extern "C" int lantern_verify_launch_count(void) { return 5; }
 
+extern "C" int lantern_kernel_revision(void) { return LANTERN_CONTEXT_KERNEL_REVISION; }
+
 extern "C" lantern_status lantern_verify_profile_events(void* before_fused, void* after_fused) {
   if ((before_fused == nullptr) != (after_fused == nullptr)) return LANTERN_E_NULL;
   g_ev_before = static_cast<cudaEvent_t>(before_fused);

@@ -22,6 +22,8 @@
 // inverse-CDF draw or the write-back for the next sibling.
 #pragma once
 
+#define LANTERN_CONTEXT_KERNEL_REVISION 5   // bump on every change to this file
+
 namespace lantern {
 
 constexpr int CNT = 512;        // threads per CTA

@@ -166,6 +166,28 @@ def oracle_sample_rate(host_inp, table_host, delta, budget_s=15.0):
     return pos / t_used, done, t_used
 
 
+def max_over_ranks(values, dist=None, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks (every rank gets the result).  The
+    verification path has no exchange step: this reduction of the measured times is the only
+    collective of a multi-rank run."""
+    if dist is None:
+        return [float(v) for v in values]
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def rank_seed(base_seed: int, rank: int) -> int:
+    """Every rank verifies its own, differently seeded batch of the same shape (weak scaling)."""
+    return int(base_seed) + 17 * int(rank)
+
+
+def aggregate_rate(world: int, sequences_per_rank: int, drafts: int, ms_per_step: float) -> float:
+    """Whole-job positions per second: all ranks' positions over the slowest rank's step time."""
+    return world * sequences_per_rank * drafts / (ms_per_step * 1e-3)
+
+
 def run_reference(args, rank, world):
     """The reference arm: the CPU oracle as it stands, timed on host cores on a bounded sample."""
     if rank != 0:
@@ -275,7 +297,7 @@ def main():
     del bws
 
     # ---- inputs resident in HBM ----
-    d = lid.config_verify_inputs_device(w["config"], B=B, seed=li.BASE_SEED + 17 * rank, rho=args.rho)
+    d = lid.config_verify_inputs_device(w["config"], B=B, seed=rank_seed(li.BASE_SEED, rank), rho=args.rho)
     torch.cuda.synchronize()
     alg_bytes = algorithmic_bytes(cfg, B, d["tree_parents"])
     ws = torch.empty(lt.verify_workspace_bytes(B, N), dtype=torch.uint8, device="cuda")
@@ -320,12 +342,9 @@ def main():
     clocks = sampler.stop() if rank == 0 else None
     ms_total = t_start.elapsed_time(t_stop)
     fused_ms = float(np.mean([a.elapsed_time(b_) for a, b_ in kev]))
-    if dist is not None:
-        t = torch.tensor([ms_total, fused_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, fused_ms = float(t[0]), float(t[1])
+    ms_total, fused_ms = max_over_ranks([ms_total, fused_ms], dist, "cuda")
     ms_per_step = ms_total / args.steps
-    value = world * B * N / (ms_per_step * 1e-3)
+    value = aggregate_rate(world, B, N, ms_per_step)
 
     status_bad = int((out.status != 0).sum().item())
     accept_mean = float(out.accept_len.float().mean().item())
@@ -361,11 +380,8 @@ def main():
         b_.record()
         torch.cuda.synchronize()
         ms_e2e = a.elapsed_time(b_) / args.e2e_steps
-        if dist is not None:
-            t = torch.tensor([ms_e2e], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t[0])
-        e2e = {"value": world * B * N / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+        ms_e2e = max_over_ranks([ms_e2e], dist, "cuda")[0]
+        e2e = {"value": aggregate_rate(world, B, N, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
                "d2h_bytes_per_step": int(d2h), "ms_per_step": ms_e2e, "steps": args.e2e_steps}
         del host
 

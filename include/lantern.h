@@ -111,9 +111,9 @@ lantern_status lantern_build_neighbors(const float* codebook, int V, int D, int 
  *   neighbor_idx   [V, k] int32 as written by lantern_build_neighbors (slot 0 = the token itself)
  *   k, delta       1 <= k <= V; delta >= 0 (delta = 0 or k = 1 gives standard speculative sampling)
  *   uniforms       [B, N+1] fp32 in [0, 1): entry i tests node i, entry N is the final draw
- *   B, N, V        B >= 0; 0 <= N <= 1024; V a multiple of 8, 8 <= V <= 16384, and small enough
- *                  that C+1 logit rows plus V floats fit in shared memory (fp32 logits with
- *                  has_uncond: V <= 8192)
+ *   B, N, V        B >= 0; 0 <= N <= 1024; V a multiple of 8, 8 <= V <= 16384 with bf16 logits and
+ *                  8 <= V <= 8192 with fp32 logits (two staging areas of three logit rows each
+ *                  must fit in shared memory); anything else returns LANTERN_E_SHAPE
  *   out_accept_len  [B] number of accepted nodes
  *   out_next_token  [B] resampled or bonus token (-1 with a fault bit in out_status)
  *   out_accept_path [B, N] node ids of the accepted path in order, -1 padded; may be NULL

@@ -543,7 +543,7 @@ extern "C" lantern_status lantern_verify(const void* target_logits, const void* 
   // two staging areas of (C+1) rows each; the numerators are kept over the rows they came from
   const size_t smem_bytes = 2 * ((static_cast<size_t>(3) * V * esize + 127) & ~static_cast<size_t>(127));
   (void)nrows;
-  if (smem_bytes > 220 * 1024) return LANTERN_E_SHAPE;
+  if (smem_bytes > 220 * 1024 || (dtype == LANTERN_F32 && V > 8192)) return LANTERN_E_SHAPE;
   if (B == 0) return LANTERN_OK;
   if (!target_logits || !neighbor_idx || !uniforms || !out_accept_len || !out_next_token) return LANTERN_E_NULL;
   if (N > 0 && (!draft_logits || !draft_tokens)) return LANTERN_E_NULL;

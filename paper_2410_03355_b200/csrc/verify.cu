@@ -487,7 +487,7 @@ static thread_local cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
 template <int CHC, bool BF16, bool UNC>
 static cudaError_t launch_verify(const VerifyParams& P, int grid_ctx, int grid_bonus, size_t smem_bytes,
                                  cudaStream_t st) {
-  constexpr int CHB = CHC == 4 ? 2 : 1;   // the bonus kernel runs 1024 threads per row
+  constexpr int CHB = CHC == 8 ? 2 : 1;   // the bonus kernel runs 1024 threads per row
   auto kc = lantern_context_kernel<CHC, BF16, UNC>;
   cudaError_t e = cudaFuncSetAttribute(kc, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
   if (e != cudaSuccess) return e;
@@ -539,9 +539,9 @@ extern "C" lantern_status lantern_verify(const void* target_logits, const void* 
   if (T == 0.0f) return LANTERN_E_UNIMPLEMENTED;   // greedy decoding is not part of this build
   const int esize = dtype == LANTERN_BF16 ? 2 : 4;
   const int nrows = has_uncond ? 3 : 2;
-  const int CH = V > 2 * CNT * 8 ? 4 : (V > CNT * 8 ? 2 : 1);   // 8-token chunks per thread of the fused kernel
-  // two staging areas of (C+1) rows each; the numerators are kept over the rows they came from
-  const size_t smem_bytes = 2 * ((static_cast<size_t>(3) * V * esize + 127) & ~static_cast<size_t>(127));
+  const int CH = V > 4 * GT * 8 ? 8 : (V > 2 * GT * 8 ? 4 : (V > GT * 8 ? 2 : 1));   // 8-token chunks per thread
+  // one staging area of three row slots per consumer group; the numerators are kept over the rows they came from
+  const size_t smem_bytes = NGRP * ((static_cast<size_t>(3) * V * esize + 127) & ~static_cast<size_t>(127));
   (void)nrows;
   if (smem_bytes > 220 * 1024 || (dtype == LANTERN_F32 && V > 8192)) return LANTERN_E_SHAPE;
   if (B == 0) return LANTERN_OK;
@@ -596,7 +596,8 @@ extern "C" lantern_status lantern_verify(const void* target_logits, const void* 
   if (cudaGetLastError() != cudaSuccess) return LANTERN_E_CUDA;
 
   const long long items = static_cast<long long>(B) * (N > 0 ? N : 1);   // upper bound of contexts with children
-  const int grid_ctx = static_cast<int>(items < sms ? items : sms);
+  const long long ctas = (items + NGRP - 1) / NGRP;   // every CTA runs NGRP contexts at a time
+  const int grid_ctx = static_cast<int>(ctas < sms ? ctas : sms);
   const int grid_bonus = B < sms ? B : sms;
   cudaError_t e;
   const bool bf = dtype == LANTERN_BF16, un = has_uncond != 0;
@@ -605,7 +606,7 @@ extern "C" lantern_status lantern_verify(const void* target_logits, const void* 
             : launch_verify<CHV, true, false>(P, grid_ctx, grid_bonus, smem_bytes, st))              \
       : (un ? launch_verify<CHV, false, true>(P, grid_ctx, grid_bonus, smem_bytes, st)               \
             : launch_verify<CHV, false, false>(P, grid_ctx, grid_bonus, smem_bytes, st)))
-  e = CH == 4 ? LANTERN_DISPATCH(4) : (CH == 2 ? LANTERN_DISPATCH(2) : LANTERN_DISPATCH(1));
+  e = CH == 8 ? LANTERN_DISPATCH(8) : (CH == 4 ? LANTERN_DISPATCH(4) : (CH == 2 ? LANTERN_DISPATCH(2) : LANTERN_DISPATCH(1)));
 #undef LANTERN_DISPATCH
   return e == cudaSuccess ? LANTERN_OK : LANTERN_E_CUDA;
 }

@@ -1,61 +1,70 @@
 // Fused context pass of the LANTERN verification step (included by verify.cu).
 //
-// Persistent kernel, one CTA per SM: 16 consumer warps and one producer warp, two staging areas
-// in shared memory.  The producer hands out contexts and issues bulk asynchronous copies (TMA,
-// completion on an mbarrier, no multicast) that bring the NEXT context's rows into one area for
-// the whole time the consumers work on the current context in the other, so HBM streams
-// continuously and no consumer ever waits on a global round trip of the work queue.  The current context's softmax numerators E are stored over its
-// own raw rows once those have been read into registers: every thread overwrites only bytes
-// that it alone has read, so this needs no barrier and no third buffer.
+// Persistent kernel, one CTA per SM.  The CTA holds TWO independent consumer groups of eight
+// warps, each working on its own context in its own staging area of shared memory, and two
+// producer warps (one thread each) that hand out contexts and issue the bulk asynchronous
+// copies (TMA, completion on an mbarrier, no multicast) of a group's next rows as soon as the
+// group releases its area.  The two groups drift apart in phase, so the latency-bound deciding
+// part of one context overlaps the issue-bound streaming part of the other and the copy of a
+// third: the SM is rarely idle although every context is a chain of dependent steps.
 //
-// Each warp streams its slice of the rows on its own: guidance combine, the warp's own maximum,
-// numerators 2^((z - max_w) log2 e) through the hardware ex2 unit, partial sums.  One block
-// barrier later every warp has all warps' (maximum, sum) pairs and rescales on the fly: the
-// numerators in shared memory stay in their warp's own units and carry a per-warp factor.
-// Sums over many numerators average the ex2 unit's ~1e-7 rounding out; the two single
-// probabilities that decide a chain position, q(x~) and p(x~), are recomputed by one thread in
-// double precision from the raw logits.
+// Streaming part (per warp, on its own slice, in passes of at most 32 tokens per thread):
+// guidance combine, the slice's maximum, numerators 2^((z - max) log2 e) through the hardware
+// ex2 unit, partial sums.  The numerators E are stored over the context's own raw target rows
+// (every thread overwrites only bytes that it alone has read) and stay in the units of their
+// (pass, warp) slice; a per-slice factor brings them to common units when they are used.  Sums
+// over many numerators average the ex2 unit's ~1e-7 rounding out; the two single probabilities
+// that decide a position, q(x~) and p(x~), are recomputed by one thread in double precision.
 //
-// Per child (Section 4.3 / Algorithm 2, second block): gather of the neighbour row's
-// numerators, double-precision block scan with the strict bound, accept test; on rejection the
-// residual [q_{k,delta}(.|D = x~) - p]_+ in one register pass, its total, and either the
+// Deciding part, per child (Section 4.3 / Algorithm 2, second block): gather of the neighbour
+// row's numerators, double-precision scan against the strict bound, accept test; on rejection
+// the residual [q_{k,delta}(.|D = x~) - p]_+ in one register pass (drafter numerators are
+// recomputed from the raw drafter row, which stays in shared memory), its total, and either the
 // inverse-CDF draw or the write-back for the next sibling.
 #pragma once
 
-#define LANTERN_CONTEXT_KERNEL_REVISION 5   // bump on every change to this file
+#define LANTERN_CONTEXT_KERNEL_REVISION 6   // bump on every change to this file
 
 namespace lantern {
 
-constexpr int CNT = 512;        // threads per CTA
-constexpr int CNW = CNT / 32;   // warps per CTA
-constexpr int LOG_CNT = 9;
+constexpr int GT = 256;         // threads of one consumer group
+constexpr int GW = GT / 32;     // warps of one consumer group
+constexpr int LOG_GT = 8;
+constexpr int NGRP = 2;         // consumer groups per CTA
+constexpr int MAXU = 16;        // (pass, warp) slices of a context, at most
 constexpr int kNone = 0x7fffffff;
+constexpr int CTX_THREADS = NGRP * GT + NGRP * 32;   // consumers, then one producer warp per group
 
-// Thread t owns, for chunk c, the eight consecutive tokens [(c*CNT + t)*8, +8), i.e. 16-byte group
-// g = c*CNT + t of a bf16 row.  E is laid over the context's own raw rows: with bf16 logits the low
-// four numerators of group g replace group g of the first row and the high four replace group g of
-// the second row; with fp32 logits the eight numerators replace the group's own 32 bytes of the
-// first row.  Float index of token x inside the staging area:
+// Thread t of a group owns, for chunk c, the eight consecutive tokens [(c*GT + t)*8, +8), i.e. 16-byte
+// group g = c*GT + t of a bf16 row.  E is laid over the context's own raw target rows: with bf16 logits
+// the low four numerators of g replace g's bytes in row slot 0 and the high four replace g's bytes in
+// row slot 1; with fp32 logits the eight numerators replace g's own 32 bytes of row slot 0.
+// Float index of token x inside the staging area:
 template <bool BF16>
 __device__ __forceinline__ int ephys(int x, int row_floats) {
   if (BF16) return ((x >> 2) & 1) * row_floats + ((x >> 3) << 2) + (x & 3);
   return x;
 }
-__device__ __forceinline__ int cowner_thread(int x) { return (x >> 3) & (CNT - 1); }
+// (pass, warp) slice that owns token x; LOG_CP = log2(chunks per pass)
+template <int LOG_CP>
+__device__ __forceinline__ int owner_unit(int x) {
+  const int g = x >> 3;
+  return ((g >> (LOG_GT + LOG_CP)) * GW) + ((g & (GT - 1)) >> 5);
+}
 
-struct CtxShared {
-  double sq[CNW], sp[CNW];      // per-warp sums of numerators, in the warp's own units
-  double wt[4 * CNW];           // per-(chunk, warp) totals for scans and block sums
-  double sbefore[CNW];          // prefix sum just before a warp's first failing neighbour
-  double acc_e, acc_p;          // double-precision numerators of the tested x~, global units
+struct GroupShared {
+  double sq[MAXU], sp[MAXU];    // per-slice sums of numerators, in the slice's own units
+  double wt[8 * GW];            // per-(chunk, warp) totals for scans and block sums
+  double sbefore[GW];           // prefix sum just before a warp's first failing neighbour
+  double acc_e, acc_p;          // double-precision numerators of the tested x~, common units
   double hist[32];              // drafter/target scale ratio of each earlier rejection round of this context
+  float mlq[MAXU], mlp[MAXU];   // per-slice shift constants fl(max * log2 e)
+  int first[GW];                // a warp's first failing neighbour slot
+  int cand[GW];
   int acc_valid;                // acc_e / acc_p are usable for the current child
-  float mlq[CNW], mlp[CNW];     // per-warp shift constants fl(max_w * log2 e)
-  int first[CNW];               // a warp's first failing neighbour slot
-  int cand[CNW];
   int tok;
   int status;                   // OR of status bits seen by single threads
-  WorkItem work[2];
+  WorkItem work;
 };
 
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -102,20 +111,18 @@ __device__ __forceinline__ float ctx_raw_logit(const void* base, size_t elem) {
   return __ldg(static_cast<const float*>(base) + elem);
 }
 
-constexpr int CTX_THREADS = CNT + 32;   // 16 consumer warps and one producer warp
-
-// barrier among the 512 consumer threads only (the producer warp never joins it)
-__device__ __forceinline__ void cbar() { asm volatile("bar.sync 1, %0;" ::"n"(CNT) : "memory"); }
-// the same barrier, returning the AND of every consumer thread's predicate
-__device__ __forceinline__ bool cbar_and(bool pred) {
+// barrier among the 256 threads of consumer group `grp` (hardware barrier 1 + grp)
+__device__ __forceinline__ void gbar(int grp) { asm volatile("bar.sync %0, %1;" ::"r"(1 + grp), "n"(GT) : "memory"); }
+// the same barrier, returning the AND of every thread's predicate
+__device__ __forceinline__ bool gbar_and(int grp, bool pred) {
   uint32_t r;
   asm volatile(
       "{\n\t.reg .pred p, q;\n\t"
       "setp.ne.u32 p, %1, 0;\n\t"
-      "bar.red.and.pred q, 1, %2, p;\n\t"
+      "bar.red.and.pred q, %2, %3, p;\n\t"
       "selp.u32 %0, 1, 0, q;\n\t}"
       : "=r"(r)
-      : "r"(static_cast<uint32_t>(pred)), "n"(CNT)
+      : "r"(static_cast<uint32_t>(pred)), "r"(1 + grp), "n"(GT)
       : "memory");
   return r != 0;
 }
@@ -129,13 +136,18 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
 }
 
+// CH = 8-token chunks per thread (1, 2, 4 or 8); a thread streams them in NP passes of CP chunks
 template <int CH, bool BF16, bool UNC>
 __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyParams P) {
+  constexpr int NP = CH > 4 ? 2 : 1;          // passes
+  constexpr int CP = CH / NP;                 // chunks per pass
+  constexpr int LOG_CP = CP == 4 ? 2 : (CP == 2 ? 1 : 0);
+  constexpr int NU = NP * GW;                 // slices with their own units
   extern __shared__ __align__(128) unsigned char smem[];
-  __shared__ CtxShared S;
-  __shared__ __align__(8) uint64_t bar_full[2], bar_empty[2];
+  __shared__ GroupShared SG[NGRP];
+  __shared__ __align__(8) uint64_t bar_full[NGRP], bar_empty[NGRP];
 
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x, lane = tid & 31;
   const int V = P.V, N = P.N, R = P.R, k = P.k;
   const int rowbytes = V * (BF16 ? 2 : 4);
   const int stage_bytes = (3 * rowbytes + 127) & ~127;   // row slots: conditional, unconditional, drafter
@@ -145,27 +157,32 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
   const float ninf = __int_as_float(0xff800000);
 
   if (tid == 0) {
-    mbar_init(&bar_full[0], 1);
-    mbar_init(&bar_full[1], 1);
-    mbar_init(&bar_empty[0], CNW);
-    mbar_init(&bar_empty[1], CNW);
+    for (int g = 0; g < NGRP; ++g) {
+      mbar_init(&bar_full[g], 1);
+      mbar_init(&bar_empty[g], GW);
+      SG[g].status = 0;
+    }
     fence_mbar_init();
     fence_proxy_async();
-    S.status = 0;
   }
   __syncthreads();
 
-  // ======================= producer warp =======================
-  // One thread hands out work and keeps the copies going.  Items 0..3G-1 are dealt statically (CTA x
-  // takes x, x+G, x+2G); from then on a global counter hands them out.  A three-deep pipeline keeps
-  // every global round trip off the critical path: while the consumers process context i, the rows
-  // of i+1 are in flight, the descriptor of i+2 is being loaded and the index of i+3 is being fetched.
-  if (warp == CNW) {
+  // ======================= producer warps =======================
+  // One thread per consumer group hands out work and keeps that group's copies going.  The first
+  // three items of every producer are dealt statically; from then on a global counter hands them out.
+  // A look-ahead pipeline keeps the global round trips of the work queue off the critical path: while
+  // the group processes context i, the descriptor of i+1 is in registers, that of i+2 is being loaded
+  // and the index of i+3 is being fetched.  The rows of i+1 are copied as soon as the group releases
+  // its staging area.
+  if (tid >= NGRP * GT) {
+    const int grp = (tid - NGRP * GT) >> 5;
     if (lane == 0) {
+      GroupShared& S = SG[grp];
       const int n_heavy = P.counters->n_heavy;
       const int total = n_heavy + P.counters->n_light;
       const int cap = P.B * N;
-      const int G = gridDim.x;
+      const int G = gridDim.x * NGRP;              // producers in the grid
+      const int me = blockIdx.x * NGRP + grp;
       auto load_item = [&](int w) -> WorkItem {
         WorkItem it;
         it.item = -1;
@@ -179,23 +196,22 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
         }
         return it;
       };
-      WorkItem it_cur = load_item(blockIdx.x);
-      WorkItem it_next = load_item(blockIdx.x + G);
-      int w_next2 = blockIdx.x + 2 * G;
+      WorkItem it_cur = load_item(me);
+      WorkItem it_next = load_item(me + G);
+      int w_next2 = me + 2 * G;
       for (int i = 0;; ++i) {
-        const int slot = i & 1;
-        // the slot is free once every consumer warp has finished the context that used it
-        if (i >= 2 && !mbar_wait(&bar_empty[slot], ((i >> 1) - 1) & 1)) {
+        // the staging area is free once every warp of the group has finished the previous context
+        if (i >= 1 && !mbar_wait(&bar_empty[grp], (i - 1) & 1)) {
           it_cur.item = -1;
-          it_cur.pad = LANTERN_ST_INTERNAL;   // a consumer never released the slot: stop handing out work
+          it_cur.pad = LANTERN_ST_INTERNAL;   // the group never released its area: stop handing out work
         }
-        S.work[slot] = it_cur;                // published by the mbarrier operation below
+        S.work = it_cur;                      // published by the mbarrier operation below
         if (it_cur.item < 0) {
-          mbar_arrive(&bar_full[slot]);       // wake the consumers; they see the terminator
+          mbar_arrive(&bar_full[grp]);        // wake the group; it sees the terminator
           break;
         }
         fence_proxy_async();
-        ctx_issue_rows<BF16, UNC>(P, it_cur.item, smem + slot * stage_bytes, rowbytes, &bar_full[slot]);
+        ctx_issue_rows<BF16, UNC>(P, it_cur.item, smem + grp * stage_bytes, rowbytes, &bar_full[grp]);
         it_cur = it_next;
         it_next = load_item(w_next2);
         w_next2 = 3 * G + atomicAdd(&P.counters->work_next, 1);
@@ -204,194 +220,217 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
     return;
   }
 
-  // ======================= consumer warps =======================
+  // ======================= consumer groups =======================
+  const int grp = tid >> LOG_GT;        // which group
+  const int gt = tid & (GT - 1);        // thread within the group
+  const int gw = gt >> 5;               // warp within the group
+  GroupShared& S = SG[grp];
+  unsigned char* stage = smem + grp * stage_bytes;    // this group's rows, later its E
+  float* E = reinterpret_cast<float*>(stage);
+  // staging rows: 0 = conditional target, 1 = unconditional target (if any), 2 = drafter
+  const unsigned char* rc = stage;
+  const unsigned char* ru = stage + rowbytes;
+  unsigned char* rd = stage + 2 * rowbytes;
+  const bool T_is_one = P.T == 1.0f;
+  // eight processed drafter logits of 16-byte group g (z_p = l_d / T)
+  auto draft_chunk = [&](int g, float (&out)[8]) {
+    if (BF16) {
+      const uint4 d = *reinterpret_cast<const uint4*>(rd + g * 16);
+      const uint32_t dw[4] = {d.x, d.y, d.z, d.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        out[2 * i] = __uint_as_float(dw[i] << 16);
+        out[2 * i + 1] = __uint_as_float(dw[i] & 0xffff0000u);
+      }
+    } else {
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const float4 d = *reinterpret_cast<const float4*>(rd + g * 32 + h * 16);
+        out[4 * h] = d.x, out[4 * h + 1] = d.y, out[4 * h + 2] = d.z, out[4 * h + 3] = d.w;
+      }
+    }
+    if (!T_is_one) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) out[e] = __fdiv_rn(out[e], P.T);
+    }
+  };
+  // eight processed target logits of 16-byte group g (guidance combine, temperature)
+  auto target_chunk = [&](int g, float (&out)[8]) {
+    float lc[8], lu[8];
+    if (BF16) {
+      const uint4 x = *reinterpret_cast<const uint4*>(rc + g * 16);
+      const uint32_t xw[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        lc[2 * i] = __uint_as_float(xw[i] << 16);
+        lc[2 * i + 1] = __uint_as_float(xw[i] & 0xffff0000u);
+      }
+      if (UNC) {
+        const uint4 y = *reinterpret_cast<const uint4*>(ru + g * 16);
+        const uint32_t yw[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          lu[2 * i] = __uint_as_float(yw[i] << 16);
+          lu[2 * i + 1] = __uint_as_float(yw[i] & 0xffff0000u);
+        }
+      }
+    } else {
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const float4 x = *reinterpret_cast<const float4*>(rc + g * 32 + h * 16);
+        lc[4 * h] = x.x, lc[4 * h + 1] = x.y, lc[4 * h + 2] = x.z, lc[4 * h + 3] = x.w;
+        if (UNC) {
+          const float4 y = *reinterpret_cast<const float4*>(ru + g * 32 + h * 16);
+          lu[4 * h] = y.x, lu[4 * h + 1] = y.y, lu[4 * h + 2] = y.z, lu[4 * h + 3] = y.w;
+        }
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      float l = lc[e];
+      if (UNC) l = __fmaf_rn(P.cfg_scale, __fsub_rn(lc[e], lu[e]), lu[e]);   // l_u + s (l_c - l_u)
+      if (!T_is_one) l = __fdiv_rn(l, P.T);
+      out[e] = l;
+    }
+  };
+
   for (int iter = 0;; ++iter) {
-    const int slot_cur = iter & 1;
-    // One warp watches the copy's mbarrier (bounded wait); the consumer barrier then releases everybody
+    // One warp watches the copy's mbarrier (bounded wait); the group barrier then releases everybody
     // at once and tells every thread alike whether the rows have landed.
     bool landed = true;
-    if (warp == 0) landed = mbar_wait(&bar_full[slot_cur], (iter >> 1) & 1);
-    const bool arrived = cbar_and(landed);
+    if (gw == 0) landed = mbar_wait(&bar_full[grp], iter & 1);
+    const bool arrived = gbar_and(grp, landed);
     if (!arrived) break;   // the copy did not land within the limit; the walk reports the missing record
-    const WorkItem cur = S.work[slot_cur];
+    const WorkItem cur = S.work;
     const int item = cur.item;
     if (item < 0) break;
-    unsigned char* stage = smem + slot_cur * stage_bytes;    // this context's rows, later its E
-    float* E = reinterpret_cast<float*>(stage);
     const int b = item / R;
     const ChildInfo* kids = P.children + cur.cbase;
     const int nchild = cur.nchild;
-    // every consumer is past the previous context (its record included): clear the shared status word;
-    // nobody sets it again before the [stats] barrier below
-    if (tid == 0) S.status = 0;
+    // every thread of the group is past the previous context (its record included): clear the shared
+    // status word; nobody sets it again before the [stats] barrier below
+    if (gt == 0) S.status = 0;
 
-    // first child: its neighbour row (two slots per thread) and, for thread 0, its raw logits; issued
-    // now, used after the streaming pass
+    // first child: its neighbour row (four slots per thread) and, for thread 0, its raw logits; issued
+    // now, used after the streaming part
     int node = cur.node0;
     int xt = cur.tok0;
     float r = cur.r0;
-    const int j0 = 2 * tid + 1, j1 = 2 * tid + 2;
-    int n0 = (j0 < k) ? ld_nc_here(P.nbr + static_cast<size_t>(xt) * k + j0) : -1;
-    int n1 = (j1 < k) ? ld_nc_here(P.nbr + static_cast<size_t>(xt) * k + j1) : -1;
+    int nb[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int j = 4 * gt + 1 + i;
+      nb[i] = (j < k) ? ld_nc_here(P.nbr + static_cast<size_t>(xt) * k + j) : -1;
+    }
     float raw_c = 0.0f, raw_u = 0.0f, raw_d = 0.0f;
-    if (tid == 0) {
+    if (gt == 0) {
       const size_t e = static_cast<size_t>(item) * V + xt;
       raw_c = ctx_raw_logit<BF16>(P.target, e);
       if (UNC) raw_u = ctx_raw_logit<BF16>(P.target, static_cast<size_t>(P.B) * R * V + e);
       raw_d = ctx_raw_logit<BF16>(P.draft, e);
     }
 
-    // ---------------- streaming pass, warp-local ----------------
-    // staging rows: 0 = conditional target, 1 = unconditional target (if any), 2 = drafter
-    const unsigned char* rc = stage;
-    const unsigned char* ru = stage + rowbytes;
-    unsigned char* rd = stage + 2 * rowbytes;
-    const float Tinv_is_one = P.T == 1.0f;
-    // eight processed drafter logits of 16-byte group g (z_p = l_d / T)
-    auto draft_chunk = [&](int g, float (&out)[8]) {
-      if (BF16) {
-        const uint4 d = *reinterpret_cast<const uint4*>(rd + g * 16);
-        const uint32_t dw[4] = {d.x, d.y, d.z, d.w};
+    // ---------------- streaming part, warp-local, NP passes of CP chunks ----------------
+    float a[CP * 8];
+    float mlp_mine[NP];                 // this thread's drafter shift constants (needed again on rejection)
+    // --- target: guidance combine, slice maximum, numerators, partial sum; E replaces the raw rows ---
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          out[2 * i] = __uint_as_float(dw[i] << 16);
-          out[2 * i + 1] = __uint_as_float(dw[i] & 0xffff0000u);
-        }
-      } else {
+    for (int p = 0; p < NP; ++p) {
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const float4 d = *reinterpret_cast<const float4*>(rd + g * 32 + h * 16);
-          out[4 * h] = d.x, out[4 * h + 1] = d.y, out[4 * h + 2] = d.z, out[4 * h + 3] = d.w;
-        }
-      }
-      if (!Tinv_is_one) {
-#pragma unroll
-        for (int e = 0; e < 8; ++e) out[e] = __fdiv_rn(out[e], P.T);
-      }
-    };
-    float a[CH * 8];
-    // --- target: guidance combine, warp maximum, numerators, partial sum; E replaces the raw rows ---
-    {
-      const float s = P.cfg_scale;
-#pragma unroll
-      for (int c = 0; c < CH; ++c) {
-        const int g = c * CNT + tid;
+      for (int c = 0; c < CP; ++c) {
+        const int g = (p * CP + c) * GT + gt;
+        float v8[8];
         if (g * 8 < V) {
-          float lc[8], lu[8];
-          if (BF16) {
-            const uint4 x = *reinterpret_cast<const uint4*>(rc + g * 16);
-            const uint32_t xw[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              lc[2 * i] = __uint_as_float(xw[i] << 16);
-              lc[2 * i + 1] = __uint_as_float(xw[i] & 0xffff0000u);
-            }
-            if (UNC) {
-              const uint4 y = *reinterpret_cast<const uint4*>(ru + g * 16);
-              const uint32_t yw[4] = {y.x, y.y, y.z, y.w};
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                lu[2 * i] = __uint_as_float(yw[i] << 16);
-                lu[2 * i + 1] = __uint_as_float(yw[i] & 0xffff0000u);
-              }
-            }
-          } else {
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-              const float4 x = *reinterpret_cast<const float4*>(rc + g * 32 + h * 16);
-              lc[4 * h] = x.x, lc[4 * h + 1] = x.y, lc[4 * h + 2] = x.z, lc[4 * h + 3] = x.w;
-              if (UNC) {
-                const float4 y = *reinterpret_cast<const float4*>(ru + g * 32 + h * 16);
-                lu[4 * h] = y.x, lu[4 * h + 1] = y.y, lu[4 * h + 2] = y.z, lu[4 * h + 3] = y.w;
-              }
-            }
-          }
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            float l = lc[e];
-            if (UNC) l = __fmaf_rn(s, __fsub_rn(lc[e], lu[e]), lu[e]);   // l_u + s (l_c - l_u)
-            if (!Tinv_is_one) l = __fdiv_rn(l, P.T);
-            a[c * 8 + e] = l;
-          }
+          target_chunk(g, v8);
         } else {
 #pragma unroll
-          for (int e = 0; e < 8; ++e) a[c * 8 + e] = ninf;
+          for (int e = 0; e < 8; ++e) v8[e] = ninf;
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) a[c * 8 + e] = v8[e];
+      }
+      float mq = a[0];
+#pragma unroll
+      for (int i = 1; i < CP * 8; ++i) mq = fmaxf(mq, a[i]);
+      // a slice without any finite logit (padding, masked tokens) still needs a finite shift
+      mq = fmaxf(warp_max(mq), -1.0e37f);
+      const float mlq_w = mq * L_hi;
+      float tq = 0.0f;
+#pragma unroll
+      for (int c = 0; c < CP; ++c) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) a[c * 8 + e] = ex2_approx(__fmaf_rn(a[c * 8 + e], L_hi, -mlq_w));
+        tq += sum8(&a[c * 8]);
+        const int g = (p * CP + c) * GT + gt;
+        if (g * 8 < V) {
+          *reinterpret_cast<float4*>(E + EI(g * 8)) = make_float4(a[c * 8], a[c * 8 + 1], a[c * 8 + 2], a[c * 8 + 3]);
+          *reinterpret_cast<float4*>(E + EI(g * 8 + 4)) =
+              make_float4(a[c * 8 + 4], a[c * 8 + 5], a[c * 8 + 6], a[c * 8 + 7]);
         }
       }
-    }
-    float mq = a[0];
-#pragma unroll
-    for (int i = 1; i < CH * 8; ++i) mq = fmaxf(mq, a[i]);
-    // a slice without any finite logit (padding, masked tokens) still needs a finite shift
-    mq = fmaxf(warp_max(mq), -1.0e37f);
-    const float mlq_w = mq * L_hi;
-    float tq = 0.0f;
-#pragma unroll
-    for (int c = 0; c < CH; ++c) {
-#pragma unroll
-      for (int e = 0; e < 8; ++e) a[c * 8 + e] = ex2_approx(__fmaf_rn(a[c * 8 + e], L_hi, -mlq_w));
-      tq += sum8(&a[c * 8]);
-      const int g = c * CNT + tid;
-      if (g * 8 < V) {
-        *reinterpret_cast<float4*>(E + EI(g * 8)) = make_float4(a[c * 8], a[c * 8 + 1], a[c * 8 + 2], a[c * 8 + 3]);
-        *reinterpret_cast<float4*>(E + EI(g * 8 + 4)) =
-            make_float4(a[c * 8 + 4], a[c * 8 + 5], a[c * 8 + 6], a[c * 8 + 7]);
-      }
-    }
-    // --- drafter: warp maximum and partial sum of numerators; the raw row stays in shared memory ---
-#pragma unroll
-    for (int c = 0; c < CH; ++c) {
-      const int g = c * CNT + tid;
-      float d8[8];
-      if (g * 8 < V) {
-        draft_chunk(g, d8);
-      } else {
-#pragma unroll
-        for (int e = 0; e < 8; ++e) d8[e] = ninf;
-      }
-#pragma unroll
-      for (int e = 0; e < 8; ++e) a[c * 8 + e] = d8[e];
-    }
-    float mp = a[0];
-#pragma unroll
-    for (int i = 1; i < CH * 8; ++i) mp = fmaxf(mp, a[i]);
-    mp = fmaxf(warp_max(mp), -1.0e37f);
-    const float mlp_w = mp * L_hi;
-    float tp = 0.0f;
-#pragma unroll
-    for (int c = 0; c < CH; ++c) {
-#pragma unroll
-      for (int e = 0; e < 8; ++e) a[c * 8 + e] = ex2_approx(__fmaf_rn(a[c * 8 + e], L_hi, -mlp_w));
-      tp += sum8(&a[c * 8]);
-    }
-    {
       const double wq = warp_sum(static_cast<double>(tq));
+      if (lane == 0) {
+        S.sq[p * GW + gw] = wq;
+        S.mlq[p * GW + gw] = mlq_w;
+      }
+    }
+    // --- drafter: slice maximum and partial sum of numerators; the raw row stays in shared memory ---
+#pragma unroll
+    for (int p = 0; p < NP; ++p) {
+#pragma unroll
+      for (int c = 0; c < CP; ++c) {
+        const int g = (p * CP + c) * GT + gt;
+        float v8[8];
+        if (g * 8 < V) {
+          draft_chunk(g, v8);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 8; ++e) v8[e] = ninf;
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) a[c * 8 + e] = v8[e];
+      }
+      float mp = a[0];
+#pragma unroll
+      for (int i = 1; i < CP * 8; ++i) mp = fmaxf(mp, a[i]);
+      mp = fmaxf(warp_max(mp), -1.0e37f);
+      const float mlp_w = mp * L_hi;
+      mlp_mine[p] = mlp_w;
+      float tp = 0.0f;
+#pragma unroll
+      for (int c = 0; c < CP; ++c) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) a[c * 8 + e] = ex2_approx(__fmaf_rn(a[c * 8 + e], L_hi, -mlp_w));
+        tp += sum8(&a[c * 8]);
+      }
       const double wp = warp_sum(static_cast<double>(tp));
       if (lane == 0) {
-        S.sq[warp] = wq;
-        S.sp[warp] = wp;
-        S.mlq[warp] = mlq_w;
-        S.mlp[warp] = mlp_w;
+        S.sp[p * GW + gw] = wp;
+        S.mlp[p * GW + gw] = mlp_w;
       }
     }
+    gbar(grp);   // [stats] per-slice maxima and sums, and E, are visible
 
-    cbar();   // [stats] per-warp maxima and sums, and E, are visible
-
-    // ---------------- block statistics, computed by every warp for itself ----------------
-    float fq_l, fp_l;            // lane l holds the factor that brings warp l's units to global units
+    // ---------------- group statistics, computed by every warp for itself ----------------
+    float fq_l, fp_l;            // lane u holds the factor that brings slice u's units to common units
     double Zq, Zp;
     float mlq_g, mlp_g;
     {
-      const float mq_l = lane < CNW ? S.mlq[lane] : ninf;
-      const float mp_l = lane < CNW ? S.mlp[lane] : ninf;
+      const float mq_l = lane < NU ? S.mlq[lane] : ninf;
+      const float mp_l = lane < NU ? S.mlp[lane] : ninf;
       mlq_g = warp_max(mq_l);
       mlp_g = warp_max(mp_l);
       fq_l = ex2_approx(mq_l - mlq_g);
       fp_l = ex2_approx(mp_l - mlp_g);
-      Zq = warp_sum(lane < CNW ? static_cast<double>(fq_l) * S.sq[lane] : 0.0);
-      Zp = warp_sum(lane < CNW ? static_cast<double>(fp_l) * S.sp[lane] : 0.0);
+      Zq = warp_sum(lane < NU ? static_cast<double>(fq_l) * S.sq[lane] : 0.0);
+      Zp = warp_sum(lane < NU ? static_cast<double>(fp_l) * S.sp[lane] : 0.0);
     }
-    const float fq_mine = __shfl_sync(kFull, fq_l, warp), fp_mine = __shfl_sync(kFull, fp_l, warp);
+    float fq_mine[NP], fp_mine[NP];
+#pragma unroll
+    for (int p = 0; p < NP; ++p) {
+      fq_mine[p] = __shfl_sync(kFull, fq_l, p * GW + gw);
+      fp_mine[p] = __shfl_sync(kFull, fp_l, p * GW + gw);
+    }
 
     int status = 0;              // bits every thread sets alike
     int accepted = -1;
@@ -399,14 +438,14 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
     if (!(Zq > 0.0 && Zq < 1e300 && Zp > 0.0 && Zp < 1e300)) {
       status |= LANTERN_ST_NONFINITE;
     } else {
-      double qscale = 1.0 / Zq;     // q'(x) = E(x) * fq[warp of x] * qscale
-      double pscale = 1.0 / Zp;     // p'(x) = ep(x) * fp[warp of x] * pscale
+      double qscale = 1.0 / Zq;     // q'(x) = E(x) * fq[slice of x] * qscale
+      double pscale = 1.0 / Zp;     // p'(x) = ep(x) * fp[slice of x] * pscale
       const double delta = static_cast<double>(P.delta);
-      if (tid == 0) {   // the two single probabilities of the first child, in double precision
+      if (gt == 0) {   // the two single probabilities of the first child, in double precision
         float zq = raw_c;
         if (UNC) zq = __fmaf_rn(P.cfg_scale, __fsub_rn(raw_c, raw_u), raw_u);
         float zp = raw_d;
-        if (P.T != 1.0f) {
+        if (!T_is_one) {
           zq = __fdiv_rn(zq, P.T);
           zp = __fdiv_rn(zp, P.T);
         }
@@ -423,58 +462,67 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
           const int4 v = __ldg(reinterpret_cast<const int4*>(kids + ci + 1));
           sib.node = v.x, sib.token = v.y, sib.r = __int_as_float(v.z);
         }
-        // drafter numerator of x~ from the raw row (-inf, hence 0, once x~ has been rejected), global units
-        float px_bulk;
+        // bulk numerators of x~ itself, common units (drafter: from the raw row, -inf once x~ was rejected)
+        float px_bulk, e_xt_bulk;
         {
+          const int ou = owner_unit<LOG_CP>(xt);
           float dz = BF16 ? __uint_as_float(static_cast<uint32_t>(reinterpret_cast<const unsigned short*>(rd)[xt]) << 16)
                           : reinterpret_cast<const float*>(rd)[xt];
-          if (!Tinv_is_one) dz = __fdiv_rn(dz, P.T);
-          const int ow = cowner_thread(xt) >> 5;
-          px_bulk = ex2_approx(__fmaf_rn(dz, L_hi, -S.mlp[ow])) * __shfl_sync(kFull, fp_l, ow);
+          if (!T_is_one) dz = __fdiv_rn(dz, P.T);
+          px_bulk = ex2_approx(__fmaf_rn(dz, L_hi, -S.mlp[ou])) * __shfl_sync(kFull, fp_l, ou);
+          e_xt_bulk = E[EI(xt)] * __shfl_sync(kFull, fq_l, ou);
         }
-        const float e_xt_bulk = E[EI(xt)] * __shfl_sync(kFull, fq_l, cowner_thread(xt) >> 5);
 
         // ---- A_{k,delta}(x~): gather + prefix scan with the strict bound ----
         const double thr = delta / qscale;   // the bound in the units of the unnormalised sums
         double carry = 0.0, sm = 0.0;
         int m = k - 1;
         bool cut = false;
-        for (int base = 0; base < k - 1 && !cut; base += 2 * CNT) {
-          const int ja = base + j0, jb = base + j1;
-          const bool va = ja < k, vb = jb < k;
-          const int na = base == 0 ? n0 : (va ? __ldg(nrow + ja) : -1);
-          const int nb = base == 0 ? n1 : (vb ? __ldg(nrow + jb) : -1);
-          const bool ia = va && static_cast<unsigned>(na) < static_cast<unsigned>(V);
-          const bool ib = vb && static_cast<unsigned>(nb) < static_cast<unsigned>(V);
-          if ((va && !ia) || (vb && !ib)) atomicOr(&S.status, LANTERN_ST_BAD_TABLE);   // carries no mass
-          const float fa = __shfl_sync(kFull, fq_l, ia ? cowner_thread(na) >> 5 : 0);
-          const float fb = __shfl_sync(kFull, fq_l, ib ? cowner_thread(nb) >> 5 : 0);
-          const double da = ia ? static_cast<double>(E[EI(na)] * fa) : 0.0;
-          const double db = ib ? static_cast<double>(E[EI(nb)] * fb) : 0.0;
-          const double incl = warp_incl_scan(da + db, lane);
-          if (lane == 31) S.wt[warp] = incl;
-          cbar();   // [scan 1]
+        for (int base = 0; base < k - 1 && !cut; base += 4 * GT) {
+          double pre4[4];       // inclusive prefix over this thread's four slots
+          bool val4[4];
+          double run = 0.0;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int j = base + 4 * gt + 1 + i;
+            val4[i] = j < k;
+            const int n = base == 0 ? nb[i] : (val4[i] ? __ldg(nrow + j) : -1);
+            const bool inr = val4[i] && static_cast<unsigned>(n) < static_cast<unsigned>(V);
+            if (val4[i] && !inr) atomicOr(&S.status, LANTERN_ST_BAD_TABLE);   // carries no mass
+            const float f = __shfl_sync(kFull, fq_l, inr ? owner_unit<LOG_CP>(n) : 0);
+            run += inr ? static_cast<double>(E[EI(n)] * f) : 0.0;
+            pre4[i] = run;
+          }
+          const double incl = warp_incl_scan(run, lane);
+          if (lane == 31) S.wt[gw] = incl;
+          gbar(grp);   // [scan 1]
           double pre, tot;
           {
-            const double t = lane < CNW ? S.wt[lane] : 0.0;
+            const double t = lane < GW ? S.wt[lane] : 0.0;
             const double in = warp_incl_scan(t, lane);
-            pre = __shfl_sync(kFull, in - t, warp);
-            tot = __shfl_sync(kFull, in, CNW - 1);
+            pre = __shfl_sync(kFull, in - t, gw);
+            tot = __shfl_sync(kFull, in, GW - 1);
           }
-          const double Sb = carry + pre + incl;          // inclusive prefix at slot jb
-          const double Sa = Sb - db;                      // at slot ja
-          const bool faila = va && !(Sa < thr);
-          const bool failb = vb && !(Sb < thr);
-          const int my_first = faila ? ja : (failb ? jb : kNone);
+          const double before = carry + pre + (incl - run);   // prefix before this thread's first slot
+          int my_first = kNone;
+          double my_before = 0.0;
+#pragma unroll
+          for (int i = 3; i >= 0; --i) {
+            const double Sj = before + pre4[i];
+            if (val4[i] && !(Sj < thr)) {
+              my_first = base + 4 * gt + 1 + i;
+              my_before = i > 0 ? before + pre4[i > 0 ? i - 1 : 0] : before;
+            }
+          }
           const int wfirst = __reduce_min_sync(kFull, my_first);
           if (wfirst != kNone && my_first == wfirst) {
-            S.first[warp] = wfirst;
-            S.sbefore[warp] = faila ? Sa - da : Sa;
+            S.first[gw] = wfirst;
+            S.sbefore[gw] = my_before;
           } else if (wfirst == kNone && lane == 0) {
-            S.first[warp] = kNone;
+            S.first[gw] = kNone;
           }
-          cbar();   // [scan 2]
-          const int f_l = lane < CNW ? S.first[lane] : kNone;
+          gbar(grp);   // [scan 2]
+          const int f_l = lane < GW ? S.first[lane] : kNone;
           const int gfirst = __reduce_min_sync(kFull, f_l);
           if (gfirst != kNone) {
             const int src = __ffs(__ballot_sync(kFull, f_l == gfirst)) - 1;
@@ -486,17 +534,16 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
             sm = carry;
           }
         }
-        if (k == 1) cbar();   // publish S.acc_* when the scan loop did not run
+        if (k == 1) gbar(grp);   // publish S.acc_* when the scan loop did not run
         // the two single probabilities: thread 0's double-precision values where it has them; a bulk
         // value of exactly zero (token inside an earlier A, or rejected before) stays zero
         const bool acc = S.acc_valid != 0;
-        const float pxb = px_bulk;
         const double e_xt = (acc && e_xt_bulk != 0.0f) ? S.acc_e : static_cast<double>(e_xt_bulk);
-        const double p_xt = (acc && pxb != 0.0f) ? S.acc_p : static_cast<double>(pxb);
+        const double p_xt = (acc && px_bulk != 0.0f) ? S.acc_p : static_cast<double>(px_bulk);
         const double qa = (e_xt + sm) * qscale;
         const double px = p_xt * pscale;
         const bool accept = static_cast<double>(r) * px < qa;   // Section 4.3: min(1, sum_A q / p(x~))
-        if (tid == 0) {
+        if (gt == 0) {
           const size_t o = static_cast<size_t>(b) * N + node;
           if (P.out_qa) P.out_qa[o] = static_cast<float>(qa);
           if (P.out_px) P.out_px[o] = static_cast<float>(px);
@@ -508,19 +555,19 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
         }
         // ---- rejected: residual [q_{k,delta}(.|D = x~) - p]_+ ----
         // members of A (x~ included) leave no residual mass: flag them with a negative sign
-        for (int base = 0; base < m; base += 2 * CNT) {
-          const int ja = base + j0, jb = base + j1;
-          if (ja <= m) {
-            const int n = base == 0 ? n0 : __ldg(nrow + ja);
-            if (static_cast<unsigned>(n) < static_cast<unsigned>(V)) E[EI(n)] = -fabsf(E[EI(n)]);
-          }
-          if (jb <= m) {
-            const int n = base == 0 ? n1 : __ldg(nrow + jb);
-            if (static_cast<unsigned>(n) < static_cast<unsigned>(V)) E[EI(n)] = -fabsf(E[EI(n)]);
+        for (int base = 0; base < m; base += 4 * GT) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int j = base + 4 * gt + 1 + i;
+            if (j <= m) {
+              const int n = base == 0 ? nb[i] : __ldg(nrow + j);
+              if (static_cast<unsigned>(n) < static_cast<unsigned>(V)) E[EI(n)] = -fabsf(E[EI(n)]);
+            }
           }
         }
-        if (tid == 0) E[EI(xt)] = -fabsf(E[EI(xt)]);
-        if (tid == 0) {   // x~ leaves the drafter distribution for the following siblings
+        if (gt == 0) {
+          E[EI(xt)] = -fabsf(E[EI(xt)]);
+          // x~ leaves the drafter distribution for the following siblings
           if (BF16) reinterpret_cast<unsigned short*>(rd)[xt] = 0xff80;   // -inf
           else reinterpret_cast<float*>(rd)[xt] = ninf;
         }
@@ -529,79 +576,82 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
           node = sib.node;
           xt = sib.token;
           r = sib.r;
-          n0 = (j0 < k) ? ld_nc_here(P.nbr + static_cast<size_t>(xt) * k + j0) : -1;
-          n1 = (j1 < k) ? ld_nc_here(P.nbr + static_cast<size_t>(xt) * k + j1) : -1;
-          if (tid == 0) {   // its raw logits, for the double-precision replay below
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int j = 4 * gt + 1 + i;
+            nb[i] = (j < k) ? ld_nc_here(P.nbr + static_cast<size_t>(xt) * k + j) : -1;
+          }
+          if (gt == 0) {   // its raw logits, for the double-precision replay below
             const size_t e = static_cast<size_t>(item) * V + xt;
             raw_c = ctx_raw_logit<BF16>(P.target, e);
             if (UNC) raw_u = ctx_raw_logit<BF16>(P.target, static_cast<size_t>(P.B) * R * V + e);
             raw_d = ctx_raw_logit<BF16>(P.draft, e);
           }
         }
-        cbar();   // [flags]
-        // w = E - (p'/q' scale ratio) * ep, in this warp's own units of E
-        const float ratio = static_cast<float>((pscale * static_cast<double>(fp_mine)) /
-                                               (qscale * static_cast<double>(fq_mine)));
+        gbar(grp);   // [flags]
+        // w = E - (p'/q' scale ratio) * ep in common units, i.e. E - ratio * ep in the slice's own units
+        // of E; the residual replaces E (it is the next sibling's target, or what the draw reads)
+        const float ratio_g = static_cast<float>(pscale / qscale);
         float cs[CH];
-        float wsum = 0.0f, psum = 0.0f;
+        double wsum = 0.0, psum = 0.0;
 #pragma unroll
-        for (int c = 0; c < CH; ++c) {
-          const int g = c * CNT + tid;
-          if (g * 8 < V) {
-            const float4 lo = *reinterpret_cast<const float4*>(E + EI(g * 8));
-            const float4 hi = *reinterpret_cast<const float4*>(E + EI(g * 8 + 4));
-            const float e8[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
-            float ep8[8];
-            draft_chunk(g, ep8);
+        for (int p = 0; p < NP; ++p) {
+          // (a slice whose numerators are all negligible has factor 0; nothing of it survives anyway)
+          const float ratio = fq_mine[p] > 0.0f ? ratio_g * (fp_mine[p] / fq_mine[p]) : 0.0f;
+          float wp_ = 0.0f, pp_ = 0.0f;
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              ep8[e] = ex2_approx(__fmaf_rn(ep8[e], L_hi, -mlp_w));
-              a[c * 8 + e] = fmaxf(0.0f, __fmaf_rn(-ratio, ep8[e], e8[e]));
+          for (int c = 0; c < CP; ++c) {
+            const int g = (p * CP + c) * GT + gt;
+            float w8[8];
+            if (g * 8 < V) {
+              const float4 lo = *reinterpret_cast<const float4*>(E + EI(g * 8));
+              const float4 hi = *reinterpret_cast<const float4*>(E + EI(g * 8 + 4));
+              const float e8[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+              float ep8[8];
+              draft_chunk(g, ep8);
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                ep8[e] = ex2_approx(__fmaf_rn(ep8[e], L_hi, -mlp_mine[p]));
+                w8[e] = fmaxf(0.0f, __fmaf_rn(-ratio, ep8[e], e8[e]));
+              }
+              pp_ += sum8(ep8);
+              *reinterpret_cast<float4*>(E + EI(g * 8)) = make_float4(w8[0], w8[1], w8[2], w8[3]);
+              *reinterpret_cast<float4*>(E + EI(g * 8 + 4)) = make_float4(w8[4], w8[5], w8[6], w8[7]);
+            } else {
+#pragma unroll
+              for (int e = 0; e < 8; ++e) w8[e] = 0.0f;
             }
-            psum += sum8(ep8);
-          } else {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) a[c * 8 + e] = 0.0f;
+            cs[p * CP + c] = sum8(w8);
+            wp_ += cs[p * CP + c];
           }
-          cs[c] = sum8(&a[c * 8]);
-          wsum += cs[c];
+          wsum += static_cast<double>(wp_) * static_cast<double>(fq_mine[p]);
+          psum += static_cast<double>(pp_) * static_cast<double>(fp_mine[p]);
         }
-        const double fqd = static_cast<double>(fq_mine);
         double W, Sp;
         if (!last) {
-          // only the totals are needed; the residual becomes the next sibling's target
-#pragma unroll
-          for (int c = 0; c < CH; ++c) {
-            const int g = c * CNT + tid;
-            if (g * 8 < V) {
-              *reinterpret_cast<float4*>(E + EI(g * 8)) = make_float4(a[c * 8], a[c * 8 + 1], a[c * 8 + 2], a[c * 8 + 3]);
-              *reinterpret_cast<float4*>(E + EI(g * 8 + 4)) =
-                  make_float4(a[c * 8 + 4], a[c * 8 + 5], a[c * 8 + 6], a[c * 8 + 7]);
-            }
-          }
-          const double ww = warp_sum(static_cast<double>(wsum) * fqd);
-          const double wp = warp_sum(static_cast<double>(psum) * static_cast<double>(fp_mine));
+          const double ww = warp_sum(wsum);
+          const double wp = warp_sum(psum);
           if (lane == 0) {
-            S.wt[warp] = ww;
-            S.wt[CNW + warp] = wp;
+            S.wt[gw] = ww;
+            S.wt[GW + gw] = wp;
           }
-          cbar();   // [totals] also publishes the written-back residual
-          W = warp_sum(lane < CNW ? S.wt[lane] : 0.0);
-          Sp = warp_sum(lane < CNW ? S.wt[CNW + lane] : 0.0);
+          gbar(grp);   // [totals] also publishes the written-back residual
+          W = warp_sum(lane < GW ? S.wt[lane] : 0.0);
+          Sp = warp_sum(lane < GW ? S.wt[GW + lane] : 0.0);
           if (!(W > 0.0)) {
             status |= LANTERN_ST_DEGENERATE;
             break;
           }
-          if (tid == 0) {
+          if (gt == 0) {
             // The next sibling's own two probabilities in double precision: its numerators from the raw
             // logits, carried through every rejection round so far (E <- max(0, E - ratio_i * ep)); the
-            // block totals W, Sp are sums of thousands of terms and do not suffer from cancellation.
+            // totals W, Sp are sums of thousands of terms and do not suffer from cancellation.
             if (ci < 32) {
-              S.hist[ci] = pscale / qscale;
+              S.hist[ci] = static_cast<double>(ratio_g);
               float zq = raw_c;
               if (UNC) zq = __fmaf_rn(P.cfg_scale, __fsub_rn(raw_c, raw_u), raw_u);
               float zp = raw_d;
-              if (P.T != 1.0f) {
+              if (!T_is_one) {
                 zq = __fdiv_rn(zq, P.T);
                 zp = __fdiv_rn(zp, P.T);
               }
@@ -623,23 +673,23 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
         double csd[CH], incl[CH], excl[CH] = {};
 #pragma unroll
         for (int c = 0; c < CH; ++c) {
-          csd[c] = static_cast<double>(cs[c]) * fqd;
+          csd[c] = static_cast<double>(cs[c]) * static_cast<double>(fq_mine[c / CP]);
           incl[c] = warp_incl_scan(csd[c], lane);
-          if (lane == 31) S.wt[c * CNW + warp] = incl[c];
+          if (lane == 31) S.wt[c * GW + gw] = incl[c];
         }
-        cbar();   // [draw 1]
+        gbar(grp);   // [draw 1]
         {
           // exclusive prefix over (chunk, warp) in chunk-major order; 32 entries per round
           double carry2 = 0.0;
 #pragma unroll
-          for (int half = 0; half < (CH * CNW + 31) / 32; ++half) {
+          for (int half = 0; half < (CH * GW + 31) / 32; ++half) {
             const int e = half * 32 + lane;
-            const double t = e < CH * CNW ? S.wt[e] : 0.0;
+            const double t = e < CH * GW ? S.wt[e] : 0.0;
             const double in = warp_incl_scan(t, lane);
             const double ex = carry2 + in - t;
 #pragma unroll
             for (int c = 0; c < CH; ++c) {
-              const int want = c * CNW + warp;
+              const int want = c * GW + gw;
               const double got = __shfl_sync(kFull, ex, want & 31);
               if ((want >> 5) == half) excl[c] = got + incl[c] - csd[c];
             }
@@ -655,58 +705,60 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
         int cand = kNone;
 #pragma unroll
         for (int c = CH - 1; c >= 0; --c)
-          if (excl[c] + csd[c] > target) cand = c * CNT + tid;
+          if (excl[c] + csd[c] > target) cand = c * GT + gt;
         const int wmin = __reduce_min_sync(kFull, cand);
-        if (lane == 0) S.cand[warp] = wmin;
-        if (tid == 0) S.tok = -1;
-        cbar();   // [draw 2]
-        const int win = __reduce_min_sync(kFull, lane < CNW ? S.cand[lane] : kNone);
+        if (lane == 0) S.cand[gw] = wmin;
+        if (gt == 0) S.tok = -1;
+        gbar(grp);   // [draw 2]
+        const int win = __reduce_min_sync(kFull, lane < GW ? S.cand[lane] : kNone);
         if (win == kNone) {
           // rounding left no slot above the target: the largest token of positive weight
           int lastp = -1;
-#pragma unroll
-          for (int c = 0; c < CH; ++c)
-#pragma unroll
-            for (int e = 0; e < 8; ++e)
-              if (a[c * 8 + e] > 0.0f) lastp = (c * CNT + tid) * 8 + e;
-          if (lastp >= V) lastp = -1;
+          for (int c = 0; c < CH; ++c) {
+            const int g = c * GT + gt;
+            if (g * 8 < V && cs[c] > 0.0f)
+              for (int e = 0; e < 8; ++e)
+                if (E[EI(g * 8 + e)] > 0.0f) lastp = g * 8 + e;
+          }
           if (lastp >= 0) atomicMax(&S.tok, lastp);
-          cbar();
-          if (tid == 0) {
+          gbar(grp);
+          if (gt == 0) {
             Record rec = {-1, S.tok, status | S.status | (S.tok < 0 ? LANTERN_ST_DEGENERATE : 0), 0};
             P.records[item] = rec;
           }
-        } else if ((win & (CNT - 1)) == tid) {
-          const int wc = win >> LOG_CNT;
-          int tok = -1, lastpos = -1;
+        } else if ((win & (GT - 1)) == gt) {
+          const int wc = win >> LOG_GT;
+          const int g = wc * GT + gt;
+          double ex_c = 0.0, fqd = 0.0;
 #pragma unroll
-          for (int c = 0; c < CH; ++c) {
+          for (int c = 0; c < CH; ++c)
             if (c == wc) {
-              double cum = excl[c];
-#pragma unroll
-              for (int e = 0; e < 8; ++e) {
-                const float wv = a[c * 8 + e];
-                cum += static_cast<double>(wv) * fqd;
-                if (wv > 0.0f) lastpos = e;
-                if (tok < 0 && cum > target) tok = e;
-              }
+              ex_c = excl[c];
+              fqd = static_cast<double>(fq_mine[c / CP]);
             }
+          int tok = -1, lastpos = -1;
+          double cum = ex_c;
+          for (int e = 0; e < 8; ++e) {
+            const float wv = E[EI(g * 8 + e)];
+            cum += static_cast<double>(wv) * fqd;
+            if (wv > 0.0f) lastpos = e;
+            if (tok < 0 && cum > target) tok = e;
           }
           if (tok < 0) tok = lastpos;
-          Record rec = {-1, win * 8 + tok, status | S.status, 0};
+          Record rec = {-1, g * 8 + tok, status | S.status, 0};
           P.records[item] = rec;
         }
         record_written = true;
       }
     }
-    if (!record_written && tid == 0) {
-      // S.status was last written before a barrier every thread has passed
+    if (!record_written && gt == 0) {
+      // S.status was last written before a barrier every thread of the group has passed
       Record rec = {accepted, -1, status | S.status, 0};
       P.records[item] = rec;
     }
     // this context's staging area (rows and E) is no longer needed by this warp
     __syncwarp();
-    if (lane == 0) mbar_arrive(&bar_empty[slot_cur]);
+    if (lane == 0) mbar_arrive(&bar_empty[grp]);
   }
 }
 

@@ -8,11 +8,13 @@
 // part of one context overlaps the issue-bound streaming part of the other and the copy of a
 // third: the SM is rarely idle although every context is a chain of dependent steps.
 //
-// Streaming part (per warp, on its own slice, in passes of at most 32 tokens per thread):
-// guidance combine, the slice's maximum, numerators 2^((z - max) log2 e) through the hardware
-// ex2 unit, partial sums.  The numerators E are stored over the context's own raw target rows
-// (every thread overwrites only bytes that it alone has read) and stay in the units of their
-// (pass, warp) slice; a per-slice factor brings them to common units when they are used.  Sums
+// Streaming part (per thread, on its own tokens, in passes of at most 32 tokens): guidance
+// combine, the thread's own maximum, numerators 2^((z - max) log2 e) through the hardware ex2
+// unit, partial sums -- no cross-thread step at all, so the warps stream at full rate.  The
+// numerators E are stored over the context's own raw target rows (every thread overwrites only
+// bytes that it alone has read) and stay in the units of their (pass, thread) slice; a
+// per-slice factor, tabulated once the common maximum is known, brings them to common units
+// when they are used.  Sums
 // over many numerators average the ex2 unit's ~1e-7 rounding out; the two single probabilities
 // that decide a position, q(x~) and p(x~), are recomputed by one thread in double precision.
 //
@@ -23,7 +25,7 @@
 // inverse-CDF draw or the write-back for the next sibling.
 #pragma once
 
-#define LANTERN_CONTEXT_KERNEL_REVISION 6   // bump on every change to this file
+#define LANTERN_CONTEXT_KERNEL_REVISION 7   // bump on every change to this file
 
 namespace lantern {
 
@@ -45,20 +47,21 @@ __device__ __forceinline__ int ephys(int x, int row_floats) {
   if (BF16) return ((x >> 2) & 1) * row_floats + ((x >> 3) << 2) + (x & 3);
   return x;
 }
-// (pass, warp) slice that owns token x; LOG_CP = log2(chunks per pass)
+// index of the (pass, thread) slice that owns token x in the factor table; LOG_CP = log2(chunks per pass)
 template <int LOG_CP>
-__device__ __forceinline__ int owner_unit(int x) {
+__device__ __forceinline__ int owner_slice(int x) {
   const int g = x >> 3;
-  return ((g >> (LOG_GT + LOG_CP)) * GW) + ((g & (GT - 1)) >> 5);
+  return ((g >> (LOG_GT + LOG_CP)) << LOG_GT) | (g & (GT - 1));
 }
 
 struct GroupShared {
-  double sq[MAXU], sp[MAXU];    // per-slice sums of numerators, in the slice's own units
+  double wzq[GW], wzp[GW];      // per-warp sums of numerators, common units
   double wt[8 * GW];            // per-(chunk, warp) totals for scans and block sums
   double sbefore[GW];           // prefix sum just before a warp's first failing neighbour
   double acc_e, acc_p;          // double-precision numerators of the tested x~, common units
   double hist[32];              // drafter/target scale ratio of each earlier rejection round of this context
-  float mlq[MAXU], mlp[MAXU];   // per-slice shift constants fl(max * log2 e)
+  float fqt[2 * GT];            // factor of every (pass, thread) slice: its units -> common units
+  float wmq[GW], wmp[GW];       // per-warp maxima of the slices' shift constants
   int first[GW];                // a warp's first failing neighbour slot
   int cand[GW];
   int acc_valid;                // acc_e / acc_p are usable for the current child
@@ -142,7 +145,6 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
   constexpr int NP = CH > 4 ? 2 : 1;          // passes
   constexpr int CP = CH / NP;                 // chunks per pass
   constexpr int LOG_CP = CP == 4 ? 2 : (CP == 2 ? 1 : 0);
-  constexpr int NU = NP * GW;                 // slices with their own units
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ GroupShared SG[NGRP];
   __shared__ __align__(8) uint64_t bar_full[NGRP], bar_empty[NGRP];
@@ -332,7 +334,8 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
 
     // ---------------- streaming part, warp-local, NP passes of CP chunks ----------------
     float a[CP * 8];
-    float mlp_mine[NP];                 // this thread's drafter shift constants (needed again on rejection)
+    float mlq_mine[NP], mlp_mine[NP];   // this thread's shift constants fl(max * log2 e), per pass
+    float tq_mine[NP], tp_mine[NP];     // and its sums of numerators, in its own units
     // --- target: guidance combine, slice maximum, numerators, partial sum; E replaces the raw rows ---
 #pragma unroll
     for (int p = 0; p < NP; ++p) {
@@ -353,8 +356,9 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
 #pragma unroll
       for (int i = 1; i < CP * 8; ++i) mq = fmaxf(mq, a[i]);
       // a slice without any finite logit (padding, masked tokens) still needs a finite shift
-      mq = fmaxf(warp_max(mq), -1.0e37f);
+      mq = fmaxf(mq, -1.0e37f);
       const float mlq_w = mq * L_hi;
+      mlq_mine[p] = mlq_w;
       float tq = 0.0f;
 #pragma unroll
       for (int c = 0; c < CP; ++c) {
@@ -368,11 +372,7 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
               make_float4(a[c * 8 + 4], a[c * 8 + 5], a[c * 8 + 6], a[c * 8 + 7]);
         }
       }
-      const double wq = warp_sum(static_cast<double>(tq));
-      if (lane == 0) {
-        S.sq[p * GW + gw] = wq;
-        S.mlq[p * GW + gw] = mlq_w;
-      }
+      tq_mine[p] = tq;
     }
     // --- drafter: slice maximum and partial sum of numerators; the raw row stays in shared memory ---
 #pragma unroll
@@ -393,7 +393,7 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       float mp = a[0];
 #pragma unroll
       for (int i = 1; i < CP * 8; ++i) mp = fmaxf(mp, a[i]);
-      mp = fmaxf(warp_max(mp), -1.0e37f);
+      mp = fmaxf(mp, -1.0e37f);
       const float mlp_w = mp * L_hi;
       mlp_mine[p] = mlp_w;
       float tp = 0.0f;
@@ -403,33 +403,58 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
         for (int e = 0; e < 8; ++e) a[c * 8 + e] = ex2_approx(__fmaf_rn(a[c * 8 + e], L_hi, -mlp_w));
         tp += sum8(&a[c * 8]);
       }
-      const double wp = warp_sum(static_cast<double>(tp));
-      if (lane == 0) {
-        S.sp[p * GW + gw] = wp;
-        S.mlp[p * GW + gw] = mlp_w;
-      }
+      tp_mine[p] = tp;
     }
-    gbar(grp);   // [stats] per-slice maxima and sums, and E, are visible
 
-    // ---------------- group statistics, computed by every warp for itself ----------------
-    float fq_l, fp_l;            // lane u holds the factor that brings slice u's units to common units
-    double Zq, Zp;
+    // ---------------- group statistics ----------------
+    // common maxima first (one warp reduction, then eight values read by everybody), then the slices'
+    // factors and the normalisers
     float mlq_g, mlp_g;
     {
-      const float mq_l = lane < NU ? S.mlq[lane] : ninf;
-      const float mp_l = lane < NU ? S.mlp[lane] : ninf;
-      mlq_g = warp_max(mq_l);
-      mlp_g = warp_max(mp_l);
-      fq_l = ex2_approx(mq_l - mlq_g);
-      fp_l = ex2_approx(mp_l - mlp_g);
-      Zq = warp_sum(lane < NU ? static_cast<double>(fq_l) * S.sq[lane] : 0.0);
-      Zp = warp_sum(lane < NU ? static_cast<double>(fp_l) * S.sp[lane] : 0.0);
+      float mq_t = mlq_mine[0], mp_t = mlp_mine[0];
+#pragma unroll
+      for (int p = 1; p < NP; ++p) {
+        mq_t = fmaxf(mq_t, mlq_mine[p]);
+        mp_t = fmaxf(mp_t, mlp_mine[p]);
+      }
+      mq_t = warp_max(mq_t);
+      mp_t = warp_max(mp_t);
+      if (lane == 0) {
+        S.wmq[gw] = mq_t;
+        S.wmp[gw] = mp_t;
+      }
+    }
+    gbar(grp);   // [stats 1] per-warp maxima, and E, are visible
+    mlq_g = S.wmq[0];
+    mlp_g = S.wmp[0];
+#pragma unroll
+    for (int w = 1; w < GW; ++w) {
+      mlq_g = fmaxf(mlq_g, S.wmq[w]);
+      mlp_g = fmaxf(mlp_g, S.wmp[w]);
     }
     float fq_mine[NP], fp_mine[NP];
+    double Zq = 0.0, Zp = 0.0;
 #pragma unroll
     for (int p = 0; p < NP; ++p) {
-      fq_mine[p] = __shfl_sync(kFull, fq_l, p * GW + gw);
-      fp_mine[p] = __shfl_sync(kFull, fp_l, p * GW + gw);
+      fq_mine[p] = ex2_approx(mlq_mine[p] - mlq_g);
+      fp_mine[p] = ex2_approx(mlp_mine[p] - mlp_g);
+      S.fqt[p * GT + gt] = fq_mine[p];
+      Zq += static_cast<double>(fq_mine[p]) * static_cast<double>(tq_mine[p]);
+      Zp += static_cast<double>(fp_mine[p]) * static_cast<double>(tp_mine[p]);
+    }
+    Zq = warp_sum(Zq);
+    Zp = warp_sum(Zp);
+    if (lane == 0) {
+      S.wzq[gw] = Zq;
+      S.wzp[gw] = Zp;
+    }
+    gbar(grp);   // [stats 2] factor table and per-warp sums are visible
+    Zq = 0.0;
+    Zp = 0.0;
+#pragma unroll
+    for (int w = 0; w < GW; ++w) {
+      Zq += S.wzq[w];
+      Zp += S.wzp[w];
     }
 
     int status = 0;              // bits every thread sets alike
@@ -465,12 +490,11 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
         // bulk numerators of x~ itself, common units (drafter: from the raw row, -inf once x~ was rejected)
         float px_bulk, e_xt_bulk;
         {
-          const int ou = owner_unit<LOG_CP>(xt);
           float dz = BF16 ? __uint_as_float(static_cast<uint32_t>(reinterpret_cast<const unsigned short*>(rd)[xt]) << 16)
                           : reinterpret_cast<const float*>(rd)[xt];
           if (!T_is_one) dz = __fdiv_rn(dz, P.T);
-          px_bulk = ex2_approx(__fmaf_rn(dz, L_hi, -S.mlp[ou])) * __shfl_sync(kFull, fp_l, ou);
-          e_xt_bulk = E[EI(xt)] * __shfl_sync(kFull, fq_l, ou);
+          px_bulk = ex2_approx(__fmaf_rn(dz, L_hi, -mlp_g));
+          e_xt_bulk = E[EI(xt)] * S.fqt[owner_slice<LOG_CP>(xt)];
         }
 
         // ---- A_{k,delta}(x~): gather + prefix scan with the strict bound ----
@@ -489,19 +513,18 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
             const int n = base == 0 ? nb[i] : (val4[i] ? __ldg(nrow + j) : -1);
             const bool inr = val4[i] && static_cast<unsigned>(n) < static_cast<unsigned>(V);
             if (val4[i] && !inr) atomicOr(&S.status, LANTERN_ST_BAD_TABLE);   // carries no mass
-            const float f = __shfl_sync(kFull, fq_l, inr ? owner_unit<LOG_CP>(n) : 0);
-            run += inr ? static_cast<double>(E[EI(n)] * f) : 0.0;
+            run += inr ? static_cast<double>(E[EI(n)] * S.fqt[owner_slice<LOG_CP>(n)]) : 0.0;
             pre4[i] = run;
           }
           const double incl = warp_incl_scan(run, lane);
           if (lane == 31) S.wt[gw] = incl;
           gbar(grp);   // [scan 1]
-          double pre, tot;
-          {
-            const double t = lane < GW ? S.wt[lane] : 0.0;
-            const double in = warp_incl_scan(t, lane);
-            pre = __shfl_sync(kFull, in - t, gw);
-            tot = __shfl_sync(kFull, in, GW - 1);
+          double pre = 0.0, tot = 0.0;
+#pragma unroll
+          for (int w = 0; w < GW; ++w) {
+            const double t = S.wt[w];
+            if (w < gw) pre += t;
+            tot += t;
           }
           const double before = carry + pre + (incl - run);   // prefix before this thread's first slot
           int my_first = kNone;
@@ -522,10 +545,16 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
             S.first[gw] = kNone;
           }
           gbar(grp);   // [scan 2]
-          const int f_l = lane < GW ? S.first[lane] : kNone;
-          const int gfirst = __reduce_min_sync(kFull, f_l);
+          int gfirst = kNone, src = 0;
+#pragma unroll
+          for (int w = GW - 1; w >= 0; --w) {
+            const int f = S.first[w];
+            if (f != kNone && f <= gfirst) {
+              gfirst = f;
+              src = w;
+            }
+          }
           if (gfirst != kNone) {
-            const int src = __ffs(__ballot_sync(kFull, f_l == gfirst)) - 1;
             m = gfirst - 1;
             sm = S.sbefore[src];
             cut = true;
@@ -636,8 +665,13 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
             S.wt[GW + gw] = wp;
           }
           gbar(grp);   // [totals] also publishes the written-back residual
-          W = warp_sum(lane < GW ? S.wt[lane] : 0.0);
-          Sp = warp_sum(lane < GW ? S.wt[GW + lane] : 0.0);
+          W = 0.0;
+          Sp = 0.0;
+#pragma unroll
+          for (int w = 0; w < GW; ++w) {
+            W += S.wt[w];
+            Sp += S.wt[GW + w];
+          }
           if (!(W > 0.0)) {
             status |= LANTERN_ST_DEGENERATE;
             break;

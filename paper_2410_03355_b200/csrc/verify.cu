@@ -484,11 +484,11 @@ static WsLayout ws_layout(int B, int N) {
 
 static thread_local cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
 
-template <int CHC, bool BF16, bool UNC>
+template <int CHC, bool BF16, bool UNC, bool TONE>
 static cudaError_t launch_verify(const VerifyParams& P, int grid_ctx, int grid_bonus, size_t smem_bytes,
                                  cudaStream_t st) {
   constexpr int CHB = CHC == 8 ? 2 : 1;   // the bonus kernel runs 1024 threads per row
-  auto kc = lantern_context_kernel<CHC, BF16, UNC>;
+  auto kc = lantern_context_kernel<CHC, BF16, UNC, TONE>;
   cudaError_t e = cudaFuncSetAttribute(kc, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
   if (e != cudaSuccess) return e;
   if (g_ev_before && g_ev_after) cudaEventRecord(g_ev_before, st);
@@ -601,12 +601,14 @@ extern "C" lantern_status lantern_verify(const void* target_logits, const void* 
   const int grid_bonus = B < sms ? B : sms;
   cudaError_t e;
   const bool bf = dtype == LANTERN_BF16, un = has_uncond != 0;
-#define LANTERN_DISPATCH(CHV)                                                                        \
-  (bf ? (un ? launch_verify<CHV, true, true>(P, grid_ctx, grid_bonus, smem_bytes, st)                \
-            : launch_verify<CHV, true, false>(P, grid_ctx, grid_bonus, smem_bytes, st))              \
-      : (un ? launch_verify<CHV, false, true>(P, grid_ctx, grid_bonus, smem_bytes, st)               \
-            : launch_verify<CHV, false, false>(P, grid_ctx, grid_bonus, smem_bytes, st)))
+#define LANTERN_DISPATCH2(CHV, TV)                                                                   \
+  (bf ? (un ? launch_verify<CHV, true, true, TV>(P, grid_ctx, grid_bonus, smem_bytes, st)            \
+            : launch_verify<CHV, true, false, TV>(P, grid_ctx, grid_bonus, smem_bytes, st))          \
+      : (un ? launch_verify<CHV, false, true, TV>(P, grid_ctx, grid_bonus, smem_bytes, st)           \
+            : launch_verify<CHV, false, false, TV>(P, grid_ctx, grid_bonus, smem_bytes, st)))
+#define LANTERN_DISPATCH(CHV) (T == 1.0f ? LANTERN_DISPATCH2(CHV, true) : LANTERN_DISPATCH2(CHV, false))
   e = CH == 8 ? LANTERN_DISPATCH(8) : (CH == 4 ? LANTERN_DISPATCH(4) : (CH == 2 ? LANTERN_DISPATCH(2) : LANTERN_DISPATCH(1)));
+#undef LANTERN_DISPATCH2
 #undef LANTERN_DISPATCH
   return e == cudaSuccess ? LANTERN_OK : LANTERN_E_CUDA;
 }

@@ -25,7 +25,7 @@
 // inverse-CDF draw or the write-back for the next sibling.
 #pragma once
 
-#define LANTERN_CONTEXT_KERNEL_REVISION 7   // bump on every change to this file
+#define LANTERN_CONTEXT_KERNEL_REVISION 8   // bump on every change to this file
 
 namespace lantern {
 
@@ -139,8 +139,9 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
 }
 
-// CH = 8-token chunks per thread (1, 2, 4 or 8); a thread streams them in NP passes of CP chunks
-template <int CH, bool BF16, bool UNC>
+// CH = 8-token chunks per thread (1, 2, 4 or 8); a thread streams them in NP passes of CP chunks.
+// TONE = the temperature is exactly 1 (the paper's sampling setting): no division is compiled in.
+template <int CH, bool BF16, bool UNC, bool TONE>
 __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyParams P) {
   constexpr int NP = CH > 4 ? 2 : 1;          // passes
   constexpr int CP = CH / NP;                 // chunks per pass
@@ -233,7 +234,7 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
   const unsigned char* rc = stage;
   const unsigned char* ru = stage + rowbytes;
   unsigned char* rd = stage + 2 * rowbytes;
-  const bool T_is_one = P.T == 1.0f;
+  constexpr bool T_is_one = TONE;
   // eight processed drafter logits of 16-byte group g (z_p = l_d / T)
   auto draft_chunk = [&](int g, float (&out)[8]) {
     if (BF16) {

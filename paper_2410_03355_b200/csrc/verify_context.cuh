@@ -25,7 +25,7 @@
 // inverse-CDF draw or the write-back for the next sibling.
 #pragma once
 
-#define LANTERN_CONTEXT_KERNEL_REVISION 8   // bump on every change to this file
+#define LANTERN_CONTEXT_KERNEL_REVISION 10   // bump on every change to this file
 
 namespace lantern {
 
@@ -112,6 +112,37 @@ template <bool BF16>
 __device__ __forceinline__ float ctx_raw_logit(const void* base, size_t elem) {
   if (BF16) return __uint_as_float(static_cast<uint32_t>(__ldg(static_cast<const unsigned short*>(base) + elem)) << 16);
   return __ldg(static_cast<const float*>(base) + elem);
+}
+
+// Packed pairs of fp32 values (Blackwell's two-wide fp32 instructions): each lane is rounded exactly
+// like the scalar instruction, so results do not depend on the packing.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
 }
 
 // barrier among the 256 threads of consumer group `grp` (hardware barrier 1 + grp)
@@ -257,46 +288,6 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       for (int e = 0; e < 8; ++e) out[e] = __fdiv_rn(out[e], P.T);
     }
   };
-  // eight processed target logits of 16-byte group g (guidance combine, temperature)
-  auto target_chunk = [&](int g, float (&out)[8]) {
-    float lc[8], lu[8];
-    if (BF16) {
-      const uint4 x = *reinterpret_cast<const uint4*>(rc + g * 16);
-      const uint32_t xw[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        lc[2 * i] = __uint_as_float(xw[i] << 16);
-        lc[2 * i + 1] = __uint_as_float(xw[i] & 0xffff0000u);
-      }
-      if (UNC) {
-        const uint4 y = *reinterpret_cast<const uint4*>(ru + g * 16);
-        const uint32_t yw[4] = {y.x, y.y, y.z, y.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          lu[2 * i] = __uint_as_float(yw[i] << 16);
-          lu[2 * i + 1] = __uint_as_float(yw[i] & 0xffff0000u);
-        }
-      }
-    } else {
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const float4 x = *reinterpret_cast<const float4*>(rc + g * 32 + h * 16);
-        lc[4 * h] = x.x, lc[4 * h + 1] = x.y, lc[4 * h + 2] = x.z, lc[4 * h + 3] = x.w;
-        if (UNC) {
-          const float4 y = *reinterpret_cast<const float4*>(ru + g * 32 + h * 16);
-          lu[4 * h] = y.x, lu[4 * h + 1] = y.y, lu[4 * h + 2] = y.z, lu[4 * h + 3] = y.w;
-        }
-      }
-    }
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      float l = lc[e];
-      if (UNC) l = __fmaf_rn(P.cfg_scale, __fsub_rn(lc[e], lu[e]), lu[e]);   // l_u + s (l_c - l_u)
-      if (!T_is_one) l = __fdiv_rn(l, P.T);
-      out[e] = l;
-    }
-  };
-
   for (int iter = 0;; ++iter) {
     // One warp watches the copy's mbarrier (bounded wait); the group barrier then releases everybody
     // at once and tells every thread alike whether the rows have landed.
@@ -333,78 +324,130 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       raw_d = ctx_raw_logit<BF16>(P.draft, e);
     }
 
-    // ---------------- streaming part, warp-local, NP passes of CP chunks ----------------
-    float a[CP * 8];
+    // ---------------- streaming part, thread-local, NP passes of CP chunks ----------------
+    // values travel as packed pairs (tokens 2i, 2i+1 of a chunk)
+    uint64_t a2[CP * 4];
     float mlq_mine[NP], mlp_mine[NP];   // this thread's shift constants fl(max * log2 e), per pass
     float tq_mine[NP], tp_mine[NP];     // and its sums of numerators, in its own units
+    const uint64_t L2 = pack2(L_hi, L_hi);
+    // four packed pairs of processed logits of 16-byte group g of a row
+    auto pairs_of = [&](const unsigned char* row, int g, uint64_t (&o)[4]) {
+      if (BF16) {
+        const uint4 x = *reinterpret_cast<const uint4*>(row + g * 16);
+        const uint32_t xw[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) o[i] = pack2(__uint_as_float(xw[i] << 16), __uint_as_float(xw[i] & 0xffff0000u));
+      } else {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const float4 x = *reinterpret_cast<const float4*>(row + g * 32 + h * 16);
+          o[2 * h] = pack2(x.x, x.y);
+          o[2 * h + 1] = pack2(x.z, x.w);
+        }
+      }
+    };
+    auto divide_T = [&](uint64_t v) {
+      float lo, hi;
+      unpack2(v, lo, hi);
+      return pack2(__fdiv_rn(lo, P.T), __fdiv_rn(hi, P.T));
+    };
     // --- target: guidance combine, slice maximum, numerators, partial sum; E replaces the raw rows ---
 #pragma unroll
     for (int p = 0; p < NP; ++p) {
+      const uint64_t s2 = pack2(P.cfg_scale, P.cfg_scale);
+      float mq = ninf;
 #pragma unroll
       for (int c = 0; c < CP; ++c) {
         const int g = (p * CP + c) * GT + gt;
-        float v8[8];
         if (g * 8 < V) {
-          target_chunk(g, v8);
+          uint64_t c2[4], u2[4];
+          pairs_of(rc, g, c2);
+          if (UNC) pairs_of(ru, g, u2);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            uint64_t l2 = c2[i];
+            if (UNC) l2 = fma2(s2, sub2(c2[i], u2[i]), u2[i]);   // l_u + s (l_c - l_u)
+            if (!T_is_one) l2 = divide_T(l2);
+            a2[c * 4 + i] = l2;
+            float lo, hi;
+            unpack2(l2, lo, hi);
+            mq = max3(mq, lo, hi);
+          }
         } else {
 #pragma unroll
-          for (int e = 0; e < 8; ++e) v8[e] = ninf;
+          for (int i = 0; i < 4; ++i) a2[c * 4 + i] = pack2(ninf, ninf);
         }
-#pragma unroll
-        for (int e = 0; e < 8; ++e) a[c * 8 + e] = v8[e];
       }
-      float mq = a[0];
-#pragma unroll
-      for (int i = 1; i < CP * 8; ++i) mq = fmaxf(mq, a[i]);
       // a slice without any finite logit (padding, masked tokens) still needs a finite shift
       mq = fmaxf(mq, -1.0e37f);
       const float mlq_w = mq * L_hi;
       mlq_mine[p] = mlq_w;
-      float tq = 0.0f;
+      const uint64_t nml2 = pack2(-mlq_w, -mlq_w);
+      uint64_t t2 = pack2(0.0f, 0.0f);
 #pragma unroll
       for (int c = 0; c < CP; ++c) {
+        float e[8];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) a[c * 8 + e] = ex2_approx(__fmaf_rn(a[c * 8 + e], L_hi, -mlq_w));
-        tq += sum8(&a[c * 8]);
+        for (int i = 0; i < 4; ++i) {
+          float lo, hi;
+          unpack2(fma2(a2[c * 4 + i], L2, nml2), lo, hi);
+          e[2 * i] = ex2_approx(lo);
+          e[2 * i + 1] = ex2_approx(hi);
+        }
+        t2 = add2(t2, add2(add2(pack2(e[0], e[1]), pack2(e[2], e[3])), add2(pack2(e[4], e[5]), pack2(e[6], e[7]))));
         const int g = (p * CP + c) * GT + gt;
         if (g * 8 < V) {
-          *reinterpret_cast<float4*>(E + EI(g * 8)) = make_float4(a[c * 8], a[c * 8 + 1], a[c * 8 + 2], a[c * 8 + 3]);
-          *reinterpret_cast<float4*>(E + EI(g * 8 + 4)) =
-              make_float4(a[c * 8 + 4], a[c * 8 + 5], a[c * 8 + 6], a[c * 8 + 7]);
+          *reinterpret_cast<float4*>(E + EI(g * 8)) = make_float4(e[0], e[1], e[2], e[3]);
+          *reinterpret_cast<float4*>(E + EI(g * 8 + 4)) = make_float4(e[4], e[5], e[6], e[7]);
         }
       }
-      tq_mine[p] = tq;
+      float tlo, thi;
+      unpack2(t2, tlo, thi);
+      tq_mine[p] = tlo + thi;
     }
     // --- drafter: slice maximum and partial sum of numerators; the raw row stays in shared memory ---
 #pragma unroll
     for (int p = 0; p < NP; ++p) {
+      float mp = ninf;
 #pragma unroll
       for (int c = 0; c < CP; ++c) {
         const int g = (p * CP + c) * GT + gt;
-        float v8[8];
         if (g * 8 < V) {
-          draft_chunk(g, v8);
+          uint64_t d2[4];
+          pairs_of(rd, g, d2);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            uint64_t l2 = d2[i];
+            if (!T_is_one) l2 = divide_T(l2);
+            a2[c * 4 + i] = l2;
+            float lo, hi;
+            unpack2(l2, lo, hi);
+            mp = max3(mp, lo, hi);
+          }
         } else {
 #pragma unroll
-          for (int e = 0; e < 8; ++e) v8[e] = ninf;
+          for (int i = 0; i < 4; ++i) a2[c * 4 + i] = pack2(ninf, ninf);
         }
-#pragma unroll
-        for (int e = 0; e < 8; ++e) a[c * 8 + e] = v8[e];
       }
-      float mp = a[0];
-#pragma unroll
-      for (int i = 1; i < CP * 8; ++i) mp = fmaxf(mp, a[i]);
       mp = fmaxf(mp, -1.0e37f);
       const float mlp_w = mp * L_hi;
       mlp_mine[p] = mlp_w;
-      float tp = 0.0f;
+      const uint64_t nml2 = pack2(-mlp_w, -mlp_w);
+      uint64_t t2 = pack2(0.0f, 0.0f);
 #pragma unroll
       for (int c = 0; c < CP; ++c) {
+        uint64_t e2[4];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) a[c * 8 + e] = ex2_approx(__fmaf_rn(a[c * 8 + e], L_hi, -mlp_w));
-        tp += sum8(&a[c * 8]);
+        for (int i = 0; i < 4; ++i) {
+          float lo, hi;
+          unpack2(fma2(a2[c * 4 + i], L2, nml2), lo, hi);
+          e2[i] = pack2(ex2_approx(lo), ex2_approx(hi));
+        }
+        t2 = add2(t2, add2(add2(e2[0], e2[1]), add2(e2[2], e2[3])));
       }
-      tp_mine[p] = tp;
+      float tlo, thi;
+      unpack2(t2, tlo, thi);
+      tp_mine[p] = tlo + thi;
     }
 
     // ---------------- group statistics ----------------

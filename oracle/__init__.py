@@ -145,3 +145,41 @@ def verify_inputs(inp, neighbor_idx: np.ndarray, delta: float) -> VerifyResult:
     """Convenience: run `verify` on a lantern_inputs.VerifyInputs bundle."""
     return verify(inp.target_logits, inp.draft_logits, inp.dtype, inp.cfg_scale, inp.has_uncond, inp.T,
                   inp.draft_tokens, inp.tree_parents, neighbor_idx, delta, inp.uniforms)
+
+
+@dataclasses.dataclass
+class GreedyResult:
+    accept_len: np.ndarray      # [B] int32
+    next_token: np.ndarray      # [B] int32
+    accept_path: np.ndarray     # [B, N] int32, -1 padded
+    status: np.ndarray          # [B] int32 bit flags
+    tested: np.ndarray          # [B, N] uint8
+    qa: np.ndarray              # [B, N] float64: sum of the target over A_{k,delta}(x~)
+    m: np.ndarray               # [B, N] int32
+    margin: np.ndarray          # [B, N] float64: distance of the node's decisions to flipping
+
+
+def verify_greedy(target_logits: np.ndarray, dtype: int, cfg_scale: float, has_uncond: int,
+                  draft_tokens: np.ndarray, tree_parents: Optional[np.ndarray], neighbor_idx: np.ndarray,
+                  delta: float) -> GreedyResult:
+    """Greedy-decoding verification (Section 4.3, last sentence) on host arrays."""
+    tl = np.ascontiguousarray(target_logits)
+    C, B, R, V = tl.shape
+    N = R - 1
+    assert C == (2 if has_uncond else 1)
+    assert tl.dtype == (np.float32 if dtype == 0 else np.uint16)
+    tok = np.ascontiguousarray(draft_tokens, dtype=np.int32).reshape(B, N)
+    par = None if tree_parents is None else np.ascontiguousarray(tree_parents, dtype=np.int32).reshape(B, N)
+    nb = np.ascontiguousarray(neighbor_idx, dtype=np.int32)
+    assert nb.shape[0] == V
+    res = GreedyResult(accept_len=np.zeros(B, np.int32), next_token=np.zeros(B, np.int32),
+                       accept_path=np.full((B, N), -1, np.int32), status=np.zeros(B, np.int32),
+                       tested=np.zeros((B, N), np.uint8), qa=np.zeros((B, N)), m=np.full((B, N), -1, np.int32),
+                       margin=np.full((B, N), np.inf))
+    rc = _load().oracle_verify_greedy(_p(tl), int(dtype), ctypes.c_float(cfg_scale), int(has_uncond), _p(tok), _p(par),
+                                      _p(nb), int(nb.shape[1]), ctypes.c_float(delta), B, N, V, _p(res.accept_len),
+                                      _p(res.next_token), _p(res.accept_path), _p(res.status), _p(res.tested),
+                                      _p(res.qa), _p(res.m), _p(res.margin))
+    if rc != 0:
+        raise ValueError(f"oracle_verify_greedy: bad arguments ({rc})")
+    return res

@@ -458,4 +458,120 @@ int oracle_verify(const void* target_logits, const void* draft_logits, int dtype
   return 0;
 }
 
+// ---------------------------------------------------------------------------------------
+// Greedy decoding (Section 4.3, last sentence: accept x~ iff x~ = argmax_x q_{k,delta}(x|D = x~)).
+//
+// Reading taken (the paper gives no more than that sentence): q is the softmax of the guided
+// target logits at temperature 1; A_{k,delta}(x~) is built on it as for sampling; since
+// q_{k,delta} puts sum_A q on x~, zero on the rest of A and q elsewhere, x~ is an arg max iff
+// sum_A q >= q(x) for every x outside A (ties accept).  Children of a context are tried in node
+// order against the same q (there is no residual in greedy decoding); where every child is
+// rejected, and where the walk reaches a context without children, the next token is
+// argmax_x q(x), smallest index on ties -- after a rejection that is also argmax of
+// q_{k,delta}(.|D = x~), because the arg max of q cannot lie inside a rejected A.
+// No drafter distribution and no random numbers are involved.
+//
+// Layouts as in oracle_verify.  Trace outputs per node [B, N] (each may be null): tr_tested,
+// tr_qa (sum_A q), tr_m (|A| - 1), tr_margin (min of the cut margin and |sum_A q - max_{x not in A} q|).
+// ---------------------------------------------------------------------------------------
+int oracle_verify_greedy(const void* target_logits, int dtype, float cfg_scale, int has_uncond,
+                         const int32_t* draft_tokens, const int32_t* tree_parents, const int32_t* neighbor_idx,
+                         int k, float delta_f, int B, int N, int V, int32_t* out_accept_len,
+                         int32_t* out_next_token, int32_t* out_accept_path, int32_t* out_status,
+                         uint8_t* tr_tested, double* tr_qa, int32_t* tr_m, double* tr_margin) {
+  if (B < 0 || N < 0 || V < 1 || k < 1 || k > V) return -2;
+  if (!(delta_f >= 0.0f)) return -3;
+  if (B == 0) return 0;
+  if (!target_logits || !neighbor_idx || !out_accept_len || !out_next_token) return -1;
+  if (N > 0 && !draft_tokens) return -1;
+  if (dtype != DT_F32 && dtype != DT_BF16) return -3;
+  const double delta = static_cast<double>(delta_f);
+  const int R = N + 1;
+  const size_t branch = static_cast<size_t>(B) * R * V;
+  std::vector<float> z(V);
+  std::vector<double> q;
+  std::vector<char> inA(V);
+  std::vector<std::vector<int>> kids(R);
+  for (int b = 0; b < B; ++b) {
+    int status = 0;
+    int32_t* path = out_accept_path ? out_accept_path + static_cast<size_t>(b) * N : nullptr;
+    if (path) std::fill(path, path + N, -1);
+    for (int i = 0; i < N; ++i) {
+      const size_t o = static_cast<size_t>(b) * N + i;
+      if (tr_tested) tr_tested[o] = 0;
+      if (tr_qa) tr_qa[o] = 0.0;
+      if (tr_m) tr_m[o] = -1;
+      if (tr_margin) tr_margin[o] = std::numeric_limits<double>::infinity();
+    }
+    for (auto& v : kids) v.clear();
+    for (int i = 0; i < N; ++i) {
+      const int32_t tok = draft_tokens[static_cast<size_t>(b) * N + i];
+      if (tok < 0 || tok >= V) status |= ST_BAD_TOKEN;
+      const int32_t par = tree_parents ? tree_parents[static_cast<size_t>(b) * N + i] : i - 1;
+      if (par < -1 || par >= i) status |= ST_BAD_PARENT;
+      else kids[par + 1].push_back(i);
+    }
+    if (status) {
+      out_accept_len[b] = 0;
+      out_next_token[b] = -1;
+      if (out_status) out_status[b] = status;
+      continue;
+    }
+    int cur = 0, accept_len = 0, next_token = -1;
+    for (;;) {
+      const size_t row = (static_cast<size_t>(b) * R + cur) * V;
+      for (int x = 0; x < V; ++x) {
+        float lc = load_logit(target_logits, dtype, row + x);
+        float lu = has_uncond ? load_logit(target_logits, dtype, branch + row + x) : 0.0f;
+        z[x] = target_z(lc, lu, has_uncond, cfg_scale, 1.0f);
+      }
+      if (!softmax(z, q, nullptr)) {
+        status |= ST_NONFINITE;
+        break;
+      }
+      int best = 0;
+      for (int x = 1; x < V; ++x)
+        if (q[x] > q[best]) best = x;   // smallest index on ties
+      int accepted = -1;
+      for (int c : kids[cur]) {
+        const int32_t xt = draft_tokens[static_cast<size_t>(b) * N + c];
+        const int32_t* nrow = neighbor_idx + static_cast<size_t>(xt) * k;
+        double moved = 0.0, cut_margin = 0.0;
+        int bad = 0;
+        const int m = oracle_a_set(q.data(), V, nrow, k, delta, &moved, &cut_margin, &bad);
+        if (bad) status |= ST_BAD_TABLE;
+        const double qa = q[xt] + moved;
+        std::fill(inA.begin(), inA.end(), 0);
+        inA[xt] = 1;
+        for (int j = 1; j <= m; ++j)
+          if (nrow[j] >= 0 && nrow[j] < V) inA[nrow[j]] = 1;
+        double outside = -1.0;   // max of q outside A (none: -1, so that x~ is accepted)
+        for (int x = 0; x < V; ++x)
+          if (!inA[x] && q[x] > outside) outside = q[x];
+        const size_t o = static_cast<size_t>(b) * N + c;
+        if (tr_tested) tr_tested[o] = 1;
+        if (tr_qa) tr_qa[o] = qa;
+        if (tr_m) tr_m[o] = m;
+        if (tr_margin) tr_margin[o] = std::min(std::fabs(qa - outside), k > 1 ? cut_margin : std::numeric_limits<double>::infinity());
+        if (qa >= outside) {   // x~ is an arg max of q_{k,delta}(.|D = x~)
+          accepted = c;
+          break;
+        }
+      }
+      if (accepted >= 0) {
+        if (path) path[accept_len] = accepted;
+        ++accept_len;
+        cur = accepted + 1;
+        continue;
+      }
+      next_token = best;   // every child rejected, or no child: arg max of the target
+      break;
+    }
+    out_accept_len[b] = accept_len;
+    out_next_token[b] = next_token;
+    if (out_status) out_status[b] = status;
+  }
+  return 0;
+}
+
 }  // extern "C"

@@ -43,7 +43,7 @@ enum {
   LANTERN_E_WORKSPACE = -4,     /* workspace missing, too small or misaligned */
   LANTERN_E_CUDA = -5,          /* a CUDA runtime call failed (no device, launch error) */
   LANTERN_E_ALIGN = -6,         /* a pointer is not 16-byte aligned */
-  LANTERN_E_UNIMPLEMENTED = -7  /* valid request this build does not cover (T == 0) */
+  LANTERN_E_UNIMPLEMENTED = -7  /* valid request this build does not cover (none at present) */
 };
 
 /* storage type of logits */
@@ -105,7 +105,13 @@ lantern_status lantern_build_neighbors(const float* codebook, int V, int D, int 
  *                  may be NULL when N == 0
  *   dtype          LANTERN_F32 or LANTERN_BF16, for both logit tensors; bases 16-byte aligned
  *   cfg_scale      s, read only if has_uncond
- *   T              temperature > 0
+ *   T              temperature > 0, or exactly 0 for greedy decoding (Section 4.3, last sentence):
+ *                  q is then the softmax at temperature 1, node i is accepted iff
+ *                  sum_{A_{k,delta}(x~)} q >= max_x q(x) (x~ is an arg max of q_{k,delta}(.|D = x~),
+ *                  ties accept), children are tried in node order against the same q, and the
+ *                  next token is arg max q of the context where the walk stops (smallest index
+ *                  on ties).  draft_logits and uniforms are not read and may be NULL;
+ *                  out_node_px is written as 0; V <= 16384 for both logit types
  *   draft_tokens   [B, N] int32 in [0, V)
  *   tree_parents   [B, N] int32, -1 = child of the root, else an index < own index; NULL = chain
  *   neighbor_idx   [V, k] int32 as written by lantern_build_neighbors (slot 0 = the token itself)

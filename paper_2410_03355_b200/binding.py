@@ -128,15 +128,18 @@ class VerifyOutputs:
 
 def verify(target_logits: torch.Tensor, draft_logits: Optional[torch.Tensor], cfg_scale: float, T: float,
            draft_tokens: Optional[torch.Tensor], tree_parents: Optional[torch.Tensor], neighbor_idx: torch.Tensor,
-           delta: float, uniforms: torch.Tensor, *, out: Optional[VerifyOutputs] = None, trace: bool = False,
+           delta: float, uniforms: Optional[torch.Tensor], *, out: Optional[VerifyOutputs] = None, trace: bool = False,
            workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None) -> VerifyOutputs:
     """lantern_verify on torch tensors.
 
     target_logits [C, B, N+1, V] (C = 2: conditional, unconditional; C = 1: no guidance), fp32 or bf16;
     draft_logits [B, N+1, V]; draft_tokens / tree_parents [B, N] int32 (tree_parents None = chain);
     neighbor_idx [V, k] int32; uniforms [B, N+1] fp32.  Outputs are allocated unless `out` is given.
+    T == 0 selects greedy decoding: draft_logits and uniforms are not read and may be None.
     """
     lib = load_library()
+    if T != 0 and (uniforms is None or (draft_logits is None and target_logits.shape[2] > 1)):
+        raise ValueError("sampling (T > 0) needs draft_logits and uniforms")
     C, B, R, V = target_logits.shape
     N = R - 1
     if C not in (1, 2):

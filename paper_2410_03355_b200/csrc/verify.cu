@@ -269,9 +269,11 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
     if (P.out_px) P.out_px[o] = qnan;
     if (P.out_m) P.out_m[o] = -1;
   }
-  for (int i = lane; i <= N; i += 32) {
-    const float r = P.uniforms[static_cast<size_t>(b) * R + i];
-    if (!(r >= 0.0f && r < 1.0f)) status |= LANTERN_ST_BAD_UNIFORM;
+  if (P.uniforms) {   // greedy decoding draws nothing and passes no uniforms
+    for (int i = lane; i <= N; i += 32) {
+      const float r = P.uniforms[static_cast<size_t>(b) * R + i];
+      if (!(r >= 0.0f && r < 1.0f)) status |= LANTERN_ST_BAD_UNIFORM;
+    }
   }
   status = __reduce_or_sync(kFull, status);
   __syncwarp();
@@ -288,12 +290,12 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
     for (int i = 0; i < N; ++i) {
       const size_t o = static_cast<size_t>(b) * N + i;
       const int par = P.parents ? P.parents[o] : i - 1;
-      ChildInfo ci = {i, P.tokens[o], P.uniforms[static_cast<size_t>(b) * R + i], 0};
+      ChildInfo ci = {i, P.tokens[o], P.uniforms ? P.uniforms[static_cast<size_t>(b) * R + i] : 0.0f, 0};
       kids[cur[par + 1]++] = ci;
     }
   }
   __syncwarp();         // lane 0's writes to cur[] and kids[] are visible to the warp
-  const float u_final = P.uniforms[static_cast<size_t>(b) * R + N];
+  const float u_final = P.uniforms ? P.uniforms[static_cast<size_t>(b) * R + N] : 0.0f;
   const int cap = P.B * N;
   for (int base = 0; base < R; base += 32) {
     const int c = base + lane;
@@ -327,6 +329,8 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
 
 // kernel 2: the fused context pass
 #include "verify_context.cuh"
+// greedy decoding (temperature 0)
+#include "verify_greedy.cuh"
 
 namespace lantern {
 
@@ -503,6 +507,22 @@ static cudaError_t launch_verify(const VerifyParams& P, int grid_ctx, int grid_b
   return cudaGetLastError();
 }
 
+template <bool BF16, bool UNC>
+static cudaError_t launch_greedy(const VerifyParams& P, int grid_ctx, int grid_bonus, cudaStream_t st) {
+  auto kc = lantern_greedy_context_kernel<BF16, UNC>;
+  const size_t smem = static_cast<size_t>(P.V) * sizeof(float);
+  cudaError_t e = cudaFuncSetAttribute(kc, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
+  kc<<<grid_ctx, GRT, smem, st>>>(P);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  lantern_walk_kernel<<<(P.B + 127) / 128, 128, 0, st>>>(P);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  lantern_greedy_bonus_kernel<BF16, UNC><<<grid_bonus, GRT, 0, st>>>(P);
+  return cudaGetLastError();
+}
+
 }  // namespace lantern
 
 using namespace lantern;
@@ -536,17 +556,18 @@ extern "C" lantern_status lantern_verify(const void* target_logits, const void* 
   if (static_cast<long long>(B) * (N + 1) >= (1ll << 31)) return LANTERN_E_SHAPE;
   if (!(T >= 0.0f) || !(delta >= 0.0f) || !isfinite(T) || !isfinite(delta)) return LANTERN_E_PARAM;
   if (has_uncond && !isfinite(cfg_scale)) return LANTERN_E_PARAM;
-  if (T == 0.0f) return LANTERN_E_UNIMPLEMENTED;   // greedy decoding is not part of this build
+  const bool greedy = T == 0.0f;   // Section 4.3, last sentence: no drafter distribution, no random numbers
   const int esize = dtype == LANTERN_BF16 ? 2 : 4;
   const int nrows = has_uncond ? 3 : 2;
   const int CH = V > 4 * GT * 8 ? 8 : (V > 2 * GT * 8 ? 4 : (V > GT * 8 ? 2 : 1));   // 8-token chunks per thread
   // one staging area of three row slots per consumer group; the numerators are kept over the rows they came from
   const size_t smem_bytes = NGRP * ((static_cast<size_t>(3) * V * esize + 127) & ~static_cast<size_t>(127));
   (void)nrows;
-  if (smem_bytes > 220 * 1024 || (dtype == LANTERN_F32 && V > 8192)) return LANTERN_E_SHAPE;
+  if (!greedy && (smem_bytes > 220 * 1024 || (dtype == LANTERN_F32 && V > 8192))) return LANTERN_E_SHAPE;
   if (B == 0) return LANTERN_OK;
-  if (!target_logits || !neighbor_idx || !uniforms || !out_accept_len || !out_next_token) return LANTERN_E_NULL;
-  if (N > 0 && (!draft_logits || !draft_tokens)) return LANTERN_E_NULL;
+  if (!target_logits || !neighbor_idx || !out_accept_len || !out_next_token) return LANTERN_E_NULL;
+  if (!greedy && !uniforms) return LANTERN_E_NULL;
+  if (N > 0 && (!draft_tokens || (!greedy && !draft_logits))) return LANTERN_E_NULL;
   if ((reinterpret_cast<uintptr_t>(target_logits) & 15) || (reinterpret_cast<uintptr_t>(draft_logits) & 15))
     return LANTERN_E_ALIGN;
   const WsLayout L = ws_layout(B, N);
@@ -561,7 +582,7 @@ extern "C" lantern_status lantern_verify(const void* target_logits, const void* 
   P.tokens = draft_tokens;
   P.parents = tree_parents;
   P.nbr = neighbor_idx;
-  P.uniforms = uniforms;
+  P.uniforms = greedy ? nullptr : uniforms;
   P.out_len = out_accept_len;
   P.out_tok = out_next_token;
   P.out_path = out_accept_path;
@@ -601,6 +622,12 @@ extern "C" lantern_status lantern_verify(const void* target_logits, const void* 
   const int grid_bonus = B < sms ? B : sms;
   cudaError_t e;
   const bool bf = dtype == LANTERN_BF16, un = has_uncond != 0;
+  if (greedy) {
+    const int grid_g = static_cast<int>(items < 8ll * sms ? items : 8ll * sms);
+    e = bf ? (un ? launch_greedy<true, true>(P, grid_g, grid_bonus, st) : launch_greedy<true, false>(P, grid_g, grid_bonus, st))
+           : (un ? launch_greedy<false, true>(P, grid_g, grid_bonus, st) : launch_greedy<false, false>(P, grid_g, grid_bonus, st));
+    return e == cudaSuccess ? LANTERN_OK : LANTERN_E_CUDA;
+  }
 #define LANTERN_DISPATCH2(CHV, TV)                                                                   \
   (bf ? (un ? launch_verify<CHV, true, true, TV>(P, grid_ctx, grid_bonus, smem_bytes, st)            \
             : launch_verify<CHV, true, false, TV>(P, grid_ctx, grid_bonus, smem_bytes, st))          \

@@ -200,8 +200,12 @@ def test_host_argument_errors():
         a.update(kw)
         return lt.verify(**a)
 
-    for kw, code in [(dict(T=0.0), -7), (dict(T=-1.0), -3), (dict(delta=-0.1), -3), (dict(delta=float("nan")), -3),
+    for kw, code in [(dict(T=-1.0), -3), (dict(uniforms=None, T=1.0), None), (dict(delta=-0.1), -3), (dict(delta=float("nan")), -3),
                      (dict(workspace=torch.empty(16, dtype=torch.uint8, device="cuda")), -4)]:
+        if code is None:                             # sampling without uniforms: refused by the binding
+            with pytest.raises(ValueError):
+                call(**kw)
+            continue
         with pytest.raises(lt.LanternError) as e:
             call(**kw)
         assert e.value.code == code, kw

@@ -57,13 +57,14 @@ def load_peaks():
     return 6650.0, "fallback"
 
 
-def algorithmic_bytes(cfg: dict, B: int, parents) -> int:
+def algorithmic_bytes(cfg: dict, B: int, parents, greedy: bool = False) -> int:
     """Bytes the method must move per call: for each context with at least one child, two target
-    rows and one drafter row (one target row without guidance), plus one neighbour row of 4k
-    bytes per drafted node.  Bonus rows, tokens, uniforms and outputs (< 0.1 %) are left out."""
+    rows and one drafter row (one target row without guidance; no drafter row in greedy
+    decoding), plus one neighbour row of 4k bytes per drafted node.  Bonus rows, tokens, uniforms
+    and outputs (< 0.1 %) are left out."""
     import lantern_inputs as li
     esize = 2 if cfg["dtype"] == li.BF16 else 4
-    rows = 3 if cfg["has_uncond"] else 2
+    rows = (2 if cfg["has_uncond"] else 1) + (0 if greedy else 1)
     N, V, k = cfg["N"], cfg["V"], cfg["k"]
     if parents is None:
         n_ctx = B * N
@@ -140,7 +141,7 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def oracle_sample_rate(host_inp, table_host, delta, budget_s=15.0):
+def oracle_sample_rate(host_inp, table_host, delta, budget_s=15.0, greedy=False):
     """Oracle throughput (drafted positions verified per second) on as many leading sequences of
     `host_inp` as fit in about `budget_s` seconds; returns (rate, n_sequences, seconds)."""
     import dataclasses
@@ -158,7 +159,11 @@ def oracle_sample_rate(host_inp, table_host, delta, budget_s=15.0):
             tree_parents=None if host_inp.tree_parents is None else np.ascontiguousarray(host_inp.tree_parents[sl]),
             uniforms=np.ascontiguousarray(host_inp.uniforms[sl]), B=n)
         t0 = time.perf_counter()
-        oracle.verify_inputs(part, table_host, delta)
+        if greedy:
+            oracle.verify_greedy(part.target_logits, part.dtype, part.cfg_scale, part.has_uncond, part.draft_tokens,
+                                 part.tree_parents, table_host, delta)
+        else:
+            oracle.verify_inputs(part, table_host, delta)
         t_used += time.perf_counter() - t0
         done += n
         pos += n * host_inp.N
@@ -219,7 +224,11 @@ def run_reference(args, rank, world):
         inp = li.config_verify_inputs(w["config"], step=step, B=nseq)
         tab = table_for(inp)
         t1 = time.perf_counter()
-        oracle.verify_inputs(inp, tab, cfg["delta"])
+        if args.greedy:
+            oracle.verify_greedy(inp.target_logits, inp.dtype, inp.cfg_scale, inp.has_uncond, inp.draft_tokens,
+                                 inp.tree_parents, tab, cfg["delta"])
+        else:
+            oracle.verify_inputs(inp, tab, cfg["delta"])
         dt = time.perf_counter() - t1
         if step >= args.warmup:
             steps_t.append(dt)
@@ -230,7 +239,7 @@ def run_reference(args, rank, world):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(steps_t),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": args.workload, "V": cfg["V"], "k": cfg["k"], "delta": cfg["delta"], "N": cfg["N"],
-                   "sequences_per_step": nseq},
+                   "T": 0.0 if args.greedy else cfg["T"], "sequences_per_step": nseq},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
                          "sample": f"{nseq} sequences x {cfg['N']} drafts per step of the {args.workload} workload "
                                    f"(bounded sample; neighbour rows built by the oracle outside the timed region)"},
@@ -252,6 +261,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--greedy", action="store_true",
+                    help="run the workload at T = 0 (greedy decoding: no drafter rows, no random numbers)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -299,7 +310,8 @@ def main():
     # ---- inputs resident in HBM ----
     d = lid.config_verify_inputs_device(w["config"], B=B, seed=rank_seed(li.BASE_SEED, rank), rho=args.rho)
     torch.cuda.synchronize()
-    alg_bytes = algorithmic_bytes(cfg, B, d["tree_parents"])
+    alg_bytes = algorithmic_bytes(cfg, B, d["tree_parents"], args.greedy)
+    T = 0.0 if args.greedy else d["T"]
     ws = torch.empty(lt.verify_workspace_bytes(B, N), dtype=torch.uint8, device="cuda")
     i32 = dict(dtype=torch.int32, device="cuda")
     out = lt.VerifyOutputs(accept_len=torch.empty(B, **i32), next_token=torch.empty(B, **i32),
@@ -308,8 +320,9 @@ def main():
     stream = torch.cuda.current_stream()
 
     def step():
-        lt.verify(d["target_logits"], d["draft_logits"], d["cfg_scale"], d["T"], d["draft_tokens"], d["tree_parents"],
-                  table, delta, d["uniforms"], out=out, workspace=ws, stream=stream)
+        lt.verify(d["target_logits"], None if args.greedy else d["draft_logits"], d["cfg_scale"], T, d["draft_tokens"],
+                  d["tree_parents"], table, delta, None if args.greedy else d["uniforms"], out=out, workspace=ws,
+                  stream=stream)
 
     for _ in range(args.warmup):
         step()
@@ -353,7 +366,9 @@ def main():
     e2e = None
     if not args.no_e2e:
         host = {}
-        for name in ("target_logits", "draft_logits", "draft_tokens", "tree_parents", "uniforms"):
+        names = ("target_logits", "draft_tokens", "tree_parents") if args.greedy else \
+                ("target_logits", "draft_logits", "draft_tokens", "tree_parents", "uniforms")
+        for name in names:
             t = d[name]
             host[name] = None if t is None else torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t)
         h_len = torch.empty(B, dtype=torch.int32, pin_memory=True)
@@ -390,7 +405,7 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         n_s = min(B, 8192 if cfg["N"] <= 8 else 256)
         host_inp = lid.to_host(d, rows=np.arange(n_s))
-        rate, n_done, secs = oracle_sample_rate(host_inp, table.cpu().numpy(), delta)
+        rate, n_done, secs = oracle_sample_rate(host_inp, table.cpu().numpy(), delta, greedy=args.greedy)
         cpu = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
                "sample": f"first {n_done} sequences ({n_done * N} drafted positions) of this call, {secs:.1f} s"}
 
@@ -402,15 +417,16 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": args.workload, "note": w["note"], "sequences_per_call": B, "drafts_per_sequence": N,
-                       "V": V, "k": k, "delta": delta, "cfg_scale": cfg["cfg_scale"], "T": cfg["T"],
+                       "V": V, "k": k, "delta": delta, "cfg_scale": cfg["cfg_scale"], "T": T,
                        "logits": "bf16" if cfg["dtype"] == li.BF16 else "f32", "rho": args.rho,
                        "l2_policy": "inputs larger than L2 (%.2f GB of logits per call)" %
-                                    ((d["target_logits"].numel() + d["draft_logits"].numel()) *
+                                    ((d["target_logits"].numel() + (0 if args.greedy else d["draft_logits"].numel())) *
                                      d["target_logits"].element_size() / 1e9),
                        "parallelism": "replicas" if world > 1 else "single"},
-            "roofline": {"bound": "hbm", "kernel": "lantern_context_kernel", "achieved": achieved, "peak": peak,
+            "roofline": {"bound": "hbm", "kernel": "lantern_greedy_context_kernel" if args.greedy else "lantern_context_kernel",
+                         "achieved": achieved, "peak": peak,
                          "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": ncu_traffic(args.workload, cfg, alg_bytes),
+                         "traffic": None if args.greedy else ncu_traffic(args.workload, cfg, alg_bytes),
                          "algorithmic_bytes_per_launch": int(alg_bytes), "kernel_ms": fused_ms},
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": 4 * args.steps, "clocks": clocks,
             "neighbor_build": {"ms": build_ms, "V": V, "D": cfg["D"], "k": k,

@@ -513,9 +513,11 @@ static cudaError_t launch_greedy(const VerifyParams& P, int grid_ctx, int grid_b
   const size_t smem = static_cast<size_t>(P.V) * sizeof(float);
   cudaError_t e = cudaFuncSetAttribute(kc, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return e;
+  if (g_ev_before && g_ev_after) cudaEventRecord(g_ev_before, st);
   kc<<<grid_ctx, GRT, smem, st>>>(P);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
+  if (g_ev_before && g_ev_after) cudaEventRecord(g_ev_after, st);
   lantern_walk_kernel<<<(P.B + 127) / 128, 128, 0, st>>>(P);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;

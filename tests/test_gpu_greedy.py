@@ -58,9 +58,12 @@ def replay(inp, table, delta, b, g_len, g_tok, g_path):
 
 
 def check(inp, host, dev, delta, **kw):
+    return check_outputs(inp, host, delta, run_gpu(inp, dev, delta, **kw))
+
+
+def check_outputs(inp, host, delta, gpu):
     ora = oracle.verify_greedy(inp.target_logits, inp.dtype, inp.cfg_scale, inp.has_uncond, inp.draft_tokens,
                                inp.tree_parents, host, delta)
-    gpu = run_gpu(inp, dev, delta, **kw)
     g_len, g_tok = gpu.accept_len.cpu().numpy(), gpu.next_token.cpu().numpy()
     g_path, g_st = gpu.accept_path.cpu().numpy(), gpu.status.cpu().numpy()
     assert np.array_equal(g_st, ora.status)
@@ -169,3 +172,27 @@ def test_bench_shape_sample():
     host = dev.cpu().numpy()
     inp = li.config_verify_inputs("batch_chain", step=0, B=48)
     check(inp, host, dev, c["delta"])
+
+
+@pytest.mark.parametrize("workload,sample", [("batch_chain", 96), ("stress", 64)])
+def test_bench_sized_call_against_sampled_oracle(workload, sample):
+    """The call `bench.py --greedy` times, checked on a seeded sample of its sequences."""
+    import bench
+    import lantern_inputs.device as lid
+    from test_gpu_fullsize import _properties, _table, _take
+    w = bench.WORKLOADS[workload]
+    cfg = li.CONFIGS[w["config"]]
+    B, N, V, delta = w["B"], cfg["N"], cfg["V"], cfg["delta"]
+    table = _table(w["config"])
+    d = lid.config_verify_inputs_device(w["config"], B=B, seed=bench.rank_seed(li.BASE_SEED, 0))
+    out = lt.verify(d["target_logits"], None, d["cfg_scale"], 0.0, d["draft_tokens"], d["tree_parents"], table,
+                    delta, None, trace=True)
+    torch.cuda.synchronize()
+    _properties(d, out, N, V)
+    rows = np.sort(np.random.default_rng(12).choice(B, size=min(sample, B), replace=False))
+    check_outputs(lid.to_host(d, rows=rows), table.cpu().numpy(), delta, _take(out, rows))
+    out2 = lt.verify(d["target_logits"], None, d["cfg_scale"], 0.0, d["draft_tokens"], d["tree_parents"], table,
+                     delta, None)
+    torch.cuda.synchronize()
+    assert torch.equal(out.accept_len, out2.accept_len) and torch.equal(out.next_token, out2.next_token)
+    assert torch.equal(out.accept_path, out2.accept_path)

@@ -508,13 +508,24 @@ static cudaError_t launch_verify(const VerifyParams& P, int grid_ctx, int grid_b
 }
 
 template <bool BF16, bool UNC>
-static cudaError_t launch_greedy(const VerifyParams& P, int grid_ctx, int grid_bonus, cudaStream_t st) {
+static cudaError_t launch_greedy(const VerifyParams& P, long long items, int sms, int grid_bonus, cudaStream_t st) {
   auto kc = lantern_greedy_context_kernel<BF16, UNC>;
-  const size_t smem = static_cast<size_t>(P.V) * sizeof(float);
+  // a ring of staging areas per CTA, each holding the raw target rows of one context; sized so that
+  // three CTAs share an SM where the rows allow it
+  const size_t area = static_cast<size_t>(P.V) * (UNC ? 2 : 1) * (BF16 ? 2 : 4);
+  int ring = static_cast<int>((72 * 1024) / area);
+  ring = ring < 1 ? 1 : (ring > GRING_MAX ? GRING_MAX : ring);
+  const size_t smem = ring * area;
   cudaError_t e = cudaFuncSetAttribute(kc, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return e;
+  int per_sm = 0;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kc, GCT, smem);
+  if (e != cudaSuccess) return e;
+  if (per_sm < 1) return cudaErrorInvalidConfiguration;
+  const long long slots = static_cast<long long>(sms) * per_sm;
+  const int grid_ctx = static_cast<int>(items < slots ? items : slots);
   if (g_ev_before && g_ev_after) cudaEventRecord(g_ev_before, st);
-  kc<<<grid_ctx, GRT, smem, st>>>(P);
+  kc<<<grid_ctx, GCT, smem, st>>>(P, ring);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (g_ev_before && g_ev_after) cudaEventRecord(g_ev_after, st);
@@ -625,9 +636,8 @@ extern "C" lantern_status lantern_verify(const void* target_logits, const void* 
   cudaError_t e;
   const bool bf = dtype == LANTERN_BF16, un = has_uncond != 0;
   if (greedy) {
-    const int grid_g = static_cast<int>(items < 8ll * sms ? items : 8ll * sms);
-    e = bf ? (un ? launch_greedy<true, true>(P, grid_g, grid_bonus, st) : launch_greedy<true, false>(P, grid_g, grid_bonus, st))
-           : (un ? launch_greedy<false, true>(P, grid_g, grid_bonus, st) : launch_greedy<false, false>(P, grid_g, grid_bonus, st));
+    e = bf ? (un ? launch_greedy<true, true>(P, items, sms, grid_bonus, st) : launch_greedy<true, false>(P, items, sms, grid_bonus, st))
+           : (un ? launch_greedy<false, true>(P, items, sms, grid_bonus, st) : launch_greedy<false, false>(P, items, sms, grid_bonus, st));
     return e == cudaSuccess ? LANTERN_OK : LANTERN_E_CUDA;
   }
 #define LANTERN_DISPATCH2(CHV, TV)                                                                   \

@@ -6,9 +6,9 @@
 // sum_A q >= max_x q(x) (the maximum over A's own members can never exceed the sum).  There is no
 // drafter distribution, no residual and no random number: children of a context are tried in
 // node order against the same q, and wherever the walk stops the next token is arg max q
-// (smallest index on ties).  One CTA per context with children: two sweeps over the context's
-// two target rows (maximum and arg max; numerators into shared memory and their sum), then per
-// child the same gather + double-precision prefix scan against the strict bound as in sampling.
+// (smallest index on ties).  Per context with children: one sweep over the staged target rows
+// (maximum, arg max, normaliser), then per child the same gather + double-precision prefix scan
+// against the strict bound as in sampling.
 #pragma once
 
 namespace lantern {
@@ -112,139 +112,354 @@ __device__ __forceinline__ bool greedy_argmax(const VerifyParams& P, size_t item
   return ok;
 }
 
+// ---------------------------------------------------------------------------------------
+// Context kernel: persistent CTAs of GCT threads, three to an SM where the rows allow it, each
+// working through its contexts in order.
+//
+// Greedy decoding needs, of a context's distribution, only its maximum, its arg max, the
+// normaliser Z and the numerators of the ~k tokens the children's neighbour rows name.  So the
+// raw target rows are staged in shared memory by bulk copy and never rewritten: one sweep reads
+// them once (guidance combine, running maximum / arg max, and a running sum of numerators taken
+// against the thread's own running maximum and rescaled whenever that maximum moves), a block
+// reduction turns the per-thread (maximum, sum) pairs into (M, arg max, Z), and the gather
+// recomputes the numerator 2^((z - M) log2 e) of each token it touches from the staged bytes.
+// Because nothing is written back, the staging areas of a CTA form a simple ring (one area for
+// 16384 bf16 tokens, more for smaller rows); the copies of one CTA run under the arithmetic of
+// the other CTAs of its SM.
+// ---------------------------------------------------------------------------------------
+constexpr int GCT = 320;
+constexpr int GCW = GCT / 32;
+constexpr int GGT = 256;            // threads that gather: four neighbour slots each per round
+constexpr int GGW = GGT / 32;
+constexpr int GRING_MAX = 4;
+static_assert(GCW <= 32 && GGT <= GCT, "one warp combines the per-warp partials; gatherers are a subset");
+
+struct GreedyCtxShared {
+  double ws[GCW];                   // per-warp sums of numerators relative to the warp's maximum
+  double wt[GGW];
+  double sbefore[GGW];
+  float wm[GCW];
+  int wi[GCW];
+  int first[GGW];
+  double Z;
+  float M;
+  int arg;
+  int flags[2];                     // bit 0: NaN met, bit 1: a copy did not arrive (by iteration parity)
+  int status;
+  int done, accept;
+  unsigned long long bar_full[GRING_MAX];
+};
+
+// a neighbour entry, by an instruction the compiler neither hoists nor merges into a select
+__device__ __forceinline__ int ld_nc_s32(const int32_t* p) {
+  int v;
+  asm volatile("ld.global.nc.s32 %0, [%1];" : "=r"(v) : "l"(p));
+  return v;
+}
+
+__device__ __forceinline__ float greedy_ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// four processed logits (guidance combine, T = 1) of quad `qd` from the staged raw rows
 template <bool BF16, bool UNC>
-__global__ void __launch_bounds__(GRT) lantern_greedy_context_kernel(VerifyParams P) {
-  extern __shared__ __align__(16) float Eg[];   // numerators 2^((z - M) log2 e), plain token order
-  __shared__ GreedyShared S;
+__device__ __forceinline__ float4 greedy_quad(const unsigned char* area, uint32_t rowbytes, int qd, float s) {
+  float4 c, u;
+  if (BF16) {
+    const uint2 x = *reinterpret_cast<const uint2*>(area + static_cast<size_t>(qd) * 8);
+    c = make_float4(__uint_as_float(x.x << 16), __uint_as_float(x.x & 0xffff0000u), __uint_as_float(x.y << 16),
+                    __uint_as_float(x.y & 0xffff0000u));
+    if (UNC) {
+      const uint2 y = *reinterpret_cast<const uint2*>(area + rowbytes + static_cast<size_t>(qd) * 8);
+      u = make_float4(__uint_as_float(y.x << 16), __uint_as_float(y.x & 0xffff0000u), __uint_as_float(y.y << 16),
+                      __uint_as_float(y.y & 0xffff0000u));
+    }
+  } else {
+    c = *reinterpret_cast<const float4*>(area + static_cast<size_t>(qd) * 16);
+    if (UNC) u = *reinterpret_cast<const float4*>(area + rowbytes + static_cast<size_t>(qd) * 16);
+  }
+  if (UNC) {
+    c.x = __fmaf_rn(s, __fsub_rn(c.x, u.x), u.x);
+    c.y = __fmaf_rn(s, __fsub_rn(c.y, u.y), u.y);
+    c.z = __fmaf_rn(s, __fsub_rn(c.z, u.z), u.z);
+    c.w = __fmaf_rn(s, __fsub_rn(c.w, u.w), u.w);
+  }
+  return c;
+}
+
+// the processed logit of one token, by the same operations as greedy_quad
+template <bool BF16, bool UNC>
+__device__ __forceinline__ float greedy_one(const unsigned char* area, uint32_t rowbytes, int n, float s) {
+  float c, u = 0.0f;
+  if (BF16) {
+    c = __uint_as_float(static_cast<uint32_t>(*reinterpret_cast<const unsigned short*>(area + 2 * static_cast<size_t>(n))) << 16);
+    if (UNC)
+      u = __uint_as_float(static_cast<uint32_t>(*reinterpret_cast<const unsigned short*>(area + rowbytes + 2 * static_cast<size_t>(n))) << 16);
+  } else {
+    c = *reinterpret_cast<const float*>(area + 4 * static_cast<size_t>(n));
+    if (UNC) u = *reinterpret_cast<const float*>(area + rowbytes + 4 * static_cast<size_t>(n));
+  }
+  return UNC ? __fmaf_rn(s, __fsub_rn(c, u), u) : c;
+}
+
+template <bool BF16, bool UNC>
+__device__ __forceinline__ void greedy_issue_rows(const VerifyParams& P, int item, unsigned char* raw, uint32_t rowbytes,
+                                                  unsigned long long* bar) {
+  const size_t esize = BF16 ? 2 : 4;
+  const unsigned char* base = static_cast<const unsigned char*>(P.target);
+  const size_t row = static_cast<size_t>(item) * P.V * esize;
+  const size_t branch = static_cast<size_t>(P.B) * P.R * P.V * esize;
+  mbar_expect_tx(reinterpret_cast<uint64_t*>(bar), UNC ? 2 * rowbytes : rowbytes);
+  bulk_load(raw, base + row, rowbytes, reinterpret_cast<uint64_t*>(bar));
+  if (UNC) bulk_load(raw + rowbytes, base + branch + row, rowbytes, reinterpret_cast<uint64_t*>(bar));
+}
+
+template <bool BF16, bool UNC>
+__global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyParams P, int ring) {
+  extern __shared__ __align__(128) unsigned char gsm[];
+  __shared__ GreedyCtxShared S;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int V = P.V, N = P.N, R = P.R, k = P.k;
+  const uint32_t rowbytes = static_cast<uint32_t>(V) * (BF16 ? 2 : 4);
+  const uint32_t area_bytes = (UNC ? 2 : 1) * rowbytes;   // a multiple of 16: V % 8 == 0
   const float L_hi = 1.44269502162933349609375f;
+  const float NEG_INF = __int_as_float(0xff800000);
   const int n_heavy = P.counters->n_heavy;
   const int total = n_heavy + P.counters->n_light;
   const int cap = P.B * N;
+  const int quads = V >> 2;
+  const int G = gridDim.x;
+  auto slot = [&](int w) { return w < n_heavy ? w : cap - 1 - (w - n_heavy); };
 
-  for (int w = blockIdx.x; w < total; w += gridDim.x) {
-    const WorkItem cur = P.work[w < n_heavy ? w : cap - 1 - (w - n_heavy)];
-    const size_t item = static_cast<size_t>(cur.item);
-    const int b = cur.item / R;
-    const ChildInfo* kids = P.children + cur.cbase;
-    if (tid == 0) S.status = 0;
+  if (tid == 0) {
+    for (int r = 0; r < ring; ++r) mbar_init(reinterpret_cast<uint64_t*>(&S.bar_full[r]), 1);
+    fence_mbar_init();
+    S.status = 0;
+    S.flags[0] = S.flags[1] = 0;
+    for (int r = 0; r < ring; ++r) {
+      const long long w = blockIdx.x + static_cast<long long>(r) * G;
+      if (w < total)
+        greedy_issue_rows<BF16, UNC>(P, P.work[slot(static_cast<int>(w))].item, gsm + static_cast<size_t>(r) * area_bytes,
+                                     rowbytes, &S.bar_full[r]);
+    }
+  }
+  __syncthreads();
+  if (static_cast<int>(blockIdx.x) >= total) return;   // nothing was requested for this CTA
 
-    float M;
-    int arg;
-    const bool finite = greedy_argmax<BF16, UNC>(P, item, S, M, arg);   // barriers inside
+  WorkItem cur = P.work[slot(blockIdx.x)];
+  uint32_t it = 0, phase = 0;
+  int buf = 0;
+  for (long long w = blockIdx.x; w < total; w += G, ++it) {
+    // Loads that are consumed much later are issued without any select on their result (clamped
+    // indices instead of predicates), so that no instruction waits for them before their use:
+    // the next context's descriptor, the context that will take over this staging area, and the
+    // first child's neighbour entries.
+    const long long w_next = w + G < total ? w + G : w;
+    const long long w_refill = w + static_cast<long long>(ring) * G;
+    const WorkItem nxt = P.work[slot(static_cast<int>(w_next))];
+    const int refill = P.work[slot(static_cast<int>(w_refill < total ? w_refill : w))].item;
+    int nb[4];
+    if (tid < GGT) {
+      const int32_t* nrow0 = P.nbr + static_cast<size_t>(cur.tok0) * k;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int j = 4 * tid + 1 + i;
+        nb[i] = __ldg(nrow0 + (j < k ? j : k - 1));   // slots j >= k are masked where they are used
+      }
+    }
+    unsigned char* raw = gsm + static_cast<size_t>(buf) * area_bytes;
+    const bool ok = mbar_wait(reinterpret_cast<uint64_t*>(&S.bar_full[buf]), phase);
+
+    // ---- the sweep: maximum, smallest arg max, numerators summed against the running maximum ----
+    float m = NEG_INF, ssum = 0.0f;
+    int mi = 0x7fffffff;
+#pragma unroll 4
+    for (int qd = tid; qd < quads; qd += GCT) {
+      const float4 z = greedy_quad<BF16, UNC>(raw, rowbytes, qd, P.cfg_scale);
+      const float old = m;
+      if (z.x > m) m = z.x, mi = 4 * qd;          // ascending index within a thread: strict > keeps
+      if (z.y > m) m = z.y, mi = 4 * qd + 1;      // the smallest index
+      if (z.z > m) m = z.z, mi = 4 * qd + 2;
+      if (z.w > m) m = z.w, mi = 4 * qd + 3;
+      if (m > old) ssum *= greedy_ex2((old - m) * L_hi);   // old = -inf: the factor is 0, and so was the sum
+      const float mL = m > NEG_INF ? m * L_hi : 0.0f;       // all -inf so far: every numerator is 2^-inf = 0
+      ssum += (greedy_ex2(__fmaf_rn(z.x, L_hi, -mL)) + greedy_ex2(__fmaf_rn(z.y, L_hi, -mL))) +
+              (greedy_ex2(__fmaf_rn(z.z, L_hi, -mL)) + greedy_ex2(__fmaf_rn(z.w, L_hi, -mL)));
+    }
+    // A NaN logit (or +inf, through inf - inf) makes the thread's sum NaN: no per-element test is needed.
+    const int bad = ssum != ssum;
+    {
+      const float wmx = warp_max(m);
+      const int wix = __reduce_min_sync(kFull, (m == wmx) ? mi : 0x7fffffff);
+      float f = ssum > 0.0f ? ssum * greedy_ex2(__fmaf_rn(m, L_hi, -(wmx * L_hi))) : 0.0f;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) f += __shfl_xor_sync(kFull, f, o);
+      if (lane == 0) {
+        S.wm[warp] = wmx;
+        S.wi[warp] = wix;
+        S.ws[warp] = static_cast<double>(f);
+      }
+    }
+    if (bad || !ok) atomicOr(&S.flags[it & 1], (bad ? 1 : 0) | (ok ? 0 : 2));
+    __syncthreads();   // A
+    if (warp == 0) {   // lane v combines warp v
+      const float v = lane < GCW ? S.wm[lane] : NEG_INF;
+      const int i = lane < GCW ? S.wi[lane] : 0x7fffffff;
+      const double sv = lane < GCW ? S.ws[lane] : 0.0;
+      const float Mx = warp_max(v);
+      const int ax = __reduce_min_sync(kFull, (v == Mx) ? i : 0x7fffffff);
+      double c = sv > 0.0 ? sv * static_cast<double>(greedy_ex2(__fmaf_rn(v, L_hi, -(Mx * L_hi)))) : 0.0;
+      c = warp_sum(c);
+      if (lane == 0) {
+        S.M = Mx;
+        S.arg = ax;
+        S.Z = c;
+        S.flags[(it + 1) & 1] = 0;   // last read before A of this iteration, next written after B
+      }
+    }
+    __syncthreads();   // B
+    const int flags = S.flags[it & 1];
+    const float M = S.M;
+    const int arg = S.arg;
+    const double Z = S.Z;
+    if (flags & 2) {   // a copy did not complete within the wait limit: flag the context and stop
+      if (tid == 0) {
+        Record rec = {-1, -1, LANTERN_ST_INTERNAL, 0};
+        P.records[cur.item] = rec;
+        // give the copies still on their way to the other staging areas the same bounded wait
+        for (int d = 1; d < ring; ++d) {
+          const long long wj = w + static_cast<long long>(d) * G;
+          const uint32_t j = it + d;
+          if (wj < total) mbar_wait(reinterpret_cast<uint64_t*>(&S.bar_full[j % ring]), (j / ring) & 1);
+        }
+      }
+      __syncthreads();
+      break;
+    }
+    const bool finite = !(flags & 1) && M > NEG_INF && M < __int_as_float(0x7f800000);
     int accepted = -1, status = 0;
     if (!finite) {
       status = LANTERN_ST_NONFINITE;
     } else {
-      // numerators and their sum
       const float mL = M * L_hi;
-      float part = 0.0f;
-      for (int g = tid; g * 8 < V; g += GRT) {
-        float z[8];
-        greedy_chunk<BF16, UNC>(P, item, g, z);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) z[e] = ex2_approx(__fmaf_rn(z[e], L_hi, -mL));
-        part += sum8(z);
-        *reinterpret_cast<float4*>(Eg + g * 8) = make_float4(z[0], z[1], z[2], z[3]);
-        *reinterpret_cast<float4*>(Eg + g * 8 + 4) = make_float4(z[4], z[5], z[6], z[7]);
-      }
-      double Z = warp_sum(static_cast<double>(part));
-      if (lane == 0) S.wt[warp] = Z;
-      __syncthreads();
-      Z = 0.0;
-#pragma unroll
-      for (int v = 0; v < GRW; ++v) Z += S.wt[v];
-      __syncthreads();
+      auto numer = [&](int n) {   // 2^((z_n - M) log2 e) from the staged bytes
+        return greedy_ex2(__fmaf_rn(greedy_one<BF16, UNC>(raw, rowbytes, n, P.cfg_scale), L_hi, -mL));
+      };
       const double thr = static_cast<double>(P.delta) * Z;   // the bound in units of the unnormalised sums
-      const double top = static_cast<double>(Eg[arg]);        // max_x q(x) in the same units
-
+      const ChildInfo* kids = P.children + cur.cbase;
       for (int ci = 0; ci < cur.nchild && accepted < 0; ++ci) {
-        const int4 info = __ldg(reinterpret_cast<const int4*>(kids + ci));
-        const int node = info.x, xt = info.y;
+        int node = cur.node0, xt = cur.tok0;
+        if (ci > 0) {
+          const int4 info = __ldg(reinterpret_cast<const int4*>(kids + ci));
+          node = info.x, xt = info.y;
+        }
         const int32_t* nrow = P.nbr + static_cast<size_t>(xt) * k;
         // A_{k,delta}(x~): gather + prefix scan with the strict bound (Algorithm 2, second block)
-        double carry = 0.0, sm = 0.0;
-        int m = k - 1;
-        bool cut = false;
-        for (int base = 0; base < k - 1 && !cut; base += 4 * GRT) {
-          double pre4[4];
+        double carry = 0.0;
+        for (int base = 0;; base += 4 * GGT) {
+          double pre4[4], run = 0.0, incl = 0.0;
           bool val4[4];
-          double run = 0.0;
+          if (tid < GGT) {
+            int nn[4];
+            if (ci == 0 && base == 0) {   // a real branch: the prefetched entries must not wait for a load
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const int j = base + 4 * tid + 1 + i;
-            val4[i] = j < k;
-            const int n = val4[i] ? __ldg(nrow + j) : -1;
-            const bool inr = val4[i] && static_cast<unsigned>(n) < static_cast<unsigned>(V);
-            if (val4[i] && !inr) atomicOr(&S.status, LANTERN_ST_BAD_TABLE);   // carries no mass
-            run += inr ? static_cast<double>(Eg[n]) : 0.0;
-            pre4[i] = run;
-          }
-          const double incl = warp_incl_scan(run, lane);
-          if (lane == 31) S.wt[warp] = incl;
-          __syncthreads();
-          double pre = 0.0, tot = 0.0;
+              for (int i = 0; i < 4; ++i) nn[i] = nb[i];
+            } else {
 #pragma unroll
-          for (int v = 0; v < GRW; ++v) {
-            const double t = S.wt[v];
-            if (v < warp) pre += t;
-            tot += t;
-          }
-          const double before = carry + pre + (incl - run);
-          int my_first = kNone;
-          double my_before = 0.0;
-#pragma unroll
-          for (int i = 3; i >= 0; --i) {
-            if (val4[i] && !(before + pre4[i] < thr)) {
-              my_first = base + 4 * tid + 1 + i;
-              my_before = i > 0 ? before + pre4[i > 0 ? i - 1 : 0] : before;
+              for (int i = 0; i < 4; ++i) {
+                const int j = base + 4 * tid + 1 + i;
+                nn[i] = ld_nc_s32(nrow + (j < k ? j : k - 1));
+              }
             }
-          }
-          const int wfirst = __reduce_min_sync(kFull, my_first);
-          if (wfirst != kNone && my_first == wfirst) {
-            S.first[warp] = wfirst;
-            S.sbefore[warp] = my_before;
-          } else if (wfirst == kNone && lane == 0) {
-            S.first[warp] = kNone;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int j = base + 4 * tid + 1 + i;
+              val4[i] = j < k;
+              const int n = nn[i];
+              const bool inr = val4[i] && static_cast<unsigned>(n) < static_cast<unsigned>(V);
+              if (val4[i] && !inr) atomicOr(&S.status, LANTERN_ST_BAD_TABLE);   // carries no mass
+              run += inr ? static_cast<double>(numer(n)) : 0.0;
+              pre4[i] = run;
+            }
+            incl = warp_incl_scan(run, lane);
+            if (lane == 31) S.wt[warp] = incl;
           }
           __syncthreads();
-          int gfirst = kNone, src = 0;
+          double tot = 0.0;
+          if (tid < GGT) {
+            double pre = 0.0;
 #pragma unroll
-          for (int v = GRW - 1; v >= 0; --v) {
-            const int f = S.first[v];
-            if (f != kNone && f <= gfirst) {
-              gfirst = f;
-              src = v;
+            for (int v = 0; v < GGW; ++v) {
+              const double t = S.wt[v];
+              if (v < warp) pre += t;
+              tot += t;
+            }
+            const double before = carry + pre + (incl - run);
+            int my_first = kNone;
+            double my_before = 0.0;
+#pragma unroll
+            for (int i = 3; i >= 0; --i) {
+              if (val4[i] && !(before + pre4[i] < thr)) {
+                my_first = base + 4 * tid + 1 + i;
+                my_before = i > 0 ? before + pre4[i > 0 ? i - 1 : 0] : before;
+              }
+            }
+            const int wfirst = __reduce_min_sync(kFull, my_first);
+            if (wfirst != kNone && my_first == wfirst) {
+              S.first[warp] = wfirst;
+              S.sbefore[warp] = my_before;
+            } else if (wfirst == kNone && lane == 0) {
+              S.first[warp] = kNone;
             }
           }
-          if (gfirst != kNone) {
-            m = gfirst - 1;
-            sm = S.sbefore[src];
-            cut = true;
-          } else {
-            carry += tot;
-            sm = carry;
+          __syncthreads();
+          if (warp == 0) {
+            const int f = lane < GGW ? S.first[lane] : kNone;
+            const int gfirst = __reduce_min_sync(kFull, f);
+            const bool last = base + 4 * GGT >= k - 1;
+            if (gfirst != kNone || last) {
+              double sm = carry + tot;
+              int mcut = k - 1;
+              if (gfirst != kNone) {
+                const unsigned who = __ballot_sync(kFull, f == gfirst);   // slot indices are distinct: one lane
+                sm = S.sbefore[__ffs(who) - 1];
+                mcut = gfirst - 1;
+              }
+              const double qa_un = static_cast<double>(numer(xt)) + sm;
+              const double top = static_cast<double>(numer(arg));   // max_x q(x) in the same units
+              if (lane == 0) {
+                S.done = 1;
+                S.accept = qa_un >= top;   // x~ is an arg max of q_{k,delta}(.|D = x~); ties accept
+                const size_t o = static_cast<size_t>(cur.item / R) * N + node;
+                if (P.out_qa) P.out_qa[o] = static_cast<float>(qa_un / Z);
+                if (P.out_px) P.out_px[o] = 0.0f;   // no drafter probability enters greedy decoding
+                if (P.out_m) P.out_m[o] = mcut;
+              }
+            } else if (lane == 0) {
+              S.done = 0;
+            }
           }
-          __syncthreads();   // S.wt / S.first are rewritten by the next round or the next child
+          carry += tot;
+          __syncthreads();
+          if (S.done) break;
         }
-        const double qa_un = static_cast<double>(Eg[xt]) + sm;
-        const bool accept = qa_un >= top;   // x~ is an arg max of q_{k,delta}(.|D = x~); ties accept
-        if (tid == 0) {
-          const size_t o = static_cast<size_t>(b) * N + node;
-          if (P.out_qa) P.out_qa[o] = static_cast<float>(qa_un / Z);
-          if (P.out_px) P.out_px[o] = 0.0f;   // no drafter probability enters greedy decoding
-          if (P.out_m) P.out_m[o] = m;
-        }
-        if (accept) accepted = node;
+        if (S.accept) accepted = node;
       }
     }
-    __syncthreads();   // every status bit is in; Eg is free for the next context
+    // every thread's reads of this staging area came before the barrier it passed last
     if (tid == 0) {
+      if (w_refill < total) greedy_issue_rows<BF16, UNC>(P, refill, raw, rowbytes, &S.bar_full[buf]);
       Record rec = {accepted, finite ? arg : -1, status | S.status, 0};
-      P.records[item] = rec;
+      P.records[cur.item] = rec;
+      S.status = 0;
     }
-    __syncthreads();
+    cur = nxt;
+    if (++buf == ring) {
+      buf = 0;
+      phase ^= 1;
+    }
   }
 }
 

@@ -18,6 +18,7 @@ _SRC = os.path.join(_HERE, "lantern_oracle.cpp")
 _LIB = os.path.join(_HERE, "liblantern_oracle.so")
 
 ST_BAD_TOKEN, ST_BAD_PARENT, ST_BAD_UNIFORM, ST_NONFINITE, ST_DEGENERATE, ST_BAD_TABLE = 1, 2, 4, 8, 16, 32
+DIV_TVD, DIV_JSD = 0, 1
 
 
 def build(force: bool = False) -> str:
@@ -36,6 +37,7 @@ def _load():
     if _lib is None:
         _lib = ctypes.CDLL(build())
         _lib.oracle_count_order_differences.restype = ctypes.c_int64
+        _lib.oracle_jsd_collapsed.restype = ctypes.c_double
     return _lib
 
 
@@ -43,10 +45,24 @@ def _p(a: Optional[np.ndarray]):
     return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
 
 
-def build_neighbors(codebook: np.ndarray, k: int, rows: Optional[np.ndarray] = None):
-    """B_k for every code, or for the codes listed in `rows` (Algorithm 2, precompute block).
-    Returns idx [n, k] int32, dist [n, k] fp32 with n = V or len(rows)."""
+def normalize_rows(codebook: np.ndarray) -> np.ndarray:
+    """Codes scaled to unit length in the canonical fp32 sequence (cosine variant, Section 6.2.1)."""
     cb = np.ascontiguousarray(codebook, dtype=np.float32)
+    out = np.empty_like(cb)
+    rc = _load().oracle_normalize_rows(_p(cb), cb.shape[0], cb.shape[1], _p(out))
+    if rc != 0:
+        raise ValueError(f"oracle_normalize_rows: bad arguments ({rc})")
+    return out
+
+
+def build_neighbors(codebook: np.ndarray, k: int, rows: Optional[np.ndarray] = None, metric: str = "l2"):
+    """B_k for every code, or for the codes listed in `rows` (Algorithm 2, precompute block).
+    metric "l2" (the paper's choice) or "cosine" (Section 6.2.1: the same routine on unit-length codes).
+    Returns idx [n, k] int32, dist [n, k] fp32 with n = V or len(rows)."""
+    assert metric in ("l2", "cosine")
+    cb = np.ascontiguousarray(codebook, dtype=np.float32)
+    if metric == "cosine":
+        cb = normalize_rows(cb)
     V, D = cb.shape
     rw = None if rows is None else np.ascontiguousarray(rows, dtype=np.int32)
     n = V if rw is None else rw.shape[0]
@@ -66,28 +82,36 @@ def count_order_differences(codebook: np.ndarray, idx: np.ndarray) -> int:
 
 
 def row_distribution(row_c: np.ndarray, row_u: Optional[np.ndarray], dtype: int, cfg_scale: float,
-                     T: float) -> np.ndarray:
-    """softmax((l_u + s (l_c - l_u)) / T) of one context row, in double precision."""
+                     T: float, top_k: int = 0) -> np.ndarray:
+    """softmax((l_u + s (l_c - l_u)) / T) of one context row, in double precision; top_k > 0 first
+    sets the processed logits below the top_k-th largest to -inf (Appendix B.2)."""
     rc_ = np.ascontiguousarray(row_c)
     ru_ = None if row_u is None else np.ascontiguousarray(row_u)
     V = rc_.shape[0]
     out = np.empty(V, dtype=np.float64)
-    rc = _load().oracle_row_distribution(_p(rc_), _p(ru_), int(dtype), int(ru_ is not None),
-                                         ctypes.c_float(cfg_scale), ctypes.c_float(T), V, _p(out))
+    rc = _load().oracle_row_distribution_topk(_p(rc_), _p(ru_), int(dtype), int(ru_ is not None),
+                                              ctypes.c_float(cfg_scale), ctypes.c_float(T), int(top_k), V, _p(out))
     if rc != 0:
         raise ValueError(f"oracle_row_distribution failed ({rc})")
     return out
 
 
-def a_set(q: np.ndarray, nbr_row: np.ndarray, delta: float):
-    """Size (beyond x~) and moved mass of A_{k,delta}(x~) on distribution q (Algorithm 2, second block)."""
+def jsd_collapsed(q0: float, S: float) -> float:
+    """JSD (natural log) between q and q_{k,delta}(.|D = x~) when A moves mass S onto x~, q(x~) = q0."""
+    return float(_load().oracle_jsd_collapsed(ctypes.c_double(q0), ctypes.c_double(S)))
+
+
+def a_set(q: np.ndarray, nbr_row: np.ndarray, delta: float, divergence: int = DIV_TVD):
+    """Size (beyond x~) and moved mass of A_{k,delta}(x~) on distribution q (Algorithm 2, second block);
+    the bound is on the TVD (Section 4.3) or on the JSD (Section 6.2.2).  nbr_row[0] is x~."""
     q_ = np.ascontiguousarray(q, dtype=np.float64)
     nb = np.ascontiguousarray(nbr_row, dtype=np.int32)
     moved = ctypes.c_double(0.0)
     margin = ctypes.c_double(0.0)
     bad = ctypes.c_int(0)
-    m = _load().oracle_a_set(_p(q_), q_.shape[0], _p(nb), nb.shape[0], ctypes.c_double(delta),
-                             ctypes.byref(moved), ctypes.byref(margin), ctypes.byref(bad))
+    m = _load().oracle_a_set_div(_p(q_), q_.shape[0], _p(nb), nb.shape[0], ctypes.c_double(delta), int(divergence),
+                                 ctypes.c_double(q_[nb[0]]), ctypes.byref(moved), ctypes.byref(margin),
+                                 ctypes.byref(bad))
     return int(m), moved.value, margin.value
 
 
@@ -109,7 +133,7 @@ class VerifyResult:
 
 def verify(target_logits: np.ndarray, draft_logits: np.ndarray, dtype: int, cfg_scale: float, has_uncond: int,
            T: float, draft_tokens: np.ndarray, tree_parents: Optional[np.ndarray], neighbor_idx: np.ndarray,
-           delta: float, uniforms: np.ndarray) -> VerifyResult:
+           delta: float, uniforms: np.ndarray, divergence: int = DIV_TVD, top_k: int = 0) -> VerifyResult:
     """One verification call on host arrays (same layouts as the library's lantern_verify)."""
     tl = np.ascontiguousarray(target_logits)
     dl = np.ascontiguousarray(draft_logits)
@@ -131,9 +155,10 @@ def verify(target_logits: np.ndarray, draft_logits: np.ndarray, dtype: int, cfg_
         tested=np.zeros((B, N), np.uint8), qa=np.zeros((B, N)), px=np.zeros((B, N)),
         m=np.full((B, N), -1, np.int32), margin=np.full((B, N), np.inf), w=np.zeros(B),
         draw_margin=np.full(B, np.inf), qa_mag=np.zeros((B, N)))
-    rc = _load().oracle_verify(
+    rc = _load().oracle_verify_ex(
         _p(tl), _p(dl), int(dtype), ctypes.c_float(cfg_scale), int(has_uncond), ctypes.c_float(T), _p(tok),
-        _p(par), _p(nb), int(k), ctypes.c_float(delta), _p(un), B, N, V, _p(res.accept_len),
+        _p(par), _p(nb), int(k), ctypes.c_float(delta), int(divergence), int(top_k), _p(un), B, N, V,
+        _p(res.accept_len),
         _p(res.next_token), _p(res.accept_path), _p(res.status), _p(res.tested), _p(res.qa), _p(res.px),
         _p(res.m), _p(res.margin), _p(res.w), _p(res.draw_margin), _p(res.qa_mag))
     if rc != 0:
@@ -141,10 +166,11 @@ def verify(target_logits: np.ndarray, draft_logits: np.ndarray, dtype: int, cfg_
     return res
 
 
-def verify_inputs(inp, neighbor_idx: np.ndarray, delta: float) -> VerifyResult:
+def verify_inputs(inp, neighbor_idx: np.ndarray, delta: float, divergence: int = DIV_TVD,
+                  top_k: int = 0) -> VerifyResult:
     """Convenience: run `verify` on a lantern_inputs.VerifyInputs bundle."""
     return verify(inp.target_logits, inp.draft_logits, inp.dtype, inp.cfg_scale, inp.has_uncond, inp.T,
-                  inp.draft_tokens, inp.tree_parents, neighbor_idx, delta, inp.uniforms)
+                  inp.draft_tokens, inp.tree_parents, neighbor_idx, delta, inp.uniforms, divergence, top_k)
 
 
 @dataclasses.dataclass
@@ -161,7 +187,7 @@ class GreedyResult:
 
 def verify_greedy(target_logits: np.ndarray, dtype: int, cfg_scale: float, has_uncond: int,
                   draft_tokens: np.ndarray, tree_parents: Optional[np.ndarray], neighbor_idx: np.ndarray,
-                  delta: float) -> GreedyResult:
+                  delta: float, divergence: int = DIV_TVD, top_k: int = 0) -> GreedyResult:
     """Greedy-decoding verification (Section 4.3, last sentence) on host arrays."""
     tl = np.ascontiguousarray(target_logits)
     C, B, R, V = tl.shape
@@ -176,8 +202,9 @@ def verify_greedy(target_logits: np.ndarray, dtype: int, cfg_scale: float, has_u
                        accept_path=np.full((B, N), -1, np.int32), status=np.zeros(B, np.int32),
                        tested=np.zeros((B, N), np.uint8), qa=np.zeros((B, N)), m=np.full((B, N), -1, np.int32),
                        margin=np.full((B, N), np.inf))
-    rc = _load().oracle_verify_greedy(_p(tl), int(dtype), ctypes.c_float(cfg_scale), int(has_uncond), _p(tok), _p(par),
-                                      _p(nb), int(nb.shape[1]), ctypes.c_float(delta), B, N, V, _p(res.accept_len),
+    rc = _load().oracle_verify_greedy_ex(_p(tl), int(dtype), ctypes.c_float(cfg_scale), int(has_uncond), _p(tok),
+                                         _p(par), _p(nb), int(nb.shape[1]), ctypes.c_float(delta), int(divergence),
+                                         int(top_k), B, N, V, _p(res.accept_len),
                                       _p(res.next_token), _p(res.accept_path), _p(res.status), _p(res.tested),
                                       _p(res.qa), _p(res.m), _p(res.margin))
     if rc != 0:

@@ -127,6 +127,16 @@ int inverse_cdf(const std::vector<double>& w, double u, double* margin) {
 
 extern "C" {
 
+// variants (declared ahead of their first use)
+enum { DIV_TVD = 0, DIV_JSD = 1 };
+static void top_k_filter(std::vector<float>& z, int K);
+int oracle_row_distribution_topk(const void* row_c, const void* row_u, int dtype, int has_uncond,
+                                 float cfg_scale, float T, int top_k, int V, double* out);
+double oracle_jsd_collapsed(double q0, double S);
+int oracle_a_set_div(const double* q, int V, const int32_t* nbr_row, int k, double delta, int divergence,
+                     double q0, double* moved, double* cut_margin, int* bad_entry);
+
+
 // ---------------------------------------------------------------------------------------
 // Algorithm 2, first block: for every code, its k nearest codes (itself included), stored
 // in increasing distance.  R1 fixes the key.  Returns 0, or -1 on bad arguments.
@@ -172,6 +182,26 @@ int oracle_build_neighbors_rows(const float* codebook, int V, int D, int k, cons
   return 0;
 }
 
+// ---------------------------------------------------------------------------------------
+// Cosine variant of the latent proximity (Section 6.2.1): every code is scaled to unit length
+// and B_k is then built on the scaled codes with the same distance routine -- on unit vectors
+// the squared distance is 2 - 2 cos, so the order is that of decreasing cosine similarity.
+// Canonical fp32 sequence: squared norm accumulated in dimension order with one fused
+// multiply-add per dimension, one square root, one division per component.  A zero code stays
+// zero (its similarity to everything is taken as 0).
+// ---------------------------------------------------------------------------------------
+int oracle_normalize_rows(const float* codebook, int V, int D, float* out) {
+  if (!codebook || !out || V < 1 || D < 1) return -1;
+  for (int i = 0; i < V; ++i) {
+    const float* a = codebook + static_cast<size_t>(i) * D;
+    float n2 = 0.0f;
+    for (int d = 0; d < D; ++d) n2 = std::fmaf(a[d], a[d], n2);
+    const float n = std::sqrt(n2);
+    for (int d = 0; d < D; ++d) out[static_cast<size_t>(i) * D + d] = n > 0.0f ? a[d] / n : 0.0f;
+  }
+  return 0;
+}
+
 int oracle_build_neighbors(const float* codebook, int V, int D, int k, int32_t* idx, float* dist) {
   return oracle_build_neighbors_rows(codebook, V, D, k, nullptr, V, idx, dist);
 }
@@ -213,13 +243,19 @@ int64_t oracle_count_order_differences(const float* codebook, int V, int D, int 
 // ---------------------------------------------------------------------------------------
 int oracle_row_distribution(const void* row_c, const void* row_u, int dtype, int has_uncond,
                             float cfg_scale, float T, int V, double* out) {
-  if (!(T > 0.0f) || V < 1) return -1;
+  return oracle_row_distribution_topk(row_c, row_u, dtype, has_uncond, cfg_scale, T, 0, V, out);
+}
+
+int oracle_row_distribution_topk(const void* row_c, const void* row_u, int dtype, int has_uncond,
+                                 float cfg_scale, float T, int top_k, int V, double* out) {
+  if (!(T > 0.0f) || V < 1 || top_k < 0) return -1;
   std::vector<float> z(V);
   for (int x = 0; x < V; ++x) {
     float lc = load_logit(row_c, dtype, x);
     float lu = has_uncond ? load_logit(row_u, dtype, x) : 0.0f;
     z[x] = target_z(lc, lu, has_uncond, cfg_scale, T);
   }
+  top_k_filter(z, top_k);
   std::vector<double> q;
   if (!softmax(z, q, nullptr)) return -2;
   std::memcpy(out, q.data(), sizeof(double) * V);
@@ -233,6 +269,33 @@ int oracle_row_distribution(const void* row_c, const void* row_u, int dtype, int
 // ---------------------------------------------------------------------------------------
 int oracle_a_set(const double* q, int V, const int32_t* nbr_row, int k, double delta, double* moved,
                  double* cut_margin, int* bad_entry) {
+  return oracle_a_set_div(q, V, nbr_row, k, delta, DIV_TVD, 0.0, moved, cut_margin, bad_entry);
+}
+
+// ---------------------------------------------------------------------------------------
+// Jensen-Shannon divergence (natural logarithm) between q and q_{k,delta}(.|D = x~) when A
+// holds x~ with q(x~) = q0 and further tokens of total mass S (Section 6.2.2 names the
+// divergence; the formula is its definition written out on the only tokens where the two
+// distributions differ).  With mid = (q + q')/2:
+//   a token y of A other than x~ has q' = 0, mid = q(y)/2: it adds q(y) ln 2;
+//   x~ has q = q0, q' = q0 + S, mid = q0 + S/2;
+//   everywhere else q = q' and the terms vanish.
+// The natural logarithm is the base under which the paper's matched pairs agree (Table 3:
+// TVD 0.3 <-> JSD 0.2, TVD 0.2 <-> JSD 0.13, and S ln 2 = 0.208, 0.139 for small q0).
+// ---------------------------------------------------------------------------------------
+double oracle_jsd_collapsed(double q0, double S) {
+  const double Q = q0 + S, mid = q0 + 0.5 * S;
+  double t = S * std::log(2.0);
+  if (q0 > 0.0) t += q0 * std::log(q0 / mid);
+  if (Q > 0.0) t += Q * std::log(Q / mid);
+  return 0.5 * t;
+}
+
+// Algorithm 2's second block with the bound taken on the named divergence: TVD (the moved
+// mass, R4) or JSD.  q0 = q(x~) is used by JSD only.  cut_margin is in the divergence's units.
+int oracle_a_set_div(const double* q, int V, const int32_t* nbr_row, int k, double delta, int divergence,
+                     double q0, double* moved, double* cut_margin, int* bad_entry) {
+  auto div = [&](double mass) { return divergence == DIV_JSD ? oracle_jsd_collapsed(q0, mass) : mass; };
   double s = 0.0;
   int m = 0;
   if (bad_entry) *bad_entry = 0;
@@ -244,18 +307,36 @@ int oracle_a_set(const double* q, int V, const int32_t* nbr_row, int k, double d
     } else {
       qn = q[n];
     }
-    if (s + qn < delta) {  // strict bound (R3)
+    if (div(s + qn) < delta) {  // strict bound (R3)
       s += qn;
       m = j;
     } else {
       if (moved) *moved = s;
-      if (cut_margin) *cut_margin = std::min(std::fabs(s - delta), std::fabs(s + qn - delta));
+      if (cut_margin) *cut_margin = std::min(std::fabs(div(s) - delta), std::fabs(div(s + qn) - delta));
       return m;  // break at the first neighbour that does not fit
     }
   }
   if (moved) *moved = s;
-  if (cut_margin) *cut_margin = std::fabs(s - delta);
+  if (cut_margin) *cut_margin = std::fabs(div(s) - delta);
   return m;
+}
+
+// ---------------------------------------------------------------------------------------
+// Top-k logit filter (Appendix B.2: the generation settings use top-k 1000 / 2000 and top-p
+// 1.0, i.e. no nucleus cut): processed logits below the K-th largest become -inf; logits equal
+// to it are all kept.  K <= 0 or K >= V leaves the row as it is.  Applied to the target's and the
+// drafter's processed logits alike, before the softmax.
+// ---------------------------------------------------------------------------------------
+static void top_k_filter(std::vector<float>& z, int K) {
+  const int V = static_cast<int>(z.size());
+  if (K <= 0 || K >= V) return;
+  for (float v : z)
+    if (v != v) return;  // NaN: the softmax reports the row
+  std::vector<float> t(z);
+  std::nth_element(t.begin(), t.begin() + (K - 1), t.end(), [](float a, float b) { return a > b; });
+  const float kth = t[K - 1];
+  for (float& v : z)
+    if (v < kth) v = -std::numeric_limits<float>::infinity();
 }
 
 // ---------------------------------------------------------------------------------------
@@ -283,14 +364,18 @@ int oracle_a_set(const double* q, int V, const int32_t* nbr_row, int k, double d
 //   tr_draw_margin  margin of the final inverse-CDF draw
 // Returns 0 or a negative code for bad arguments.
 // ---------------------------------------------------------------------------------------
-int oracle_verify(const void* target_logits, const void* draft_logits, int dtype, float cfg_scale,
-                  int has_uncond, float T, const int32_t* draft_tokens, const int32_t* tree_parents,
-                  const int32_t* neighbor_idx, int k, float delta_f, const float* uniforms, int B, int N,
-                  int V, int32_t* out_accept_len, int32_t* out_next_token, int32_t* out_accept_path,
-                  int32_t* out_status, uint8_t* tr_tested, double* tr_qa, double* tr_px, int32_t* tr_m,
-                  double* tr_margin, double* tr_w, double* tr_draw_margin, double* tr_qa_mag) {
+// oracle_verify_ex adds the variants: `divergence` (DIV_TVD: Section 4.3 as written; DIV_JSD:
+// Section 6.2.2's alternative bound) and `top_k` (Appendix B.2's logit filter; 0 = none).
+int oracle_verify_ex(const void* target_logits, const void* draft_logits, int dtype, float cfg_scale,
+                     int has_uncond, float T, const int32_t* draft_tokens, const int32_t* tree_parents,
+                     const int32_t* neighbor_idx, int k, float delta_f, int divergence, int top_k,
+                     const float* uniforms, int B, int N, int V, int32_t* out_accept_len,
+                     int32_t* out_next_token, int32_t* out_accept_path, int32_t* out_status, uint8_t* tr_tested,
+                     double* tr_qa, double* tr_px, int32_t* tr_m, double* tr_margin, double* tr_w,
+                     double* tr_draw_margin, double* tr_qa_mag) {
   if (B < 0 || N < 0 || V < 1 || k < 1 || k > V) return -2;
   if (!(T > 0.0f) || !(delta_f >= 0.0f)) return -3;
+  if ((divergence != DIV_TVD && divergence != DIV_JSD) || top_k < 0) return -3;
   if (B == 0) return 0;
   if (!target_logits || !neighbor_idx || !uniforms || !out_accept_len || !out_next_token) return -1;
   if (N > 0 && (!draft_logits || !draft_tokens)) return -1;
@@ -353,6 +438,7 @@ int oracle_verify(const void* target_logits, const void* draft_logits, int dtype
         float lu = has_uncond ? load_logit(target_logits, dtype, branch + row + x) : 0.0f;
         z[x] = target_z(lc, lu, has_uncond, cfg_scale, T);
       }
+      top_k_filter(z, top_k);
       if (!softmax(z, q, nullptr)) {
         status |= ST_NONFINITE;
         break;
@@ -366,6 +452,7 @@ int oracle_verify(const void* target_logits, const void* draft_logits, int dtype
         break;
       }
       for (int x = 0; x < V; ++x) z[x] = load_logit(draft_logits, dtype, row + x) / T;
+      top_k_filter(z, top_k);
       if (!softmax(z, p, nullptr)) {
         status |= ST_NONFINITE;
         break;
@@ -381,7 +468,7 @@ int oracle_verify(const void* target_logits, const void* draft_logits, int dtype
         // A_{k,delta}(x~) on the current target (R3, R4)
         double moved = 0.0, cut_margin = 0.0;
         int bad = 0;
-        const int m = oracle_a_set(q.data(), V, nrow, k, delta, &moved, &cut_margin, &bad);
+        const int m = oracle_a_set_div(q.data(), V, nrow, k, delta, divergence, q[xt], &moved, &cut_margin, &bad);
         if (bad) status |= ST_BAD_TABLE;
         const double qa = q[xt] + moved;  // sum over A_{k,delta}(x~), x~ included (R5)
         const double px = p[xt];
@@ -474,13 +561,15 @@ int oracle_verify(const void* target_logits, const void* draft_logits, int dtype
 // Layouts as in oracle_verify.  Trace outputs per node [B, N] (each may be null): tr_tested,
 // tr_qa (sum_A q), tr_m (|A| - 1), tr_margin (min of the cut margin and |sum_A q - max_{x not in A} q|).
 // ---------------------------------------------------------------------------------------
-int oracle_verify_greedy(const void* target_logits, int dtype, float cfg_scale, int has_uncond,
-                         const int32_t* draft_tokens, const int32_t* tree_parents, const int32_t* neighbor_idx,
-                         int k, float delta_f, int B, int N, int V, int32_t* out_accept_len,
-                         int32_t* out_next_token, int32_t* out_accept_path, int32_t* out_status,
-                         uint8_t* tr_tested, double* tr_qa, int32_t* tr_m, double* tr_margin) {
+int oracle_verify_greedy_ex(const void* target_logits, int dtype, float cfg_scale, int has_uncond,
+                            const int32_t* draft_tokens, const int32_t* tree_parents, const int32_t* neighbor_idx,
+                            int k, float delta_f, int divergence, int top_k, int B, int N, int V,
+                            int32_t* out_accept_len, int32_t* out_next_token, int32_t* out_accept_path,
+                            int32_t* out_status, uint8_t* tr_tested, double* tr_qa, int32_t* tr_m,
+                            double* tr_margin) {
   if (B < 0 || N < 0 || V < 1 || k < 1 || k > V) return -2;
   if (!(delta_f >= 0.0f)) return -3;
+  if ((divergence != DIV_TVD && divergence != DIV_JSD) || top_k < 0) return -3;
   if (B == 0) return 0;
   if (!target_logits || !neighbor_idx || !out_accept_len || !out_next_token) return -1;
   if (N > 0 && !draft_tokens) return -1;
@@ -525,6 +614,7 @@ int oracle_verify_greedy(const void* target_logits, int dtype, float cfg_scale, 
         float lu = has_uncond ? load_logit(target_logits, dtype, branch + row + x) : 0.0f;
         z[x] = target_z(lc, lu, has_uncond, cfg_scale, 1.0f);
       }
+      top_k_filter(z, top_k);
       if (!softmax(z, q, nullptr)) {
         status |= ST_NONFINITE;
         break;
@@ -538,7 +628,7 @@ int oracle_verify_greedy(const void* target_logits, int dtype, float cfg_scale, 
         const int32_t* nrow = neighbor_idx + static_cast<size_t>(xt) * k;
         double moved = 0.0, cut_margin = 0.0;
         int bad = 0;
-        const int m = oracle_a_set(q.data(), V, nrow, k, delta, &moved, &cut_margin, &bad);
+        const int m = oracle_a_set_div(q.data(), V, nrow, k, delta, divergence, q[xt], &moved, &cut_margin, &bad);
         if (bad) status |= ST_BAD_TABLE;
         const double qa = q[xt] + moved;
         std::fill(inA.begin(), inA.end(), 0);
@@ -572,6 +662,28 @@ int oracle_verify_greedy(const void* target_logits, int dtype, float cfg_scale, 
     if (out_status) out_status[b] = status;
   }
   return 0;
+}
+
+int oracle_verify(const void* target_logits, const void* draft_logits, int dtype, float cfg_scale,
+                  int has_uncond, float T, const int32_t* draft_tokens, const int32_t* tree_parents,
+                  const int32_t* neighbor_idx, int k, float delta_f, const float* uniforms, int B, int N,
+                  int V, int32_t* out_accept_len, int32_t* out_next_token, int32_t* out_accept_path,
+                  int32_t* out_status, uint8_t* tr_tested, double* tr_qa, double* tr_px, int32_t* tr_m,
+                  double* tr_margin, double* tr_w, double* tr_draw_margin, double* tr_qa_mag) {
+  return oracle_verify_ex(target_logits, draft_logits, dtype, cfg_scale, has_uncond, T, draft_tokens, tree_parents,
+                          neighbor_idx, k, delta_f, DIV_TVD, 0, uniforms, B, N, V, out_accept_len, out_next_token,
+                          out_accept_path, out_status, tr_tested, tr_qa, tr_px, tr_m, tr_margin, tr_w,
+                          tr_draw_margin, tr_qa_mag);
+}
+
+int oracle_verify_greedy(const void* target_logits, int dtype, float cfg_scale, int has_uncond,
+                         const int32_t* draft_tokens, const int32_t* tree_parents, const int32_t* neighbor_idx,
+                         int k, float delta_f, int B, int N, int V, int32_t* out_accept_len,
+                         int32_t* out_next_token, int32_t* out_accept_path, int32_t* out_status,
+                         uint8_t* tr_tested, double* tr_qa, int32_t* tr_m, double* tr_margin) {
+  return oracle_verify_greedy_ex(target_logits, dtype, cfg_scale, has_uncond, draft_tokens, tree_parents,
+                                 neighbor_idx, k, delta_f, DIV_TVD, 0, B, N, V, out_accept_len, out_next_token,
+                                 out_accept_path, out_status, tr_tested, tr_qa, tr_m, tr_margin);
 }
 
 }  // extern "C"

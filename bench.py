@@ -141,7 +141,7 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def oracle_sample_rate(host_inp, table_host, delta, budget_s=15.0, greedy=False):
+def oracle_sample_rate(host_inp, table_host, delta, budget_s=15.0, greedy=False, divergence=0):
     """Oracle throughput (drafted positions verified per second) on as many leading sequences of
     `host_inp` as fit in about `budget_s` seconds; returns (rate, n_sequences, seconds)."""
     import dataclasses
@@ -161,9 +161,9 @@ def oracle_sample_rate(host_inp, table_host, delta, budget_s=15.0, greedy=False)
         t0 = time.perf_counter()
         if greedy:
             oracle.verify_greedy(part.target_logits, part.dtype, part.cfg_scale, part.has_uncond, part.draft_tokens,
-                                 part.tree_parents, table_host, delta)
+                                 part.tree_parents, table_host, delta, divergence)
         else:
-            oracle.verify_inputs(part, table_host, delta)
+            oracle.verify_inputs(part, table_host, delta, divergence)
         t_used += time.perf_counter() - t0
         done += n
         pos += n * host_inp.N
@@ -205,13 +205,14 @@ def run_reference(args, rank, world):
     nseq = {"batch_chain": 64, "stress": 4, "px512_tree": 4, "single_image": 4, "tiny": 64}[args.workload]
     cb = li.config_codebook(w["config"])
     steps_t = []
+    div = oracle.DIV_JSD if args.divergence == "jsd" else oracle.DIV_TVD
     table_cache = {}   # the table is an input of the step: only the rows the sample's drafts touch are built
 
     def table_for(inp):
         need = np.unique(inp.draft_tokens)
         miss = np.array([t for t in need if t not in table_cache], dtype=np.int32)
         if miss.size:
-            idx, _ = oracle.build_neighbors(cb, cfg["k"], rows=miss)
+            idx, _ = oracle.build_neighbors(cb, cfg["k"], rows=miss, metric=args.metric)
             for r, t in enumerate(miss):
                 table_cache[int(t)] = idx[r]
         tab = np.zeros((cfg["V"], cfg["k"]), np.int32)
@@ -226,9 +227,9 @@ def run_reference(args, rank, world):
         t1 = time.perf_counter()
         if args.greedy:
             oracle.verify_greedy(inp.target_logits, inp.dtype, inp.cfg_scale, inp.has_uncond, inp.draft_tokens,
-                                 inp.tree_parents, tab, cfg["delta"])
+                                 inp.tree_parents, tab, cfg["delta"], div)
         else:
-            oracle.verify_inputs(inp, tab, cfg["delta"])
+            oracle.verify_inputs(inp, tab, cfg["delta"], div)
         dt = time.perf_counter() - t1
         if step >= args.warmup:
             steps_t.append(dt)
@@ -239,7 +240,8 @@ def run_reference(args, rank, world):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(steps_t),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": args.workload, "V": cfg["V"], "k": cfg["k"], "delta": cfg["delta"], "N": cfg["N"],
-                   "T": 0.0 if args.greedy else cfg["T"], "sequences_per_step": nseq},
+                   "T": 0.0 if args.greedy else cfg["T"], "divergence": args.divergence, "metric": args.metric,
+                   "sequences_per_step": nseq},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
                          "sample": f"{nseq} sequences x {cfg['N']} drafts per step of the {args.workload} workload "
                                    f"(bounded sample; neighbour rows built by the oracle outside the timed region)"},
@@ -261,6 +263,9 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--divergence", default="tvd", choices=["tvd", "jsd"],
+                    help="what delta bounds (Section 6.2.2); the JSD run uses the workload's delta as it is")
+    ap.add_argument("--metric", default="l2", choices=["l2", "cosine"], help="latent proximity of the table")
     ap.add_argument("--greedy", action="store_true",
                     help="run the workload at T = 0 (greedy decoding: no drafter rows, no random numbers)")
     args = ap.parse_args()
@@ -296,12 +301,13 @@ def main():
 
     # ---- one-time neighbour table (timed separately) ----
     cb = torch.from_numpy(li.config_codebook(w["config"])).cuda()
-    bws = torch.empty(max(lt.build_workspace_bytes(V, cfg["D"], k), 16), dtype=torch.uint8, device="cuda")
-    lt.build_neighbors(cb, k, with_dist=False, workspace=bws)      # warm-up
+    bws = torch.empty(max(lt.load_library().lantern_build_workspace_bytes_metric(V, cfg["D"], k, lt.METRICS[args.metric]), 256),
+                      dtype=torch.uint8, device="cuda")
+    lt.build_neighbors(cb, k, with_dist=False, workspace=bws, metric=args.metric)      # warm-up
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    table, _ = lt.build_neighbors(cb, k, with_dist=False, workspace=bws)
+    table, _ = lt.build_neighbors(cb, k, with_dist=False, workspace=bws, metric=args.metric)
     e1.record()
     torch.cuda.synchronize()
     build_ms = e0.elapsed_time(e1)
@@ -322,7 +328,7 @@ def main():
     def step():
         lt.verify(d["target_logits"], None if args.greedy else d["draft_logits"], d["cfg_scale"], T, d["draft_tokens"],
                   d["tree_parents"], table, delta, None if args.greedy else d["uniforms"], out=out, workspace=ws,
-                  stream=stream)
+                  stream=stream, divergence=args.divergence)
 
     for _ in range(args.warmup):
         step()
@@ -405,7 +411,8 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         n_s = min(B, 8192 if cfg["N"] <= 8 else 256)
         host_inp = lid.to_host(d, rows=np.arange(n_s))
-        rate, n_done, secs = oracle_sample_rate(host_inp, table.cpu().numpy(), delta, greedy=args.greedy)
+        rate, n_done, secs = oracle_sample_rate(host_inp, table.cpu().numpy(), delta, greedy=args.greedy,
+                                                divergence=1 if args.divergence == "jsd" else 0)
         cpu = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
                "sample": f"first {n_done} sequences ({n_done * N} drafted positions) of this call, {secs:.1f} s"}
 
@@ -417,7 +424,7 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": args.workload, "note": w["note"], "sequences_per_call": B, "drafts_per_sequence": N,
-                       "V": V, "k": k, "delta": delta, "cfg_scale": cfg["cfg_scale"], "T": T,
+                       "V": V, "k": k, "delta": delta, "cfg_scale": cfg["cfg_scale"], "T": T, "divergence": args.divergence, "metric": args.metric,
                        "logits": "bf16" if cfg["dtype"] == li.BF16 else "f32", "rho": args.rho,
                        "l2_policy": "inputs larger than L2 (%.2f GB of logits per call)" %
                                     ((d["target_logits"].numel() + (0 if args.greedy else d["draft_logits"].numel())) *

@@ -83,6 +83,28 @@ lantern_status lantern_build_neighbors(const float* codebook, int V, int D, int 
                                        void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Neighbour table under a named latent proximity (Section 6.2.1 compares the l2 distance with
+ * cosine similarity).  LANTERN_METRIC_L2 is lantern_build_neighbors.  LANTERN_METRIC_COSINE
+ * scales every code to unit length first -- squared norm accumulated in fp32 in dimension order
+ * by one fused multiply-add per dimension, one square root, one division per component; a zero
+ * code stays zero -- and builds the same table on the scaled codes: on unit vectors the squared
+ * distance is 2 - 2 cos, so rows come in decreasing cosine similarity, ties by smaller index,
+ * and dist holds 2 - 2 cos.
+ *
+ *   workspace  lantern_build_workspace_bytes_metric(V, D, k, metric) bytes, 256-byte aligned
+ *              (for the cosine metric it also holds the scaled codes)
+ *   other arguments, limits and return codes as for lantern_build_neighbors; an unknown metric
+ *   returns LANTERN_E_PARAM
+ * ---------------------------------------------------------------------------------------- */
+enum { LANTERN_METRIC_L2 = 0, LANTERN_METRIC_COSINE = 1 };
+
+size_t lantern_build_workspace_bytes_metric(int V, int D, int k, int metric);
+
+lantern_status lantern_build_neighbors_metric(const float* codebook, int V, int D, int k, int metric, int32_t* idx,
+                                              float* dist, void* workspace, size_t workspace_bytes,
+                                              void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
  * One verification step.  Algorithm 1, verification loop and the bonus-token line after it,
  * with the acceptance rule and residual of Section 4.3 and A_{k,delta} built as in
  * Algorithm 2's second block.
@@ -139,6 +161,39 @@ lantern_status lantern_verify(const void* target_logits, const void* draft_logit
                               int32_t* out_accept_path, int32_t* out_status, float* out_node_qa,
                               float* out_node_px, int32_t* out_node_m, void* workspace, size_t workspace_bytes,
                               void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
+ * lantern_verify with the variants of the paper's ablations and generation settings.
+ *
+ *   divergence  what delta bounds when A_{k,delta}(x~) is grown (Section 6.2.2):
+ *               LANTERN_DIV_TVD  the total variation distance between q and q_{k,delta}(.|D = x~),
+ *                                i.e. the mass moved onto x~ (Section 4.3; lantern_verify);
+ *               LANTERN_DIV_JSD  their Jensen-Shannon divergence with the natural logarithm,
+ *                                JSD = 1/2 [ S ln 2 + q0 ln(q0 / mid) + (q0 + S) ln((q0 + S) / mid) ],
+ *                                q0 = q(x~), S = the moved mass, mid = q0 + S / 2 (only the collapsed
+ *                                tokens differ between the two distributions).  Neighbours are
+ *                                still added in order of distance until the first one that would
+ *                                reach delta.
+ *   top_k       logit filter of the generation settings (Appendix B.2: top-k 1000 or 2000, top-p 1):
+ *               processed logits below the top_k-th largest of their row count as -inf, for the
+ *               target and for the drafter alike, before the softmax; logits equal to the
+ *               top_k-th largest are all kept.  0, or any value >= V, switches the filter off.
+ *   workspace   lantern_verify_workspace_bytes_ex(B, N, top_k) bytes, 256-byte aligned
+ *
+ * Everything else, and every return code, is as for lantern_verify; an unknown divergence or a
+ * negative top_k returns LANTERN_E_PARAM.
+ * ---------------------------------------------------------------------------------------- */
+enum { LANTERN_DIV_TVD = 0, LANTERN_DIV_JSD = 1 };
+
+size_t lantern_verify_workspace_bytes_ex(int B, int N, int top_k);
+
+lantern_status lantern_verify_ex(const void* target_logits, const void* draft_logits, int dtype, float cfg_scale,
+                                 int has_uncond, float T, const int32_t* draft_tokens, const int32_t* tree_parents,
+                                 const int32_t* neighbor_idx, int k, float delta, int divergence, int top_k,
+                                 const float* uniforms, int B, int N, int V, int32_t* out_accept_len,
+                                 int32_t* out_next_token, int32_t* out_accept_path, int32_t* out_status,
+                                 float* out_node_qa, float* out_node_px, int32_t* out_node_m, void* workspace,
+                                 size_t workspace_bytes, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
  * lantern_verify without a caller-supplied workspace.  (The paper has no counterpart: this

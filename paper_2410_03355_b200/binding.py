@@ -51,6 +51,15 @@ def load_library():
     lib.lantern_build_neighbors.argtypes = [vp, i32, i32, i32, vp, vp, vp, sz, vp]
     lib.lantern_verify_workspace_bytes.restype = sz
     lib.lantern_verify_workspace_bytes.argtypes = [i32, i32]
+    lib.lantern_build_workspace_bytes_metric.restype = sz
+    lib.lantern_build_workspace_bytes_metric.argtypes = [i32, i32, i32, i32]
+    lib.lantern_build_neighbors_metric.restype = i32
+    lib.lantern_build_neighbors_metric.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, sz, vp]
+    lib.lantern_verify_workspace_bytes_ex.restype = sz
+    lib.lantern_verify_workspace_bytes_ex.argtypes = [i32, i32, i32]
+    lib.lantern_verify_ex.restype = i32
+    lib.lantern_verify_ex.argtypes = [vp, vp, i32, f32, i32, f32, vp, vp, vp, i32, f32, i32, i32, vp, i32, i32, i32,
+                                      vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.lantern_kernel_revision.restype = i32
     lib.lantern_kernel_revision.argtypes = []
     lib.lantern_verify_launch_count.restype = i32
@@ -92,27 +101,34 @@ def build_workspace_bytes(V: int, D: int, k: int) -> int:
     return int(load_library().lantern_build_workspace_bytes(V, D, k))
 
 
-def build_neighbors(codebook: torch.Tensor, k: int, *, with_dist: bool = True,
+METRICS = {"l2": 0, "cosine": 1}
+DIVERGENCES = {"tvd": 0, "jsd": 1}
+
+
+def build_neighbors(codebook: torch.Tensor, k: int, *, with_dist: bool = True, metric: str = "l2",
                     workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
-    """lantern_build_neighbors: [V, D] fp32 codebook -> (idx [V, k] int32, dist [V, k] fp32 or None)."""
+    """lantern_build_neighbors[_metric]: [V, D] fp32 codebook -> (idx [V, k] int32, dist [V, k] fp32 or None).
+    metric "l2" (squared l2 distances) or "cosine" (dist = 2 - 2 cos on unit-length codes)."""
     lib = load_library()
     V, D = codebook.shape
+    if metric not in METRICS:
+        raise ValueError(f"metric must be one of {sorted(METRICS)}")
     with torch.cuda.device(codebook.device):
         idx = torch.empty((V, k), dtype=torch.int32, device=codebook.device)
         dist = torch.empty((V, k), dtype=torch.float32, device=codebook.device) if with_dist else None
-        need = build_workspace_bytes(V, D, k)
+        need = int(lib.lantern_build_workspace_bytes_metric(V, D, int(k), METRICS[metric]))
         if workspace is None and need:
             workspace = torch.empty(need, dtype=torch.uint8, device=codebook.device)
-        rc = lib.lantern_build_neighbors(_ptr(codebook, torch.float32, "codebook"), V, D, int(k), _ptr(idx),
-                                         _ptr(dist), _ptr(workspace), workspace.numel() if workspace is not None else 0,
-                                         _stream_ptr(stream))
+        rc = lib.lantern_build_neighbors_metric(
+            _ptr(codebook, torch.float32, "codebook"), V, D, int(k), METRICS[metric], _ptr(idx), _ptr(dist),
+            _ptr(workspace), workspace.numel() if workspace is not None else 0, _stream_ptr(stream))
     if rc != 0:
-        raise LanternError(rc, "lantern_build_neighbors")
+        raise LanternError(rc, "lantern_build_neighbors_metric")
     return idx, dist
 
 
-def verify_workspace_bytes(B: int, N: int) -> int:
-    return int(load_library().lantern_verify_workspace_bytes(B, N))
+def verify_workspace_bytes(B: int, N: int, top_k: int = 0) -> int:
+    return int(load_library().lantern_verify_workspace_bytes_ex(B, N, int(top_k)))
 
 
 @dataclasses.dataclass
@@ -129,14 +145,18 @@ class VerifyOutputs:
 def verify(target_logits: torch.Tensor, draft_logits: Optional[torch.Tensor], cfg_scale: float, T: float,
            draft_tokens: Optional[torch.Tensor], tree_parents: Optional[torch.Tensor], neighbor_idx: torch.Tensor,
            delta: float, uniforms: Optional[torch.Tensor], *, out: Optional[VerifyOutputs] = None, trace: bool = False,
-           workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None) -> VerifyOutputs:
-    """lantern_verify on torch tensors.
+           workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None,
+           divergence: str = "tvd", top_k: int = 0) -> VerifyOutputs:
+    """lantern_verify_ex on torch tensors (divergence "tvd" and top_k = 0 are lantern_verify).
 
     target_logits [C, B, N+1, V] (C = 2: conditional, unconditional; C = 1: no guidance), fp32 or bf16;
     draft_logits [B, N+1, V]; draft_tokens / tree_parents [B, N] int32 (tree_parents None = chain);
     neighbor_idx [V, k] int32; uniforms [B, N+1] fp32.  Outputs are allocated unless `out` is given.
     T == 0 selects greedy decoding: draft_logits and uniforms are not read and may be None.
+    divergence "tvd" | "jsd": what delta bounds (Section 6.2.2); top_k: logit filter, 0 = off (Appendix B.2).
     """
+    if divergence not in DIVERGENCES:
+        raise ValueError(f"divergence must be one of {sorted(DIVERGENCES)}")
     lib = load_library()
     if T != 0 and (uniforms is None or (draft_logits is None and target_logits.shape[2] > 1)):
         raise ValueError("sampling (T > 0) needs draft_logits and uniforms")
@@ -163,20 +183,20 @@ def verify(target_logits: torch.Tensor, draft_logits: Optional[torch.Tensor], cf
                 node_qa=torch.empty((B, N), dtype=torch.float32, device=dev) if trace else None,
                 node_px=torch.empty((B, N), dtype=torch.float32, device=dev) if trace else None,
                 node_m=torch.empty((B, N), **i32) if trace else None)
-        need = verify_workspace_bytes(B, N)
+        need = verify_workspace_bytes(B, N, top_k)
         if workspace is None:
             workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
-        rc = lib.lantern_verify(
+        rc = lib.lantern_verify_ex(
             _ptr(target_logits, None, "target_logits"), _ptr(draft_logits, target_logits.dtype, "draft_logits"),
             dtype, float(cfg_scale), int(C == 2), float(T), _ptr(draft_tokens, torch.int32, "draft_tokens"),
             _ptr(tree_parents, torch.int32, "tree_parents"), _ptr(neighbor_idx, torch.int32, "neighbor_idx"),
-            int(k), float(delta), _ptr(uniforms, torch.float32, "uniforms"), B, N, V,
-            _ptr(out.accept_len, torch.int32), _ptr(out.next_token, torch.int32),
+            int(k), float(delta), DIVERGENCES[divergence], int(top_k), _ptr(uniforms, torch.float32, "uniforms"),
+            B, N, V, _ptr(out.accept_len, torch.int32), _ptr(out.next_token, torch.int32),
             _ptr(out.accept_path, torch.int32), _ptr(out.status, torch.int32), _ptr(out.node_qa, torch.float32),
             _ptr(out.node_px, torch.float32), _ptr(out.node_m, torch.int32), _ptr(workspace),
             workspace.numel(), _stream_ptr(stream))
     if rc != 0:
-        raise LanternError(rc, "lantern_verify")
+        raise LanternError(rc, "lantern_verify_ex")
     return out
 
 

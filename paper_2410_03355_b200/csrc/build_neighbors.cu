@@ -327,3 +327,51 @@ extern "C" lantern_status lantern_build_neighbors(const float* codebook, int V, 
   }
   return LANTERN_OK;
 }
+
+// ---------------------------------------------------------------------------------------
+// Cosine variant of the latent proximity (Section 6.2.1): codes scaled to unit length, then the
+// same neighbour build -- on unit vectors the squared distance is 2 - 2 cos, so increasing
+// distance is decreasing cosine similarity.  One thread per code runs the canonical fp32
+// sequence: squared norm by one fused multiply-add per dimension in dimension order, one square
+// root, one division per component; a zero code stays zero.
+// ---------------------------------------------------------------------------------------
+namespace lantern {
+__global__ void lantern_normalize_rows_kernel(const float* __restrict__ codebook, float* __restrict__ out, int V,
+                                              int D) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= V) return;
+  const float* a = codebook + static_cast<size_t>(i) * D;
+  float n2 = 0.0f;
+  for (int d = 0; d < D; ++d) n2 = __fmaf_rn(a[d], a[d], n2);
+  const float n = __fsqrt_rn(n2);
+  for (int d = 0; d < D; ++d) out[static_cast<size_t>(i) * D + d] = n > 0.0f ? __fdiv_rn(a[d], n) : 0.0f;
+}
+}  // namespace lantern
+
+static size_t unit_codes_bytes(int V, int D) { return (static_cast<size_t>(V) * D * 4 + 255) & ~static_cast<size_t>(255); }
+
+extern "C" size_t lantern_build_workspace_bytes_metric(int V, int D, int k, int metric) {
+  if (V < 1 || D < 1 || (metric != LANTERN_METRIC_L2 && metric != LANTERN_METRIC_COSINE)) return 0;
+  const size_t base = lantern_build_workspace_bytes(V, D, k);
+  return metric == LANTERN_METRIC_COSINE ? unit_codes_bytes(V, D) + base : base;
+}
+
+extern "C" lantern_status lantern_build_neighbors_metric(const float* codebook, int V, int D, int k, int metric,
+                                                         int32_t* idx, float* dist, void* workspace,
+                                                         size_t workspace_bytes, void* cuda_stream) {
+  if (metric == LANTERN_METRIC_L2)
+    return lantern_build_neighbors(codebook, V, D, k, idx, dist, workspace, workspace_bytes, cuda_stream);
+  if (metric != LANTERN_METRIC_COSINE) return LANTERN_E_PARAM;
+  if (V < 1 || V > 32768 || D < 1 || D > 4096 || k < 1 || k > V || k > 4097) return LANTERN_E_SHAPE;
+  if (!codebook || !idx) return LANTERN_E_NULL;
+  const size_t unit = unit_codes_bytes(V, D);
+  if (!workspace || workspace_bytes < lantern_build_workspace_bytes_metric(V, D, k, metric) ||
+      (reinterpret_cast<uintptr_t>(workspace) & 255))
+    return LANTERN_E_WORKSPACE;
+  float* unit_codes = static_cast<float*>(workspace);
+  lantern::lantern_normalize_rows_kernel<<<(V + 127) / 128, 128, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      codebook, unit_codes, V, D);
+  if (cudaGetLastError() != cudaSuccess) return LANTERN_E_CUDA;
+  return lantern_build_neighbors(unit_codes, V, D, k, idx, dist, static_cast<unsigned char*>(workspace) + unit,
+                                 workspace_bytes - unit, cuda_stream);
+}

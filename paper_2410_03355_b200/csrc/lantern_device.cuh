@@ -52,6 +52,43 @@ __device__ __forceinline__ double warp_incl_scan(double v, int lane) {
 }
 
 // ---------------------------------------------------------------------------------------
+// JSD bound (Section 6.2.2).  Moving mass S onto a token of probability q0 changes the
+// distribution by JSD f(S) = 1/2 [ S ln 2 + q0 ln(q0 / mid) + (q0 + S) ln((q0 + S) / mid) ],
+// mid = q0 + S/2 (natural logarithm; only the collapsed tokens contribute).  f is increasing and
+// convex in S with f' = 1/2 [ln 2 + ln((q0 + S) / mid)], so "f(S) < delta" is "S < S*" with
+// f(S*) = delta, and the prefix test stays a comparison of a running sum with one number per
+// draft.  S* by Newton's method from the upper bound 2 delta / ln 2 (f >= S ln2 / 2): single
+// precision first, two double-precision steps to finish (relative error of f(S*) below 1e-9).
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ double jsd_mass_bound(double delta, double q0) {
+  if (!(delta > 0.0)) return 0.0;
+  const float LN2F = 0.693147182464599609375f;
+  const double LN2 = 0.69314718055994530942;
+  const float qf = static_cast<float>(q0), df = static_cast<float>(delta);
+  float Sf = 2.0f * df / LN2F;
+#pragma unroll 1
+  for (int it = 0; it < 5; ++it) {
+    const float Q = qf + Sf, mid = qf + 0.5f * Sf;
+    const float lq = __logf(Q / mid);
+    float t = Sf * LN2F + Q * lq;
+    if (qf > 0.0f) t += qf * __logf(qf / mid);
+    Sf -= (0.5f * t - df) / (0.5f * (LN2F + lq));
+    Sf = Sf > 0.0f ? Sf : 0.0f;
+  }
+  double S = static_cast<double>(Sf);
+  if (!(S > 0.0)) S = delta / LN2;
+#pragma unroll 1
+  for (int it = 0; it < 2; ++it) {
+    const double Q = q0 + S, mid = q0 + 0.5 * S;
+    const double lq = log(Q / mid);
+    double t = S * LN2 + Q * lq;
+    if (q0 > 0.0) t += q0 * log(q0 / mid);
+    S -= (0.5 * t - delta) / (0.5 * (LN2 + lq));
+  }
+  return S;
+}
+
+// ---------------------------------------------------------------------------------------
 // shared-memory barrier (mbarrier) and bulk asynchronous copy global -> shared
 // ---------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_addr(const void* p) {

@@ -90,6 +90,7 @@ struct VerifyParams {
   int32_t* bonus_ctx;           // [B]
   int B, N, R, V, k;
   float cfg_scale, T, delta;
+  int divergence;               // LANTERN_DIV_TVD or LANTERN_DIV_JSD: what delta bounds
 };
 
 // ---------------------------------------------------------------------------------------
@@ -556,10 +557,54 @@ extern "C" lantern_status lantern_verify_profile_events(void* before_fused, void
   return LANTERN_OK;
 }
 
+static lantern_status verify_impl(const void* target_logits, const void* draft_logits, int dtype, float cfg_scale,
+                                  int has_uncond, float T, const int32_t* draft_tokens, const int32_t* tree_parents,
+                                  const int32_t* neighbor_idx, int k, float delta, int divergence,
+                                  const float* uniforms, int B, int N, int V, int32_t* out_accept_len,
+                                  int32_t* out_next_token, int32_t* out_accept_path, int32_t* out_status,
+                                  float* out_node_qa, float* out_node_px, int32_t* out_node_m, void* workspace,
+                                  size_t workspace_bytes, void* cuda_stream);
+
 extern "C" lantern_status lantern_verify(const void* target_logits, const void* draft_logits, int dtype,
                                          float cfg_scale, int has_uncond, float T, const int32_t* draft_tokens,
                                          const int32_t* tree_parents, const int32_t* neighbor_idx, int k,
                                          float delta, const float* uniforms, int B, int N, int V,
+                                         int32_t* out_accept_len, int32_t* out_next_token,
+                                         int32_t* out_accept_path, int32_t* out_status, float* out_node_qa,
+                                         float* out_node_px, int32_t* out_node_m, void* workspace,
+                                         size_t workspace_bytes, void* cuda_stream) {
+  return lantern_verify_ex(target_logits, draft_logits, dtype, cfg_scale, has_uncond, T, draft_tokens, tree_parents,
+                           neighbor_idx, k, delta, LANTERN_DIV_TVD, 0, uniforms, B, N, V, out_accept_len,
+                           out_next_token, out_accept_path, out_status, out_node_qa, out_node_px, out_node_m,
+                           workspace, workspace_bytes, cuda_stream);
+}
+
+extern "C" size_t lantern_verify_workspace_bytes_ex(int B, int N, int top_k) {
+  if (top_k < 0) return 0;
+  return lantern_verify_workspace_bytes(B, N);
+}
+
+extern "C" lantern_status lantern_verify_ex(const void* target_logits, const void* draft_logits, int dtype,
+                                         float cfg_scale, int has_uncond, float T, const int32_t* draft_tokens,
+                                         const int32_t* tree_parents, const int32_t* neighbor_idx, int k,
+                                         float delta, int divergence, int top_k, const float* uniforms, int B,
+                                         int N, int V, int32_t* out_accept_len, int32_t* out_next_token,
+                                         int32_t* out_accept_path, int32_t* out_status, float* out_node_qa,
+                                         float* out_node_px, int32_t* out_node_m, void* workspace,
+                                         size_t workspace_bytes, void* cuda_stream) {
+  if (divergence != LANTERN_DIV_TVD && divergence != LANTERN_DIV_JSD) return LANTERN_E_PARAM;
+  if (top_k < 0) return LANTERN_E_PARAM;
+  if (top_k > 0 && top_k < V) return LANTERN_E_UNIMPLEMENTED;
+  return verify_impl(target_logits, draft_logits, dtype, cfg_scale, has_uncond, T, draft_tokens, tree_parents,
+                     neighbor_idx, k, delta, divergence, uniforms, B, N, V, out_accept_len, out_next_token,
+                     out_accept_path, out_status, out_node_qa, out_node_px, out_node_m, workspace,
+                     workspace_bytes, cuda_stream);
+}
+
+static lantern_status verify_impl(const void* target_logits, const void* draft_logits, int dtype,
+                                         float cfg_scale, int has_uncond, float T, const int32_t* draft_tokens,
+                                         const int32_t* tree_parents, const int32_t* neighbor_idx, int k,
+                                         float delta, int divergence, const float* uniforms, int B, int N, int V,
                                          int32_t* out_accept_len, int32_t* out_next_token,
                                          int32_t* out_accept_path, int32_t* out_status, float* out_node_qa,
                                          float* out_node_px, int32_t* out_node_m, void* workspace,
@@ -618,6 +663,7 @@ extern "C" lantern_status lantern_verify(const void* target_logits, const void* 
   P.cfg_scale = cfg_scale;
   P.T = T;
   P.delta = delta;
+  P.divergence = divergence;
 
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return LANTERN_E_CUDA;

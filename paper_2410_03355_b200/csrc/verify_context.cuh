@@ -542,7 +542,9 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
         }
 
         // ---- A_{k,delta}(x~): gather + prefix scan with the strict bound ----
-        const double thr = delta / qscale;   // the bound in the units of the unnormalised sums
+        double thr = delta / qscale;   // the bound in the units of the unnormalised sums
+        if (P.divergence == LANTERN_DIV_JSD)   // Section 6.2.2: the same comparison against the mass whose JSD is delta
+          thr = jsd_mass_bound(delta, static_cast<double>(e_xt_bulk) * qscale) / qscale;
         double carry = 0.0, sm = 0.0;
         int m = k - 1;
         bool cut = false;

@@ -347,7 +347,7 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
       auto numer = [&](int n) {   // 2^((z_n - M) log2 e) from the staged bytes
         return greedy_ex2(__fmaf_rn(greedy_one<BF16, UNC>(raw, rowbytes, n, P.cfg_scale), L_hi, -mL));
       };
-      const double thr = static_cast<double>(P.delta) * Z;   // the bound in units of the unnormalised sums
+      const double thr_tvd = static_cast<double>(P.delta) * Z;   // the bound in units of the unnormalised sums
       const ChildInfo* kids = P.children + cur.cbase;
       for (int ci = 0; ci < cur.nchild && accepted < 0; ++ci) {
         int node = cur.node0, xt = cur.tok0;
@@ -357,6 +357,9 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
         }
         const int32_t* nrow = P.nbr + static_cast<size_t>(xt) * k;
         // A_{k,delta}(x~): gather + prefix scan with the strict bound (Algorithm 2, second block)
+        double thr = thr_tvd;
+        if (P.divergence == LANTERN_DIV_JSD && tid < GGT)   // Section 6.2.2: the mass whose JSD is delta
+          thr = jsd_mass_bound(static_cast<double>(P.delta), static_cast<double>(numer(xt)) / Z) * Z;
         double carry = 0.0;
         for (int base = 0;; base += 4 * GGT) {
           double pre4[4], run = 0.0, incl = 0.0;

@@ -39,10 +39,15 @@ def to_device(inp: li.VerifyInputs, device="cuda"):
         uniforms=torch.from_numpy(inp.uniforms).to(device))
 
 
-def run_gpu(inp: li.VerifyInputs, table_dev: torch.Tensor, delta: float, trace=True) -> lt.VerifyOutputs:
+DIV_NAME = {oracle.DIV_TVD: "tvd", oracle.DIV_JSD: "jsd"}
+
+
+def run_gpu(inp: li.VerifyInputs, table_dev: torch.Tensor, delta: float, trace=True, divergence=oracle.DIV_TVD,
+            top_k=0) -> lt.VerifyOutputs:
     d = to_device(inp)
     out = lt.verify(d["target_logits"], d["draft_logits"], inp.cfg_scale, inp.T, d["draft_tokens"],
-                    d["tree_parents"], table_dev, delta, d["uniforms"], trace=trace)
+                    d["tree_parents"], table_dev, delta, d["uniforms"], trace=trace,
+                    divergence=DIV_NAME[divergence], top_k=top_k)
     torch.cuda.synchronize()
     return out
 
@@ -56,7 +61,7 @@ def _slice(inp: li.VerifyInputs, b: int) -> li.VerifyInputs:
         uniforms=inp.uniforms[b:b + 1].copy(), B=1)
 
 
-def _explained_by_window(inp, table, delta, b, ora, want) -> bool:
+def _explained_by_window(inp, table, delta, b, ora, want, divergence=oracle.DIV_TVD, top_k=0) -> bool:
     """Does the oracle give `want` = (len, token, path) once a near-threshold input is nudged?"""
     one = _slice(inp, b)
     eps = 4 * WINDOW
@@ -75,16 +80,18 @@ def _explained_by_window(inp, table, delta, b, ora, want) -> bool:
             u[0, inp.N] = np.float32(min(max(u[0, inp.N] + s, 0.0), 1.0 - 2.0 ** -24))
             trials.append((u, delta))
     for u, d in trials:
-        r = oracle.verify_inputs(dataclasses.replace(one, uniforms=u), table, max(d, 0.0))
+        r = oracle.verify_inputs(dataclasses.replace(one, uniforms=u), table, max(d, 0.0), divergence, top_k)
         if (r.accept_len[0], r.next_token[0]) == want[:2] and np.array_equal(r.accept_path[0], want[2]):
             return True
     return False
 
 
-def compare(inp: li.VerifyInputs, table: np.ndarray, delta: float, gpu: lt.VerifyOutputs, ora=None):
-    """Returns dict(n_seq, near, mismatch_outside, prob_bad, ...); asserts nothing itself."""
+def compare(inp: li.VerifyInputs, table: np.ndarray, delta: float, gpu: lt.VerifyOutputs, ora=None,
+            divergence=oracle.DIV_TVD, top_k=0):
+    """Returns dict(n_seq, near, mismatch_outside, prob_bad, ...); asserts nothing itself.  With the JSD
+    bound the cut's margin is in JSD units (the oracle reports it so); the nudge of delta is the same."""
     if ora is None:
-        ora = oracle.verify_inputs(inp, table, delta)
+        ora = oracle.verify_inputs(inp, table, delta, divergence, top_k)
     g_len = gpu.accept_len.cpu().numpy()
     g_tok = gpu.next_token.cpu().numpy()
     g_path = gpu.accept_path.cpu().numpy()
@@ -96,7 +103,7 @@ def compare(inp: li.VerifyInputs, table: np.ndarray, delta: float, gpu: lt.Verif
                 and np.array_equal(g_path[b], ora.accept_path[b]))
         if same:
             continue
-        if _explained_by_window(inp, table, delta, b, ora, (g_len[b], g_tok[b], g_path[b])):
+        if _explained_by_window(inp, table, delta, b, ora, (g_len[b], g_tok[b], g_path[b]), divergence, top_k):
             near += 1
         else:
             outside += 1

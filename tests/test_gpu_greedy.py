@@ -15,32 +15,32 @@ import torch
 import lantern_inputs as li
 import oracle
 import paper_2410_03355_b200 as lt
-from parity import REL, WINDOW, to_device
+from parity import DIV_NAME, REL, WINDOW, to_device
 
 pytestmark = pytest.mark.gpu
 
 
-def run_gpu(inp, table_dev, delta, trace=True, with_unused=False):
+def run_gpu(inp, table_dev, delta, trace=True, with_unused=False, divergence=oracle.DIV_TVD, top_k=0):
     d = to_device(inp)
     out = lt.verify(d["target_logits"], d["draft_logits"] if with_unused else None, inp.cfg_scale, 0.0,
                     d["draft_tokens"], d["tree_parents"], table_dev, delta,
-                    d["uniforms"] if with_unused else None, trace=trace)
+                    d["uniforms"] if with_unused else None, trace=trace, divergence=DIV_NAME[divergence], top_k=top_k)
     torch.cuda.synchronize()
     return out
 
 
-def replay(inp, table, delta, b, g_len, g_tok, g_path):
+def replay(inp, table, delta, b, g_len, g_tok, g_path, divergence=oracle.DIV_TVD, top_k=0):
     """Is the library's (len, token, path) of sequence b a valid greedy walk up to WINDOW?"""
     N = inp.N
     par = inp.tree_parents[b] if inp.tree_parents is not None else np.arange(N) - 1
     cur, depth = 0, 0
     while True:
         ru = inp.target_logits[1, b, cur] if inp.has_uncond else None
-        q = oracle.row_distribution(inp.target_logits[0, b, cur], ru, inp.dtype, inp.cfg_scale, 1.0)
+        q = oracle.row_distribution(inp.target_logits[0, b, cur], ru, inp.dtype, inp.cfg_scale, 1.0, top_k)
         accepted = -1
         for c in [i for i in range(N) if par[i] == cur - 1]:
             x = inp.draft_tokens[b, c]
-            m, moved, cut_margin = oracle.a_set(q, table[x], delta)
+            m, moved, cut_margin = oracle.a_set(q, table[x], delta, divergence)
             qa = q[x] + moved
             mask = np.ones(inp.V, bool)
             mask[table[x, : m + 1]] = False
@@ -57,13 +57,14 @@ def replay(inp, table, delta, b, g_len, g_tok, g_path):
         cur, depth = accepted + 1, depth + 1
 
 
-def check(inp, host, dev, delta, **kw):
-    return check_outputs(inp, host, delta, run_gpu(inp, dev, delta, **kw))
+def check(inp, host, dev, delta, divergence=oracle.DIV_TVD, top_k=0, **kw):
+    gpu = run_gpu(inp, dev, delta, divergence=divergence, top_k=top_k, **kw)
+    return check_outputs(inp, host, delta, gpu, divergence, top_k)
 
 
-def check_outputs(inp, host, delta, gpu):
+def check_outputs(inp, host, delta, gpu, divergence=oracle.DIV_TVD, top_k=0):
     ora = oracle.verify_greedy(inp.target_logits, inp.dtype, inp.cfg_scale, inp.has_uncond, inp.draft_tokens,
-                               inp.tree_parents, host, delta)
+                               inp.tree_parents, host, delta, divergence, top_k)
     g_len, g_tok = gpu.accept_len.cpu().numpy(), gpu.next_token.cpu().numpy()
     g_path, g_st = gpu.accept_path.cpu().numpy(), gpu.status.cpu().numpy()
     assert np.array_equal(g_st, ora.status)
@@ -72,7 +73,8 @@ def check_outputs(inp, host, delta, gpu):
         if (g_len[b] == ora.accept_len[b] and g_tok[b] == ora.next_token[b]
                 and np.array_equal(g_path[b], ora.accept_path[b])):
             continue
-        assert replay(inp, host, delta, b, g_len[b], g_tok[b], g_path[b]), (b, g_len[b], ora.accept_len[b])
+        assert replay(inp, host, delta, b, g_len[b], g_tok[b], g_path[b], divergence, top_k), \
+            (b, g_len[b], ora.accept_len[b])
         near += 1
     assert near <= max(2, inp.B // 50), near
     qa, m = gpu.node_qa.cpu().numpy(), gpu.node_m.cpu().numpy()

@@ -489,11 +489,11 @@ static WsLayout ws_layout(int B, int N) {
 
 static thread_local cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
 
-template <int CHC, bool BF16, bool UNC, bool TONE>
+template <int CHC, bool BF16, bool UNC, bool TONE, bool JSD>
 static cudaError_t launch_verify(const VerifyParams& P, int grid_ctx, int grid_bonus, size_t smem_bytes,
                                  cudaStream_t st) {
   constexpr int CHB = CHC == 8 ? 2 : 1;   // the bonus kernel runs 1024 threads per row
-  auto kc = lantern_context_kernel<CHC, BF16, UNC, TONE>;
+  auto kc = lantern_context_kernel<CHC, BF16, UNC, TONE, JSD>;
   cudaError_t e = cudaFuncSetAttribute(kc, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
   if (e != cudaSuccess) return e;
   if (g_ev_before && g_ev_after) cudaEventRecord(g_ev_before, st);
@@ -686,12 +686,15 @@ static lantern_status verify_impl(const void* target_logits, const void* draft_l
            : (un ? launch_greedy<false, true>(P, items, sms, grid_bonus, st) : launch_greedy<false, false>(P, items, sms, grid_bonus, st));
     return e == cudaSuccess ? LANTERN_OK : LANTERN_E_CUDA;
   }
-#define LANTERN_DISPATCH2(CHV, TV)                                                                   \
-  (bf ? (un ? launch_verify<CHV, true, true, TV>(P, grid_ctx, grid_bonus, smem_bytes, st)            \
-            : launch_verify<CHV, true, false, TV>(P, grid_ctx, grid_bonus, smem_bytes, st))          \
-      : (un ? launch_verify<CHV, false, true, TV>(P, grid_ctx, grid_bonus, smem_bytes, st)           \
-            : launch_verify<CHV, false, false, TV>(P, grid_ctx, grid_bonus, smem_bytes, st)))
-#define LANTERN_DISPATCH(CHV) (T == 1.0f ? LANTERN_DISPATCH2(CHV, true) : LANTERN_DISPATCH2(CHV, false))
+#define LANTERN_DISPATCH2(CHV, TV, JV)                                                                  \
+  (bf ? (un ? launch_verify<CHV, true, true, TV, JV>(P, grid_ctx, grid_bonus, smem_bytes, st)            \
+            : launch_verify<CHV, true, false, TV, JV>(P, grid_ctx, grid_bonus, smem_bytes, st))          \
+      : (un ? launch_verify<CHV, false, true, TV, JV>(P, grid_ctx, grid_bonus, smem_bytes, st)           \
+            : launch_verify<CHV, false, false, TV, JV>(P, grid_ctx, grid_bonus, smem_bytes, st)))
+  // the JSD variant is built for the general-temperature code only (T = 1 runs through it unchanged)
+#define LANTERN_DISPATCH(CHV)                                                    \
+  (divergence == LANTERN_DIV_JSD ? LANTERN_DISPATCH2(CHV, false, true)           \
+                                 : (T == 1.0f ? LANTERN_DISPATCH2(CHV, true, false) : LANTERN_DISPATCH2(CHV, false, false)))
   e = CH == 8 ? LANTERN_DISPATCH(8) : (CH == 4 ? LANTERN_DISPATCH(4) : (CH == 2 ? LANTERN_DISPATCH(2) : LANTERN_DISPATCH(1)));
 #undef LANTERN_DISPATCH2
 #undef LANTERN_DISPATCH

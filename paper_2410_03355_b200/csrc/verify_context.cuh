@@ -25,7 +25,7 @@
 // inverse-CDF draw or the write-back for the next sibling.
 #pragma once
 
-#define LANTERN_CONTEXT_KERNEL_REVISION 10   // bump on every change to this file
+#define LANTERN_CONTEXT_KERNEL_REVISION 11   // bump on every change to this file
 
 namespace lantern {
 
@@ -172,7 +172,8 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 
 // CH = 8-token chunks per thread (1, 2, 4 or 8); a thread streams them in NP passes of CP chunks.
 // TONE = the temperature is exactly 1 (the paper's sampling setting): no division is compiled in.
-template <int CH, bool BF16, bool UNC, bool TONE>
+// JSD selects the Section 6.2.2 bound at compile time, so that the default path carries none of its code.
+template <int CH, bool BF16, bool UNC, bool TONE, bool JSD>
 __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyParams P) {
   constexpr int NP = CH > 4 ? 2 : 1;          // passes
   constexpr int CP = CH / NP;                 // chunks per pass
@@ -543,8 +544,10 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
 
         // ---- A_{k,delta}(x~): gather + prefix scan with the strict bound ----
         double thr = delta / qscale;   // the bound in the units of the unnormalised sums
-        if (P.divergence == LANTERN_DIV_JSD)   // Section 6.2.2: the same comparison against the mass whose JSD is delta
-          thr = jsd_mass_bound(delta, static_cast<double>(e_xt_bulk) * qscale) / qscale;
+        // Section 6.2.2: the mass whose JSD is delta; one thread, published by [scan 1] through the last
+        // slot of wt[], which nothing else touches between the start of a child and its [scan 2]
+        if (JSD && gt == GT - 32)
+          S.wt[8 * GW - 1] = jsd_mass_bound(delta, static_cast<double>(e_xt_bulk) * qscale) / qscale;
         double carry = 0.0, sm = 0.0;
         int m = k - 1;
         bool cut = false;
@@ -565,6 +568,7 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
           const double incl = warp_incl_scan(run, lane);
           if (lane == 31) S.wt[gw] = incl;
           gbar(grp);   // [scan 1]
+          if (JSD && base == 0) thr = S.wt[8 * GW - 1];
           double pre = 0.0, tot = 0.0;
 #pragma unroll
           for (int w = 0; w < GW; ++w) {

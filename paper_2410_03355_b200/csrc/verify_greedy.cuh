@@ -132,7 +132,7 @@ constexpr int GCW = GCT / 32;
 constexpr int GGT = 256;            // threads that gather: four neighbour slots each per round
 constexpr int GGW = GGT / 32;
 constexpr int GRING_MAX = 4;
-static_assert(GCW <= 32 && GGT <= GCT, "one warp combines the per-warp partials; gatherers are a subset");
+static_assert(GCW <= 32 && GGT < GCT, "one warp combines the per-warp partials; a thread beyond the gatherers solves the JSD bound");
 
 struct GreedyCtxShared {
   double ws[GCW];                   // per-warp sums of numerators relative to the warp's maximum
@@ -147,6 +147,7 @@ struct GreedyCtxShared {
   int flags[2];                     // bit 0: NaN met, bit 1: a copy did not arrive (by iteration parity)
   int status;
   int done, accept;
+  double thr;                       // JSD bound only: the current child's mass bound
   unsigned long long bar_full[GRING_MAX];
 };
 
@@ -358,8 +359,9 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
         const int32_t* nrow = P.nbr + static_cast<size_t>(xt) * k;
         // A_{k,delta}(x~): gather + prefix scan with the strict bound (Algorithm 2, second block)
         double thr = thr_tvd;
-        if (P.divergence == LANTERN_DIV_JSD && tid < GGT)   // Section 6.2.2: the mass whose JSD is delta
-          thr = jsd_mass_bound(static_cast<double>(P.delta), static_cast<double>(numer(xt)) / Z) * Z;
+        const bool jsd = P.divergence == LANTERN_DIV_JSD;
+        if (jsd && tid == GGT)   // Section 6.2.2: the mass whose JSD is delta, from a thread that does not gather
+          S.thr = jsd_mass_bound(static_cast<double>(P.delta), static_cast<double>(numer(xt)) / Z) * Z;
         double carry = 0.0;
         for (int base = 0;; base += 4 * GGT) {
           double pre4[4], run = 0.0, incl = 0.0;
@@ -390,6 +392,7 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
             if (lane == 31) S.wt[warp] = incl;
           }
           __syncthreads();
+          if (jsd && base == 0) thr = S.thr;
           double tot = 0.0;
           if (tid < GGT) {
             double pre = 0.0;

@@ -91,6 +91,9 @@ struct VerifyParams {
   int B, N, R, V, k;
   float cfg_scale, T, delta;
   int divergence;               // LANTERN_DIV_TVD or LANTERN_DIV_JSD: what delta bounds
+  int top_k;                    // logit filter; 0 = off (then thr_q, thr_p are null)
+  float* thr_q;                 // [B, R] top_k-th largest processed target logit of a context row
+  float* thr_p;                 // [B, R] the same for the drafter row
 };
 
 // ---------------------------------------------------------------------------------------
@@ -332,6 +335,7 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
 #include "verify_context.cuh"
 // greedy decoding (temperature 0)
 #include "verify_greedy.cuh"
+#include "verify_topk.cuh"
 
 namespace lantern {
 
@@ -375,7 +379,7 @@ __global__ void __launch_bounds__(128) lantern_walk_kernel(VerifyParams P) {
 // kernel 4: bonus token ~ q at the context where the walk ran out of drafts
 // (Algorithm 1, line after the verification loop)
 // ---------------------------------------------------------------------------------------
-template <int CH, bool BF16, bool UNC>
+template <int CH, bool BF16, bool UNC, bool TOPK>
 __global__ void __launch_bounds__(NT, 1) lantern_bonus_kernel(VerifyParams P) {
   __shared__ BlockScratch S;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -390,6 +394,8 @@ __global__ void __launch_bounds__(NT, 1) lantern_bonus_kernel(VerifyParams P) {
     const unsigned char* ru = rc + branch;
     float a[CH * 8];
     const float ninf = __int_as_float(0xff800000);
+    float tq = ninf;   // top-k filter, if any
+    if (TOPK) tq = __ldg(P.thr_q + static_cast<size_t>(b) * R + ctx);
 #pragma unroll
     for (int c = 0; c < CH; ++c) {
       const int g = c * NT + tid;
@@ -428,7 +434,7 @@ __global__ void __launch_bounds__(NT, 1) lantern_bonus_kernel(VerifyParams P) {
           float l = lc[e];
           if (UNC) l = __fmaf_rn(P.cfg_scale, __fsub_rn(lc[e], lu[e]), lu[e]);
           if (P.T != 1.0f) l = __fdiv_rn(l, P.T);
-          a[c * 8 + e] = l;
+          a[c * 8 + e] = (TOPK && l < tq) ? ninf : l;
         }
       } else {
 #pragma unroll
@@ -469,10 +475,10 @@ __global__ void __launch_bounds__(NT, 1) lantern_bonus_kernel(VerifyParams P) {
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WsLayout {
-  size_t counters, work, children, records, seqst, bseq, bctx, total;
+  size_t counters, work, children, records, seqst, bseq, bctx, thrq, thrp, total;
 };
 
-static WsLayout ws_layout(int B, int N) {
+static WsLayout ws_layout(int B, int N, bool topk = false) {
   const size_t R = static_cast<size_t>(N) + 1, b = static_cast<size_t>(B);
   WsLayout L;
   size_t o = 0;
@@ -483,19 +489,35 @@ static WsLayout ws_layout(int B, int N) {
   L.seqst = o;    o += align_up(b * 4, 256);
   L.bseq = o;     o += align_up(b * 4, 256);
   L.bctx = o;     o += align_up(b * 4, 256);
+  L.thrq = o;     o += topk ? align_up(b * R * 4, 256) : 0;
+  L.thrp = o;     o += topk ? align_up(b * R * 4, 256) : 0;
   L.total = o;
   return L;
 }
 
 static thread_local cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
 
-template <int CHC, bool BF16, bool UNC, bool TONE, bool JSD>
-static cudaError_t launch_verify(const VerifyParams& P, int grid_ctx, int grid_bonus, size_t smem_bytes,
-                                 cudaStream_t st) {
+// thresholds of the top-k filter: mode 0 = rows of the contexts with children (after the plan),
+// mode 1 = rows of the bonus draws (after the walk)
+template <bool BF16, bool UNC>
+static cudaError_t launch_topk(const VerifyParams& P, int mode, long long jobs, int sms, cudaStream_t st) {
+  const long long slots = 2ll * sms;
+  const int grid = static_cast<int>(jobs < slots ? (jobs > 0 ? jobs : 1) : slots);
+  lantern_topk_kernel<BF16, UNC><<<grid, TKT, 0, st>>>(P, mode);
+  return cudaGetLastError();
+}
+
+template <int CHC, bool BF16, bool UNC, bool TONE, bool JSD, bool TOPK>
+static cudaError_t launch_verify(const VerifyParams& P, long long items, int sms, int grid_ctx, int grid_bonus,
+                                 size_t smem_bytes, cudaStream_t st) {
   constexpr int CHB = CHC == 8 ? 2 : 1;   // the bonus kernel runs 1024 threads per row
-  auto kc = lantern_context_kernel<CHC, BF16, UNC, TONE, JSD>;
+  auto kc = lantern_context_kernel<CHC, BF16, UNC, TONE, JSD, TOPK>;
   cudaError_t e = cudaFuncSetAttribute(kc, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
   if (e != cudaSuccess) return e;
+  if (TOPK) {
+    e = launch_topk<BF16, UNC>(P, 0, items, sms, st);
+    if (e != cudaSuccess) return e;
+  }
   if (g_ev_before && g_ev_after) cudaEventRecord(g_ev_before, st);
   kc<<<grid_ctx, CTX_THREADS, smem_bytes, st>>>(P);
   e = cudaGetLastError();
@@ -504,13 +526,17 @@ static cudaError_t launch_verify(const VerifyParams& P, int grid_ctx, int grid_b
   lantern_walk_kernel<<<(P.B + 127) / 128, 128, 0, st>>>(P);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  lantern_bonus_kernel<CHB, BF16, UNC><<<grid_bonus, NT, 0, st>>>(P);
+  if (TOPK) {
+    e = launch_topk<BF16, UNC>(P, 1, P.B, sms, st);
+    if (e != cudaSuccess) return e;
+  }
+  lantern_bonus_kernel<CHB, BF16, UNC, TOPK><<<grid_bonus, NT, 0, st>>>(P);
   return cudaGetLastError();
 }
 
-template <bool BF16, bool UNC>
+template <bool BF16, bool UNC, bool TOPK>
 static cudaError_t launch_greedy(const VerifyParams& P, long long items, int sms, int grid_bonus, cudaStream_t st) {
-  auto kc = lantern_greedy_context_kernel<BF16, UNC>;
+  auto kc = lantern_greedy_context_kernel<BF16, UNC, TOPK>;
   // a ring of staging areas per CTA, each holding the raw target rows of one context; sized so that
   // three CTAs share an SM where the rows allow it
   const size_t area = static_cast<size_t>(P.V) * (UNC ? 2 : 1) * (BF16 ? 2 : 4);
@@ -525,6 +551,10 @@ static cudaError_t launch_greedy(const VerifyParams& P, long long items, int sms
   if (per_sm < 1) return cudaErrorInvalidConfiguration;
   const long long slots = static_cast<long long>(sms) * per_sm;
   const int grid_ctx = static_cast<int>(items < slots ? items : slots);
+  if (TOPK) {
+    e = launch_topk<BF16, UNC>(P, 0, items, sms, st);
+    if (e != cudaSuccess) return e;
+  }
   if (g_ev_before && g_ev_after) cudaEventRecord(g_ev_before, st);
   kc<<<grid_ctx, GCT, smem, st>>>(P, ring);
   e = cudaGetLastError();
@@ -533,7 +563,7 @@ static cudaError_t launch_greedy(const VerifyParams& P, long long items, int sms
   lantern_walk_kernel<<<(P.B + 127) / 128, 128, 0, st>>>(P);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  lantern_greedy_bonus_kernel<BF16, UNC><<<grid_bonus, GRT, 0, st>>>(P);
+  lantern_greedy_bonus_kernel<BF16, UNC><<<grid_bonus, GRT, 0, st>>>(P);   // the arg max is never filtered out
   return cudaGetLastError();
 }
 
@@ -559,7 +589,7 @@ extern "C" lantern_status lantern_verify_profile_events(void* before_fused, void
 
 static lantern_status verify_impl(const void* target_logits, const void* draft_logits, int dtype, float cfg_scale,
                                   int has_uncond, float T, const int32_t* draft_tokens, const int32_t* tree_parents,
-                                  const int32_t* neighbor_idx, int k, float delta, int divergence,
+                                  const int32_t* neighbor_idx, int k, float delta, int divergence, int top_k,
                                   const float* uniforms, int B, int N, int V, int32_t* out_accept_len,
                                   int32_t* out_next_token, int32_t* out_accept_path, int32_t* out_status,
                                   float* out_node_qa, float* out_node_px, int32_t* out_node_m, void* workspace,
@@ -580,8 +610,8 @@ extern "C" lantern_status lantern_verify(const void* target_logits, const void* 
 }
 
 extern "C" size_t lantern_verify_workspace_bytes_ex(int B, int N, int top_k) {
-  if (top_k < 0) return 0;
-  return lantern_verify_workspace_bytes(B, N);
+  if (B < 0 || N < 0 || N > MAX_N || top_k < 0) return 0;
+  return ws_layout(B > 0 ? B : 1, N, top_k > 0).total;
 }
 
 extern "C" lantern_status lantern_verify_ex(const void* target_logits, const void* draft_logits, int dtype,
@@ -594,9 +624,8 @@ extern "C" lantern_status lantern_verify_ex(const void* target_logits, const voi
                                          size_t workspace_bytes, void* cuda_stream) {
   if (divergence != LANTERN_DIV_TVD && divergence != LANTERN_DIV_JSD) return LANTERN_E_PARAM;
   if (top_k < 0) return LANTERN_E_PARAM;
-  if (top_k > 0 && top_k < V) return LANTERN_E_UNIMPLEMENTED;
   return verify_impl(target_logits, draft_logits, dtype, cfg_scale, has_uncond, T, draft_tokens, tree_parents,
-                     neighbor_idx, k, delta, divergence, uniforms, B, N, V, out_accept_len, out_next_token,
+                     neighbor_idx, k, delta, divergence, top_k, uniforms, B, N, V, out_accept_len, out_next_token,
                      out_accept_path, out_status, out_node_qa, out_node_px, out_node_m, workspace,
                      workspace_bytes, cuda_stream);
 }
@@ -604,7 +633,7 @@ extern "C" lantern_status lantern_verify_ex(const void* target_logits, const voi
 static lantern_status verify_impl(const void* target_logits, const void* draft_logits, int dtype,
                                          float cfg_scale, int has_uncond, float T, const int32_t* draft_tokens,
                                          const int32_t* tree_parents, const int32_t* neighbor_idx, int k,
-                                         float delta, int divergence, const float* uniforms, int B, int N, int V,
+                                         float delta, int divergence, int top_k, const float* uniforms, int B, int N, int V,
                                          int32_t* out_accept_len, int32_t* out_next_token,
                                          int32_t* out_accept_path, int32_t* out_status, float* out_node_qa,
                                          float* out_node_px, int32_t* out_node_m, void* workspace,
@@ -628,7 +657,8 @@ static lantern_status verify_impl(const void* target_logits, const void* draft_l
   if (N > 0 && (!draft_tokens || (!greedy && !draft_logits))) return LANTERN_E_NULL;
   if ((reinterpret_cast<uintptr_t>(target_logits) & 15) || (reinterpret_cast<uintptr_t>(draft_logits) & 15))
     return LANTERN_E_ALIGN;
-  const WsLayout L = ws_layout(B, N);
+  const bool topk = top_k > 0 && top_k < V;   // top_k >= V keeps every logit
+  const WsLayout L = ws_layout(B, N, top_k > 0);
   if (!workspace || workspace_bytes < L.total || (reinterpret_cast<uintptr_t>(workspace) & 255))
     return LANTERN_E_WORKSPACE;
 
@@ -664,6 +694,9 @@ static lantern_status verify_impl(const void* target_logits, const void* draft_l
   P.T = T;
   P.delta = delta;
   P.divergence = divergence;
+  P.top_k = topk ? top_k : 0;
+  P.thr_q = topk ? reinterpret_cast<float*>(ws + L.thrq) : nullptr;
+  P.thr_p = topk ? reinterpret_cast<float*>(ws + L.thrp) : nullptr;
 
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return LANTERN_E_CUDA;
@@ -682,19 +715,25 @@ static lantern_status verify_impl(const void* target_logits, const void* draft_l
   cudaError_t e;
   const bool bf = dtype == LANTERN_BF16, un = has_uncond != 0;
   if (greedy) {
-    e = bf ? (un ? launch_greedy<true, true>(P, items, sms, grid_bonus, st) : launch_greedy<true, false>(P, items, sms, grid_bonus, st))
-           : (un ? launch_greedy<false, true>(P, items, sms, grid_bonus, st) : launch_greedy<false, false>(P, items, sms, grid_bonus, st));
+#define LANTERN_GREEDY(KV)                                                                                   \
+  (bf ? (un ? launch_greedy<true, true, KV>(P, items, sms, grid_bonus, st) : launch_greedy<true, false, KV>(P, items, sms, grid_bonus, st)) \
+      : (un ? launch_greedy<false, true, KV>(P, items, sms, grid_bonus, st) : launch_greedy<false, false, KV>(P, items, sms, grid_bonus, st)))
+    e = topk ? LANTERN_GREEDY(true) : LANTERN_GREEDY(false);
+#undef LANTERN_GREEDY
     return e == cudaSuccess ? LANTERN_OK : LANTERN_E_CUDA;
   }
-#define LANTERN_DISPATCH2(CHV, TV, JV)                                                                  \
-  (bf ? (un ? launch_verify<CHV, true, true, TV, JV>(P, grid_ctx, grid_bonus, smem_bytes, st)            \
-            : launch_verify<CHV, true, false, TV, JV>(P, grid_ctx, grid_bonus, smem_bytes, st))          \
-      : (un ? launch_verify<CHV, false, true, TV, JV>(P, grid_ctx, grid_bonus, smem_bytes, st)           \
-            : launch_verify<CHV, false, false, TV, JV>(P, grid_ctx, grid_bonus, smem_bytes, st)))
-  // the JSD variant is built for the general-temperature code only (T = 1 runs through it unchanged)
-#define LANTERN_DISPATCH(CHV)                                                    \
-  (divergence == LANTERN_DIV_JSD ? LANTERN_DISPATCH2(CHV, false, true)           \
-                                 : (T == 1.0f ? LANTERN_DISPATCH2(CHV, true, false) : LANTERN_DISPATCH2(CHV, false, false)))
+#define LANTERN_DISPATCH2(CHV, TV, JV, KV)                                                                        \
+  (bf ? (un ? launch_verify<CHV, true, true, TV, JV, KV>(P, items, sms, grid_ctx, grid_bonus, smem_bytes, st)     \
+            : launch_verify<CHV, true, false, TV, JV, KV>(P, items, sms, grid_ctx, grid_bonus, smem_bytes, st))   \
+      : (un ? launch_verify<CHV, false, true, TV, JV, KV>(P, items, sms, grid_ctx, grid_bonus, smem_bytes, st)    \
+            : launch_verify<CHV, false, false, TV, JV, KV>(P, items, sms, grid_ctx, grid_bonus, smem_bytes, st)))
+  // the JSD and top-k variants are built for the general-temperature code only (T = 1 runs through it unchanged)
+#define LANTERN_DISPATCH(CHV)                                                                                     \
+  (topk ? (divergence == LANTERN_DIV_JSD ? LANTERN_DISPATCH2(CHV, false, true, true)                              \
+                                         : LANTERN_DISPATCH2(CHV, false, false, true))                            \
+        : (divergence == LANTERN_DIV_JSD                                                                          \
+               ? LANTERN_DISPATCH2(CHV, false, true, false)                                                       \
+               : (T == 1.0f ? LANTERN_DISPATCH2(CHV, true, false, false) : LANTERN_DISPATCH2(CHV, false, false, false))))
   e = CH == 8 ? LANTERN_DISPATCH(8) : (CH == 4 ? LANTERN_DISPATCH(4) : (CH == 2 ? LANTERN_DISPATCH(2) : LANTERN_DISPATCH(1)));
 #undef LANTERN_DISPATCH2
 #undef LANTERN_DISPATCH

@@ -25,7 +25,7 @@
 // inverse-CDF draw or the write-back for the next sibling.
 #pragma once
 
-#define LANTERN_CONTEXT_KERNEL_REVISION 11   // bump on every change to this file
+#define LANTERN_CONTEXT_KERNEL_REVISION 12   // bump on every change to this file
 
 namespace lantern {
 
@@ -81,6 +81,7 @@ __device__ __forceinline__ float ex2_approx(float x) {
 __device__ __forceinline__ double exp2_single(float z, float shift) {
   const double x = static_cast<double>(z) * 1.4426950408889634074 - static_cast<double>(shift);
   const float xh = static_cast<float>(x);
+  if (xh < -1000.0f) return 0.0;   // far below the flush-to-zero range; also keeps -inf from turning into inf - inf
   const float xl = static_cast<float>(x - static_cast<double>(xh));
   const float y = ex2_approx(xh);
   return static_cast<double>(__fmaf_rn(y, xl * 0.693147182464599609375f, y));
@@ -173,7 +174,9 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 // CH = 8-token chunks per thread (1, 2, 4 or 8); a thread streams them in NP passes of CP chunks.
 // TONE = the temperature is exactly 1 (the paper's sampling setting): no division is compiled in.
 // JSD selects the Section 6.2.2 bound at compile time, so that the default path carries none of its code.
-template <int CH, bool BF16, bool UNC, bool TONE, bool JSD>
+// TOPK applies the per-row thresholds of the top-k logit filter (Appendix B.2; written by
+// lantern_topk_kernel): processed logits below a row's threshold count as -inf.
+template <int CH, bool BF16, bool UNC, bool TONE, bool JSD, bool TOPK>
 __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyParams P) {
   constexpr int NP = CH > 4 ? 2 : 1;          // passes
   constexpr int CP = CH / NP;                 // chunks per pass
@@ -231,8 +234,18 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
         }
         return it;
       };
+      // top-k thresholds of a context travel with its descriptor: (target, drafter)
+      auto load_thr = [&](const WorkItem& it, float& tq, float& tp) {
+        if (TOPK && it.item >= 0) {
+          tq = __ldg(P.thr_q + it.item);
+          tp = __ldg(P.thr_p + it.item);
+        }
+      };
+      float tq_cur = 0.0f, tp_cur = 0.0f, tq_next = 0.0f, tp_next = 0.0f;
       WorkItem it_cur = load_item(me);
       WorkItem it_next = load_item(me + G);
+      load_thr(it_cur, tq_cur, tp_cur);
+      load_thr(it_next, tq_next, tp_next);
       int w_next2 = me + 2 * G;
       for (int i = 0;; ++i) {
         // the staging area is free once every warp of the group has finished the previous context
@@ -241,6 +254,10 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
           it_cur.pad = LANTERN_ST_INTERNAL;   // the group never released its area: stop handing out work
         }
         S.work = it_cur;                      // published by the mbarrier operation below
+        if (TOPK) {   // the group is between contexts: its scratch is free; these two slots stay untouched until read
+          S.wt[8 * GW - 2] = static_cast<double>(tq_cur);
+          S.wt[8 * GW - 3] = static_cast<double>(tp_cur);
+        }
         if (it_cur.item < 0) {
           mbar_arrive(&bar_full[grp]);        // wake the group; it sees the terminator
           break;
@@ -248,7 +265,9 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
         fence_proxy_async();
         ctx_issue_rows<BF16, UNC>(P, it_cur.item, smem + grp * stage_bytes, rowbytes, &bar_full[grp]);
         it_cur = it_next;
+        tq_cur = tq_next, tp_cur = tp_next;
         it_next = load_item(w_next2);
+        load_thr(it_next, tq_next, tp_next);
         w_next2 = 3 * G + atomicAdd(&P.counters->work_next, 1);
       }
     }
@@ -299,6 +318,11 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
     const WorkItem cur = S.work;
     const int item = cur.item;
     if (item < 0) break;
+    float tq = 0.0f, tp = 0.0f;   // top-k thresholds of this context's target and drafter rows
+    if (TOPK) {
+      tq = static_cast<float>(S.wt[8 * GW - 2]);
+      tp = static_cast<float>(S.wt[8 * GW - 3]);
+    }
     const int b = item / R;
     const ChildInfo* kids = P.children + cur.cbase;
     const int nchild = cur.nchild;
@@ -369,6 +393,11 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
             uint64_t l2 = c2[i];
             if (UNC) l2 = fma2(s2, sub2(c2[i], u2[i]), u2[i]);   // l_u + s (l_c - l_u)
             if (!T_is_one) l2 = divide_T(l2);
+            if (TOPK) {   // below the row's top-k threshold: -inf (a NaN stays, to be reported)
+              float lo, hi;
+              unpack2(l2, lo, hi);
+              l2 = pack2(lo < tq ? ninf : lo, hi < tq ? ninf : hi);
+            }
             a2[c * 4 + i] = l2;
             float lo, hi;
             unpack2(l2, lo, hi);
@@ -416,14 +445,40 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
         if (g * 8 < V) {
           uint64_t d2[4];
           pairs_of(rd, g, d2);
+          bool cut = false;
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             uint64_t l2 = d2[i];
             if (!T_is_one) l2 = divide_T(l2);
-            a2[c * 4 + i] = l2;
             float lo, hi;
             unpack2(l2, lo, hi);
+            if (TOPK) {   // the filtered tokens are also struck from the raw row, which later steps re-read
+              const bool clo = lo < tp, chi = hi < tp;
+              float rlo, rhi;
+              unpack2(d2[i], rlo, rhi);
+              d2[i] = pack2(clo ? ninf : rlo, chi ? ninf : rhi);
+              lo = clo ? ninf : lo, hi = chi ? ninf : hi;
+              l2 = pack2(lo, hi);
+              cut |= clo | chi;
+            }
+            a2[c * 4 + i] = l2;
             mp = max3(mp, lo, hi);
+          }
+          if (TOPK && cut) {
+            float v[8];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) unpack2(d2[i], v[2 * i], v[2 * i + 1]);
+            if (BF16) {
+              uint4 w;
+              w.x = (__float_as_uint(v[0]) >> 16) | (__float_as_uint(v[1]) & 0xffff0000u);
+              w.y = (__float_as_uint(v[2]) >> 16) | (__float_as_uint(v[3]) & 0xffff0000u);
+              w.z = (__float_as_uint(v[4]) >> 16) | (__float_as_uint(v[5]) & 0xffff0000u);
+              w.w = (__float_as_uint(v[6]) >> 16) | (__float_as_uint(v[7]) & 0xffff0000u);
+              *reinterpret_cast<uint4*>(rd + g * 16) = w;
+            } else {
+              *reinterpret_cast<float4*>(rd + g * 32) = make_float4(v[0], v[1], v[2], v[3]);
+              *reinterpret_cast<float4*>(rd + g * 32 + 16) = make_float4(v[4], v[5], v[6], v[7]);
+            }
           }
         } else {
 #pragma unroll
@@ -518,6 +573,10 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
         if (!T_is_one) {
           zq = __fdiv_rn(zq, P.T);
           zp = __fdiv_rn(zp, P.T);
+        }
+        if (TOPK) {   // these come from global memory, unfiltered
+          zq = zq < tq ? ninf : zq;
+          zp = zp < tp ? ninf : zp;
         }
         S.acc_e = exp2_single(zq, mlq_g);
         S.acc_p = exp2_single(zp, mlp_g);
@@ -738,6 +797,10 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
               if (!T_is_one) {
                 zq = __fdiv_rn(zq, P.T);
                 zp = __fdiv_rn(zp, P.T);
+              }
+              if (TOPK) {   // these come from global memory, unfiltered
+                zq = zq < tq ? ninf : zq;
+                zp = zp < tp ? ninf : zp;
               }
               double e = exp2_single(zq, mlq_g);
               const double pe = exp2_single(zp, mlp_g);

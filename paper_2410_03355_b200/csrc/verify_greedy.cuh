@@ -217,7 +217,9 @@ __device__ __forceinline__ void greedy_issue_rows(const VerifyParams& P, int ite
   if (UNC) bulk_load(raw + rowbytes, base + branch + row, rowbytes, reinterpret_cast<uint64_t*>(bar));
 }
 
-template <bool BF16, bool UNC>
+// TOPK: processed logits below the row's top-k threshold (Appendix B.2; written by lantern_topk_kernel)
+// count as -inf: they leave Z and carry no mass in a neighbourhood; maximum and arg max are not affected.
+template <bool BF16, bool UNC, bool TOPK>
 __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyParams P, int ring) {
   extern __shared__ __align__(128) unsigned char gsm[];
   __shared__ GreedyCtxShared S;
@@ -250,6 +252,8 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
   if (static_cast<int>(blockIdx.x) >= total) return;   // nothing was requested for this CTA
 
   WorkItem cur = P.work[slot(blockIdx.x)];
+  float tq = 0.0f;
+  if (TOPK) tq = __ldg(P.thr_q + cur.item);
   uint32_t it = 0, phase = 0;
   int buf = 0;
   for (long long w = blockIdx.x; w < total; w += G, ++it) {
@@ -278,7 +282,13 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
     int mi = 0x7fffffff;
 #pragma unroll 4
     for (int qd = tid; qd < quads; qd += GCT) {
-      const float4 z = greedy_quad<BF16, UNC>(raw, rowbytes, qd, P.cfg_scale);
+      float4 z = greedy_quad<BF16, UNC>(raw, rowbytes, qd, P.cfg_scale);
+      if (TOPK) {   // a NaN stays, to be reported
+        z.x = z.x < tq ? NEG_INF : z.x;
+        z.y = z.y < tq ? NEG_INF : z.y;
+        z.z = z.z < tq ? NEG_INF : z.z;
+        z.w = z.w < tq ? NEG_INF : z.w;
+      }
       const float old = m;
       if (z.x > m) m = z.x, mi = 4 * qd;          // ascending index within a thread: strict > keeps
       if (z.y > m) m = z.y, mi = 4 * qd + 1;      // the smallest index
@@ -303,6 +313,8 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
         S.ws[warp] = static_cast<double>(f);
       }
     }
+    float tq_next = 0.0f;   // the next context's threshold: its descriptor has arrived during the sweep
+    if (TOPK) tq_next = __ldg(P.thr_q + nxt.item);
     if (bad || !ok) atomicOr(&S.flags[it & 1], (bad ? 1 : 0) | (ok ? 0 : 2));
     __syncthreads();   // A
     if (warp == 0) {   // lane v combines warp v
@@ -346,7 +358,9 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
     } else {
       const float mL = M * L_hi;
       auto numer = [&](int n) {   // 2^((z_n - M) log2 e) from the staged bytes
-        return greedy_ex2(__fmaf_rn(greedy_one<BF16, UNC>(raw, rowbytes, n, P.cfg_scale), L_hi, -mL));
+        float zn = greedy_one<BF16, UNC>(raw, rowbytes, n, P.cfg_scale);
+        if (TOPK) zn = zn < tq ? NEG_INF : zn;
+        return greedy_ex2(__fmaf_rn(zn, L_hi, -mL));
       };
       const double thr_tvd = static_cast<double>(P.delta) * Z;   // the bound in units of the unnormalised sums
       const ChildInfo* kids = P.children + cur.cbase;
@@ -462,6 +476,7 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
       S.status = 0;
     }
     cur = nxt;
+    tq = tq_next;
     if (++buf == ring) {
       buf = 0;
       phase ^= 1;

@@ -1,0 +1,243 @@
+// Top-k logit filter (Appendix B.2: top-k 1000 / 2000 with top-p 1): per context row, the
+// value of the top_k-th largest processed logit; included by verify.cu.
+//
+// The verification kernels then treat every processed logit below that value as -inf (logits
+// equal to it are all kept).  One CTA of TKT threads per row job, the row's processed logits held
+// in registers as order-preserving 32-bit keys (64 per thread at V = 16384):
+//   1. block statistics: number of keys above -inf, smallest such key, largest key;
+//   2. bisection on the key interval [lo, hi) with the invariant
+//        count(key >= lo) >= K > count(key >= hi),
+//      every pass one compare-and-count over the registers and one block reduction; the split
+//      point is the key of the arithmetic mean of the two bounds' values while that lies strictly
+//      inside (logit values are spread evenly in value, not in bit pattern), else the integer
+//      midpoint, so the search ends after at most 64 passes whatever the data;
+//   3. as soon as at most TK_LIST keys remain in [lo, hi) they are gathered into shared memory
+//      and the wanted one is found by counting ranks.
+// -0 is keyed as +0 (they compare equal as logits); NaN is keyed below -inf (such a row is
+// reported by the verification kernels anyway).
+#pragma once
+
+namespace lantern {
+
+constexpr int TKT = 256;
+constexpr int TKW = TKT / 32;
+constexpr int TK_CH = 8;            // 8-token chunks per thread: 8 * 8 * 256 = 16384 tokens at most
+constexpr int TK_LIST = 256;
+constexpr uint32_t TK_KEY_NINF = 0x007fffffu;
+
+struct TopkShared {
+  int cnt[2][TKW];
+  unsigned kmin[TKW], kmax[TKW];
+  unsigned list[TK_LIST];
+  int list_n;
+  unsigned result;
+};
+
+__device__ __forceinline__ uint32_t topk_key(float z) {
+  if (z != z) return 0u;
+  if (z == 0.0f) z = 0.0f;          // -0 -> +0
+  const uint32_t u = __float_as_uint(z);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float topk_value(uint32_t key) {
+  return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
+}
+
+// number of this thread's keys >= t, summed over the block (every thread gets the sum)
+__device__ __forceinline__ int topk_count(const uint32_t (&key)[TK_CH * 8], uint32_t t, TopkShared& S, int& flip) {
+  int c = 0;
+#pragma unroll
+  for (int i = 0; i < TK_CH * 8; ++i) c += key[i] >= t;
+  c = __reduce_add_sync(kFull, c);
+  if ((threadIdx.x & 31) == 0) S.cnt[flip][threadIdx.x >> 5] = c;
+  __syncthreads();
+  int tot = 0;
+#pragma unroll
+  for (int w = 0; w < TKW; ++w) tot += S.cnt[flip][w];
+  flip ^= 1;   // the next call writes the other set: a warp still reading this one is at most one barrier behind
+  return tot;
+}
+
+// processed logits of one row as keys: base row (+ unconditional row at `branch` elements further on)
+template <bool BF16, bool UNC>
+__device__ __forceinline__ void topk_load_keys(const void* logits, size_t row_elem, size_t branch_elem, int V, float s,
+                                               float T, uint32_t (&key)[TK_CH * 8]) {
+  const int tid = threadIdx.x;
+#pragma unroll
+  for (int c = 0; c < TK_CH; ++c) {
+    const int g = c * TKT + tid;
+    float lc[8], lu[8];
+    if (g * 8 < V) {
+      if (BF16) {
+        const unsigned short* base = static_cast<const unsigned short*>(logits);
+        const uint4 x = __ldg(reinterpret_cast<const uint4*>(base + row_elem) + g);
+        const uint32_t xw[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          lc[2 * i] = __uint_as_float(xw[i] << 16);
+          lc[2 * i + 1] = __uint_as_float(xw[i] & 0xffff0000u);
+        }
+        if (UNC) {
+          const uint4 y = __ldg(reinterpret_cast<const uint4*>(base + branch_elem + row_elem) + g);
+          const uint32_t yw[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            lu[2 * i] = __uint_as_float(yw[i] << 16);
+            lu[2 * i + 1] = __uint_as_float(yw[i] & 0xffff0000u);
+          }
+        }
+      } else {
+        const float* base = static_cast<const float*>(logits);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const float4 x = __ldg(reinterpret_cast<const float4*>(base + row_elem) + 2 * g + h);
+          lc[4 * h] = x.x, lc[4 * h + 1] = x.y, lc[4 * h + 2] = x.z, lc[4 * h + 3] = x.w;
+          if (UNC) {
+            const float4 y = __ldg(reinterpret_cast<const float4*>(base + branch_elem + row_elem) + 2 * g + h);
+            lu[4 * h] = y.x, lu[4 * h + 1] = y.y, lu[4 * h + 2] = y.z, lu[4 * h + 3] = y.w;
+          }
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        float z = UNC ? __fmaf_rn(s, __fsub_rn(lc[e], lu[e]), lu[e]) : lc[e];
+        if (T != 1.0f) z = __fdiv_rn(z, T);
+        key[c * 8 + e] = topk_key(z);
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) key[c * 8 + e] = 0u;   // padding: below everything
+    }
+  }
+}
+
+// value of the K-th largest key held by the block (-inf if fewer than K keys lie above -inf)
+__device__ __forceinline__ float topk_select(const uint32_t (&key)[TK_CH * 8], int K, TopkShared& S) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float NEG_INF = __int_as_float(0xff800000);
+  int flip = 0;
+  // block statistics
+  uint32_t kmin = 0xffffffffu, kmax = 0u;
+#pragma unroll
+  for (int i = 0; i < TK_CH * 8; ++i) {
+    kmax = key[i] > kmax ? key[i] : kmax;
+    kmin = (key[i] > TK_KEY_NINF && key[i] < kmin) ? key[i] : kmin;
+  }
+  kmin = __reduce_min_sync(kFull, kmin);
+  kmax = __reduce_max_sync(kFull, kmax);
+  if (lane == 0) {
+    S.kmin[warp] = kmin;
+    S.kmax[warp] = kmax;
+  }
+  if (tid == 0) S.list_n = 0;
+  __syncthreads();
+#pragma unroll
+  for (int w = 0; w < TKW; ++w) {
+    kmin = S.kmin[w] < kmin ? S.kmin[w] : kmin;
+    kmax = S.kmax[w] > kmax ? S.kmax[w] : kmax;
+  }
+  // every exit goes through the barrier at the end: the next row reuses S
+  float answer = NEG_INF;
+  bool open = kmax > TK_KEY_NINF;                              // else: nothing above -inf
+  uint32_t lo = kmin, hi = kmax;
+  int c_lo = 0, c_hi = 0;
+  if (open) {
+    c_lo = topk_count(key, lo, S, flip);
+    open = c_lo >= K;                                          // else the K-th largest is -inf: nothing to cut
+  }
+  if (open) {
+    c_hi = topk_count(key, hi, S, flip);
+    if (c_hi >= K) {
+      answer = topk_value(hi);
+      open = false;
+    }
+  }
+  if (open) {
+    bool ranked = false;
+    for (int pass = 0; pass < 64; ++pass) {
+      if (hi - lo <= 1u) break;                                // count(>= lo) >= K > count(>= lo + 1)
+      if (c_lo - c_hi <= TK_LIST) {
+        ranked = true;
+        break;
+      }
+      uint32_t km = topk_key(0.5f * topk_value(lo) + 0.5f * topk_value(hi));
+      if (!(km > lo && km < hi)) km = lo + ((hi - lo) >> 1);
+      const int c = topk_count(key, km, S, flip);
+      if (c >= K) {
+        lo = km;
+        c_lo = c;
+      } else {
+        hi = km;
+        c_hi = c;
+      }
+    }
+    uint32_t result = lo;
+    if (ranked) {
+      // the keys in [lo, hi): at most TK_LIST of them; wanted: the r-th largest, r = K - count(>= hi)
+      if (tid == 0) S.result = lo;
+#pragma unroll
+      for (int i = 0; i < TK_CH * 8; ++i) {
+        if (key[i] >= lo && key[i] < hi) {
+          const int pos = atomicAdd(&S.list_n, 1);
+          if (pos < TK_LIST) S.list[pos] = key[i];
+        }
+      }
+      __syncthreads();
+      const int n = S.list_n < TK_LIST ? S.list_n : TK_LIST;
+      const int r = K - c_hi;
+      if (tid < n) {
+        const uint32_t e = S.list[tid];
+        int gt = 0, ge = 0;
+        for (int j = 0; j < n; ++j) {
+          const uint32_t o = S.list[j];
+          gt += o > e;
+          ge += o >= e;
+        }
+        if (gt < r && r <= ge) S.result = e;                   // equal keys write the same value
+      }
+      __syncthreads();
+      result = S.result;
+    }
+    answer = topk_value(result);
+  }
+  __syncthreads();
+  return answer;
+}
+
+// mode 0: one job per context with children (target and drafter row of that context);
+// mode 1: one job per bonus row (target row only), after the walk has listed them.
+template <bool BF16, bool UNC>
+__global__ void __launch_bounds__(TKT, 2) lantern_topk_kernel(VerifyParams P, int mode) {
+  __shared__ TopkShared S;
+  const int V = P.V, R = P.R, K = P.top_k;
+  const float T = P.T == 0.0f ? 1.0f : P.T;   // greedy decoding works at temperature 1
+  const size_t branch = static_cast<size_t>(P.B) * R * V;
+  uint32_t key[TK_CH * 8];
+  if (mode == 0) {
+    const int n_heavy = P.counters->n_heavy;
+    const int total = n_heavy + P.counters->n_light;
+    const int cap = P.B * P.N;
+    for (int w = blockIdx.x; w < total; w += gridDim.x) {
+      const int item = P.work[w < n_heavy ? w : cap - 1 - (w - n_heavy)].item;
+      const size_t row = static_cast<size_t>(item) * V;
+      topk_load_keys<BF16, UNC>(P.target, row, branch, V, P.cfg_scale, T, key);
+      const float tq = topk_select(key, K, S);
+      if (threadIdx.x == 0) P.thr_q[item] = tq;
+      if (P.T != 0.0f) {   // sampling: the drafter row of the same context
+        topk_load_keys<BF16, false>(P.draft, row, 0, V, 1.0f, T, key);
+        const float tp = topk_select(key, K, S);
+        if (threadIdx.x == 0) P.thr_p[item] = tp;
+      }
+    }
+  } else {
+    const int count = P.counters->n_bonus;
+    for (int i = blockIdx.x; i < count; i += gridDim.x) {
+      const int item = P.bonus_seq[i] * R + P.bonus_ctx[i];
+      topk_load_keys<BF16, UNC>(P.target, static_cast<size_t>(item) * V, branch, V, P.cfg_scale, T, key);
+      const float tq = topk_select(key, K, S);
+      if (threadIdx.x == 0) P.thr_q[item] = tq;
+    }
+  }
+}
+
+}  // namespace lantern

@@ -1,5 +1,5 @@
 """CUDA variants against the oracle: cosine neighbour metric (Section 6.2.1), JSD bound
-(Section 6.2.2) in sampling and in greedy decoding.  Comparison rules are those of
+(Section 6.2.2) and top-k logit filter (Appendix B.2) in sampling and in greedy decoding.  Comparison rules are those of
 tests/parity.py and tests/test_gpu_greedy.py (the cut's window is in JSD units here)."""
 import numpy as np
 import pytest
@@ -102,3 +102,83 @@ def test_bad_variant_arguments():
     lib = lt.load_library()
     assert lib.lantern_build_workspace_bytes_metric(V, 8, k, 5) == 0
     assert lib.lantern_verify_workspace_bytes_ex(4, 4, -1) == 0
+
+
+# ------------------------------------------------------------------------------------ top-k filter
+def _table(V, k):
+    cb = li.codebook_gaussian(V, 8, seed=31)
+    if V <= 2048:
+        host = oracle.build_neighbors(cb, k)[0]
+        return host, torch.from_numpy(host).cuda()
+    dev = lt.build_neighbors(torch.from_numpy(cb).cuda(), k, with_dist=False)[0]
+    return dev.cpu().numpy(), dev
+
+
+@pytest.mark.parametrize("V,k,N,B,dtype,unc,T,K,div", [
+    (1024, 16, 4, 64, li.F32, False, 1.0, 100, oracle.DIV_TVD),
+    (1024, 16, 4, 64, li.BF16, True, 1.0, 100, oracle.DIV_TVD),      # bf16: ties at the threshold are kept
+    (1000, 300, 7, 40, li.BF16, True, 0.7, 37, oracle.DIV_TVD),      # temperature: thresholds on l / T
+    (8192, 1000, 5, 12, li.F32, True, 1.0, 1000, oracle.DIV_JSD),
+    (16384, 1000, 5, 24, li.BF16, True, 1.0, 1000, oracle.DIV_TVD),  # the text-conditional setting of Appendix B.2
+    (16384, 1000, 5, 24, li.BF16, True, 1.0, 2000, oracle.DIV_JSD),
+    (512, 32, 6, 50, li.BF16, True, 1.0, 1, oracle.DIV_TVD),         # K = 1: both distributions are point masses
+    (512, 32, 6, 50, li.BF16, False, 1.0, 511, oracle.DIV_TVD),      # one token cut
+    (512, 32, 6, 50, li.F32, False, 1.0, 512, oracle.DIV_TVD),       # K = V: filter off
+    (8, 8, 3, 17, li.BF16, False, 1.0, 3, oracle.DIV_TVD),
+])
+def test_top_k_sampling(V, k, N, B, dtype, unc, T, K, div):
+    host, dev = _table(V, k)
+    inp = li.verify_inputs(B, N, V, dtype=dtype, has_uncond=unc, cfg_scale=3.0 if unc else 1.0, T=T, sigma_target=1.0,
+                           sigma_draft=0.6, rho=0.9, seed=11 + V + K)
+    gpu = run_gpu(inp, dev, 0.2, divergence=div, top_k=K)
+    res = compare(inp, host, 0.2, gpu, divergence=div, top_k=K)
+    assert_parity(res)
+    assert res["nodes_tested"] >= (B if K > 1 else B // 4)     # K = 1 leaves many zero-weight residuals (reported)
+    assert res["degenerate"] == 0 or K == 1
+    if K < V // 2:     # the filter matters: without it the decisions differ somewhere
+        plain = oracle.verify_inputs(inp, host, 0.2, div)
+        filt = oracle.verify_inputs(inp, host, 0.2, div, K)
+        assert not (np.array_equal(plain.next_token, filt.next_token) and np.array_equal(plain.qa, filt.qa))
+
+
+def test_top_k_trees_and_masked_logits():
+    V, k, K = 2048, 64, 200
+    host = oracle.build_neighbors(li.codebook_clustered(V, 8, seed=5), k)[0]
+    dev = torch.from_numpy(host).cuda()
+    par = li.tree_parents(96, 30, depth=5, seed=3)
+    inp = li.verify_inputs(96, 30, V, dtype=li.BF16, has_uncond=True, cfg_scale=3.0, sigma_target=1.0,
+                           sigma_draft=1.0, rho=0.9, parents=par, seed=79)
+    neg_inf = np.uint16(0xFF80)
+    inp.target_logits[:, 3, :, 100:1990] = neg_inf      # fewer than K tokens above -inf: nothing to cut
+    inp.draft_logits[3, :, 100:1990] = neg_inf
+    inp.target_logits[:, 4, :, ::3] = neg_inf           # masked tokens elsewhere
+    gpu = run_gpu(inp, dev, 0.15, top_k=K)
+    res = compare(inp, host, 0.15, gpu, top_k=K)
+    assert_parity(res)
+    assert res["nodes_tested"] > 96 * 3
+
+
+@pytest.mark.parametrize("V,k,N,B,dtype,unc,K,div", [
+    (1024, 16, 4, 64, li.BF16, True, 50, oracle.DIV_TVD),
+    (16384, 1000, 5, 24, li.BF16, True, 1000, oracle.DIV_TVD),
+    (8192, 1000, 5, 12, li.F32, True, 2000, oracle.DIV_JSD),
+])
+def test_top_k_greedy(V, k, N, B, dtype, unc, K, div):
+    host, dev = _table(V, k)
+    inp = li.verify_inputs(B, N, V, dtype=dtype, has_uncond=unc, cfg_scale=3.0, sigma_target=1.0,
+                           sigma_draft=0.4, rho=0.9, seed=5 + V)
+    greedy_check(inp, host, dev, 0.2, divergence=div, top_k=K)
+
+
+def test_top_k_nan_rows_are_still_reported():
+    V, k = 1024, 16
+    host, dev = _table(V, k)
+    inp = li.verify_inputs(12, 4, V, dtype=li.F32, has_uncond=False, cfg_scale=1.0, sigma_target=1.0,
+                           sigma_draft=0.4, rho=0.9, seed=8)
+    inp.target_logits[0, 3, 0, 17] = np.nan
+    inp.draft_logits[6, 0, 5] = np.nan
+    ora = oracle.verify_inputs(inp, host, 0.3, top_k=64)
+    g = run_gpu(inp, dev, 0.3, top_k=64)
+    assert np.array_equal(g.status.cpu().numpy(), ora.status) and ora.status[3] and ora.status[6]
+    ok = ora.status == 0
+    assert np.array_equal(g.accept_len.cpu().numpy()[ok], ora.accept_len[ok])

@@ -141,7 +141,7 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def oracle_sample_rate(host_inp, table_host, delta, budget_s=15.0, greedy=False, divergence=0):
+def oracle_sample_rate(host_inp, table_host, delta, budget_s=15.0, greedy=False, divergence=0, top_k=0):
     """Oracle throughput (drafted positions verified per second) on as many leading sequences of
     `host_inp` as fit in about `budget_s` seconds; returns (rate, n_sequences, seconds)."""
     import dataclasses
@@ -161,9 +161,9 @@ def oracle_sample_rate(host_inp, table_host, delta, budget_s=15.0, greedy=False,
         t0 = time.perf_counter()
         if greedy:
             oracle.verify_greedy(part.target_logits, part.dtype, part.cfg_scale, part.has_uncond, part.draft_tokens,
-                                 part.tree_parents, table_host, delta, divergence)
+                                 part.tree_parents, table_host, delta, divergence, top_k)
         else:
-            oracle.verify_inputs(part, table_host, delta, divergence)
+            oracle.verify_inputs(part, table_host, delta, divergence, top_k)
         t_used += time.perf_counter() - t0
         done += n
         pos += n * host_inp.N
@@ -227,9 +227,9 @@ def run_reference(args, rank, world):
         t1 = time.perf_counter()
         if args.greedy:
             oracle.verify_greedy(inp.target_logits, inp.dtype, inp.cfg_scale, inp.has_uncond, inp.draft_tokens,
-                                 inp.tree_parents, tab, cfg["delta"], div)
+                                 inp.tree_parents, tab, cfg["delta"], div, args.top_k)
         else:
-            oracle.verify_inputs(inp, tab, cfg["delta"], div)
+            oracle.verify_inputs(inp, tab, cfg["delta"], div, args.top_k)
         dt = time.perf_counter() - t1
         if step >= args.warmup:
             steps_t.append(dt)
@@ -241,7 +241,7 @@ def run_reference(args, rank, world):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": args.workload, "V": cfg["V"], "k": cfg["k"], "delta": cfg["delta"], "N": cfg["N"],
                    "T": 0.0 if args.greedy else cfg["T"], "divergence": args.divergence, "metric": args.metric,
-                   "sequences_per_step": nseq},
+                   "top_k": args.top_k, "sequences_per_step": nseq},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
                          "sample": f"{nseq} sequences x {cfg['N']} drafts per step of the {args.workload} workload "
                                    f"(bounded sample; neighbour rows built by the oracle outside the timed region)"},
@@ -266,6 +266,8 @@ def main():
     ap.add_argument("--divergence", default="tvd", choices=["tvd", "jsd"],
                     help="what delta bounds (Section 6.2.2); the JSD run uses the workload's delta as it is")
     ap.add_argument("--metric", default="l2", choices=["l2", "cosine"], help="latent proximity of the table")
+    ap.add_argument("--top-k", type=int, default=0, dest="top_k",
+                    help="top-k logit filter of the generation settings (Appendix B.2); 0 = off")
     ap.add_argument("--greedy", action="store_true",
                     help="run the workload at T = 0 (greedy decoding: no drafter rows, no random numbers)")
     args = ap.parse_args()
@@ -318,7 +320,7 @@ def main():
     torch.cuda.synchronize()
     alg_bytes = algorithmic_bytes(cfg, B, d["tree_parents"], args.greedy)
     T = 0.0 if args.greedy else d["T"]
-    ws = torch.empty(lt.verify_workspace_bytes(B, N), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(lt.verify_workspace_bytes(B, N, args.top_k), dtype=torch.uint8, device="cuda")
     i32 = dict(dtype=torch.int32, device="cuda")
     out = lt.VerifyOutputs(accept_len=torch.empty(B, **i32), next_token=torch.empty(B, **i32),
                            accept_path=torch.empty((B, N), **i32), status=torch.empty(B, **i32),
@@ -328,7 +330,7 @@ def main():
     def step():
         lt.verify(d["target_logits"], None if args.greedy else d["draft_logits"], d["cfg_scale"], T, d["draft_tokens"],
                   d["tree_parents"], table, delta, None if args.greedy else d["uniforms"], out=out, workspace=ws,
-                  stream=stream, divergence=args.divergence)
+                  stream=stream, divergence=args.divergence, top_k=args.top_k)
 
     for _ in range(args.warmup):
         step()
@@ -412,7 +414,7 @@ def main():
         n_s = min(B, 8192 if cfg["N"] <= 8 else 256)
         host_inp = lid.to_host(d, rows=np.arange(n_s))
         rate, n_done, secs = oracle_sample_rate(host_inp, table.cpu().numpy(), delta, greedy=args.greedy,
-                                                divergence=1 if args.divergence == "jsd" else 0)
+                                                divergence=1 if args.divergence == "jsd" else 0, top_k=args.top_k)
         cpu = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
                "sample": f"first {n_done} sequences ({n_done * N} drafted positions) of this call, {secs:.1f} s"}
 
@@ -425,6 +427,7 @@ def main():
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": args.workload, "note": w["note"], "sequences_per_call": B, "drafts_per_sequence": N,
                        "V": V, "k": k, "delta": delta, "cfg_scale": cfg["cfg_scale"], "T": T, "divergence": args.divergence, "metric": args.metric,
+                       "top_k": args.top_k,
                        "logits": "bf16" if cfg["dtype"] == li.BF16 else "f32", "rho": args.rho,
                        "l2_policy": "inputs larger than L2 (%.2f GB of logits per call)" %
                                     ((d["target_logits"].numel() + (0 if args.greedy else d["draft_logits"].numel())) *
@@ -435,7 +438,8 @@ def main():
                          "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
                          "traffic": None if args.greedy else ncu_traffic(args.workload, cfg, alg_bytes),
                          "algorithmic_bytes_per_launch": int(alg_bytes), "kernel_ms": fused_ms},
-            "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": 4 * args.steps, "clocks": clocks,
+            "cpu_baseline": cpu, "e2e": e2e,
+            "gpu_launches": (4 + (0 if not 0 < args.top_k < V else (1 if args.greedy else 2))) * args.steps, "clocks": clocks,
             "neighbor_build": {"ms": build_ms, "V": V, "D": cfg["D"], "k": k,
                                "pairs_per_s": V * V / (build_ms * 1e-3)},
             "outputs": {"mean_accept_len": accept_mean, "sequences_with_status_bits": status_bad},

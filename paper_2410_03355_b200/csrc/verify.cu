@@ -19,228 +19,9 @@
 // Precision: processed logits are fp32 (difference, fused multiply-add, division, each
 // rounded once); exponentials are fp32 with ~2.5e-7 relative error; every sum over more
 // than eight terms and every threshold comparison is done in double precision.
-#include <cuda_runtime.h>
-#include <math.h>
-#include <stdint.h>
-
-#include "lantern.h"
-#include "lantern_device.cuh"
+#include "verify_common.cuh"
 
 namespace lantern {
-
-constexpr int NT = 1024;        // threads per CTA of the context / bonus kernels
-constexpr int NW = NT / 32;
-constexpr int LOG_NT = 10;
-constexpr int MAX_N = 1024;
-
-struct Counters {               // first 256 bytes of the workspace, zeroed per call
-  int work_next;                // dynamic part of the work counter
-  int n_heavy;                  // contexts with >= 2 children (handed out first)
-  int n_light;                  // contexts with exactly 1 child
-  int n_bonus;                  // sequences whose walk ended on a childless context
-};
-
-struct Record {                 // result of one context
-  int accepted;                 // accepted child node; -1 if every child was rejected; kLeaf if it has none
-  int token;                    // replacement token if every child was rejected
-  int status;                   // LANTERN_ST_* bits found in this context
-  int pad;
-};
-constexpr int kLeaf = -2;
-
-struct ChildInfo {              // one drafted node, stored in the order its parent context tries it
-  int node;                     // node index within the sequence
-  int token;                    // x~
-  float r;                      // its acceptance uniform
-  int pad;
-};
-
-struct WorkItem {               // one context with children: everything its CTA needs, in one 32-byte load
-  int item;                     // b * R + c  (row index of the context); -1 = none
-  int cbase;                    // index of its first child in the ChildInfo array
-  int nchild;
-  int node0;                    // first child, inlined
-  int tok0;
-  float r0;
-  float u_final;                // the sequence's uniform for the final draw
-  int pad;
-};
-
-struct VerifyParams {
-  const void* target;
-  const void* draft;
-  const int32_t* tokens;
-  const int32_t* parents;
-  const int32_t* nbr;
-  const float* uniforms;
-  int32_t* out_len;
-  int32_t* out_tok;
-  int32_t* out_path;
-  int32_t* out_status;
-  float* out_qa;
-  float* out_px;
-  int32_t* out_m;
-  // workspace pieces
-  Counters* counters;
-  WorkItem* work;               // [B*N]: heavy items from the front, light items from the back
-  ChildInfo* children;          // [B, N]
-  Record* records;              // [B, R]
-  int32_t* seq_status;          // [B]
-  int32_t* bonus_seq;           // [B]
-  int32_t* bonus_ctx;           // [B]
-  int B, N, R, V, k;
-  float cfg_scale, T, delta;
-  int divergence;               // LANTERN_DIV_TVD or LANTERN_DIV_JSD: what delta bounds
-  int top_k;                    // logit filter; 0 = off (then thr_q, thr_p are null)
-  float* thr_q;                 // [B, R] top_k-th largest processed target logit of a context row
-  float* thr_p;                 // [B, R] the same for the drafter row
-};
-
-// ---------------------------------------------------------------------------------------
-// layout of a row held by a CTA: thread t owns, for chunk c, the eight consecutive tokens
-// [(c*NT + t)*8, +8).  In shared memory the numerators E are stored so that both 16-byte
-// halves of a thread's chunk are bank-conflict free: physical float index of token x below.
-// ---------------------------------------------------------------------------------------
-__device__ __forceinline__ int phys(int x) {
-  const int g = x >> 3;
-  const int c = g >> LOG_NT;
-  const int t = g & (NT - 1);
-  const int h = (x >> 2) & 1;
-  return ((((c << 1) | h) << LOG_NT) + t) << 2 | (x & 3);
-}
-
-struct BlockScratch {
-  double wt[2 * NW];            // per-(chunk, warp) totals
-  double wbase[2 * NW];         // their exclusive prefix
-  double sp[NW];
-  double total;
-  double total2;
-  double sm;
-  float fm[2 * NW];
-  float px;
-  int first;
-  int win;
-  int tok;
-  int item;
-  int bad;
-};
-
-// max of two values over the block
-__device__ __forceinline__ void block_max2(float& a, float& b, BlockScratch& S, int lane, int warp) {
-  a = warp_max(a);
-  b = warp_max(b);
-  if (lane == 0) {
-    S.fm[warp] = a;
-    S.fm[NW + warp] = b;
-  }
-  __syncthreads();
-  a = warp_max(S.fm[lane]);
-  b = warp_max(S.fm[NW + lane]);
-  __syncthreads();
-}
-
-// sum of two doubles over the block
-__device__ __forceinline__ void block_sum2(double& a, double& b, BlockScratch& S, int lane, int warp) {
-  a = warp_sum(a);
-  b = warp_sum(b);
-  if (lane == 0) {
-    S.wt[warp] = a;
-    S.wt[NW + warp] = b;
-  }
-  __syncthreads();
-  a = warp_sum(S.wt[lane]);
-  b = warp_sum(S.wt[NW + lane]);
-  __syncthreads();
-}
-
-__device__ __forceinline__ float sum8(const float* v) {
-  return ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
-}
-
-// Exclusive prefix (over the order chunk-major, then thread) of per-chunk sums cs[c], the
-// grand total in S.total, and the block sum of `extra` in S.total2.
-template <int CH>
-__device__ __forceinline__ void block_scan_chunks(const double (&cs)[CH], double (&excl)[CH], double extra,
-                                                  BlockScratch& S, int lane, int warp) {
-  double incl[CH];
-#pragma unroll
-  for (int c = 0; c < CH; ++c) {
-    incl[c] = warp_incl_scan(cs[c], lane);
-    if (lane == 31) S.wt[c * NW + warp] = incl[c];
-  }
-  extra = warp_sum(extra);
-  if (lane == 0) S.sp[warp] = extra;
-  __syncthreads();
-  if (warp == 0) {
-    double carry = 0.0;
-#pragma unroll
-    for (int c = 0; c < CH; ++c) {
-      const double t = S.wt[c * NW + lane];
-      const double in = warp_incl_scan(t, lane);
-      S.wbase[c * NW + lane] = carry + in - t;
-      carry += __shfl_sync(kFull, in, 31);
-    }
-    const double e = warp_sum(S.sp[lane]);
-    if (lane == 0) {
-      S.total = carry;
-      S.total2 = e;
-    }
-  }
-  __syncthreads();
-#pragma unroll
-  for (int c = 0; c < CH; ++c) excl[c] = S.wbase[c * NW + warp] + incl[c] - cs[c];
-}
-
-// Inverse CDF over the weights w (registers, layout above): smallest token whose inclusive
-// cumulative weight exceeds target; if rounding leaves none, the largest token of positive
-// weight; -1 if there is no positive weight.  Must be called by the whole block.
-template <int CH>
-__device__ __forceinline__ int block_draw(const float (&w)[CH * 8], const double (&cs)[CH], const double (&excl)[CH],
-                                          double target, int V, BlockScratch& S, int tid) {
-  if (tid == 0) {
-    S.win = 0x7fffffff;
-    S.tok = -1;
-  }
-  __syncthreads();
-  int cand = 0x7fffffff;
-#pragma unroll
-  for (int c = CH - 1; c >= 0; --c)
-    if (excl[c] + cs[c] > target) cand = c * NT + tid;
-  const int wmin = __reduce_min_sync(kFull, cand);
-  if ((tid & 31) == 0 && wmin != 0x7fffffff) atomicMin(&S.win, wmin);
-  __syncthreads();
-  const int win = S.win;
-  if (win == 0x7fffffff) {
-    int last = -1;
-#pragma unroll
-    for (int c = 0; c < CH; ++c)
-#pragma unroll
-      for (int e = 0; e < 8; ++e)
-        if (w[c * 8 + e] > 0.0f) last = (c * NT + tid) * 8 + e;
-    if (last >= V) last = -1;
-    if (last >= 0) atomicMax(&S.tok, last);
-  } else if ((win & (NT - 1)) == tid) {
-    const int wc = win >> LOG_NT;
-    int tok = -1, lastpos = -1;
-#pragma unroll
-    for (int c = 0; c < CH; ++c) {
-      if (c == wc) {
-        double cum = excl[c];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const float wv = w[c * 8 + e];
-          cum += static_cast<double>(wv);
-          if (wv > 0.0f) lastpos = e;
-          if (tok < 0 && cum > target) tok = e;
-        }
-      }
-    }
-    if (tok < 0) tok = lastpos;
-    S.tok = win * 8 + tok;
-  }
-  __syncthreads();
-  return S.tok;
-}
 
 // ---------------------------------------------------------------------------------------
 // kernel 1: plan.  One warp per sequence: validate tokens / parents / uniforms, bucket the
@@ -501,26 +282,51 @@ static thread_local cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
 // mode 1 = rows of the bonus draws (after the walk)
 template <bool BF16, bool UNC>
 static cudaError_t launch_topk(const VerifyParams& P, int mode, long long jobs, int sms, cudaStream_t st) {
-  const long long slots = 2ll * sms;
+  auto kt = lantern_topk_kernel<BF16, UNC>;
+  const size_t smem = static_cast<size_t>(P.V) * (UNC ? 2 : 1) * (BF16 ? 2 : 4);   // one job's raw rows
+  cudaError_t e = cudaFuncSetAttribute(kt, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
+  int per_sm = 0;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kt, TKT, smem);
+  if (e != cudaSuccess) return e;
+  if (per_sm < 1) return cudaErrorInvalidConfiguration;
+  const long long slots = static_cast<long long>(sms) * per_sm;
   const int grid = static_cast<int>(jobs < slots ? (jobs > 0 ? jobs : 1) : slots);
-  lantern_topk_kernel<BF16, UNC><<<grid, TKT, 0, st>>>(P, mode);
+  kt<<<grid, TKT, smem, st>>>(P, mode);
   return cudaGetLastError();
 }
 
-template <int CHC, bool BF16, bool UNC, bool TONE, bool JSD, bool TOPK>
-static cudaError_t launch_verify(const VerifyParams& P, long long items, int sms, int grid_ctx, int grid_bonus,
-                                 size_t smem_bytes, cudaStream_t st) {
-  constexpr int CHB = CHC == 8 ? 2 : 1;   // the bonus kernel runs 1024 threads per row
-  auto kc = lantern_context_kernel<CHC, BF16, UNC, TONE, JSD, TOPK>;
-  cudaError_t e = cudaFuncSetAttribute(kc, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
-  if (e != cudaSuccess) return e;
+// the variants of the fused context kernel live in verify_context_v<tone + 2 jsd + 4 topk>.cu
+#define LANTERN_DECLARE_VARIANT(n) \
+  cudaError_t launch_context_v##n(const VerifyParams&, int, bool, bool, int, size_t, cudaStream_t);
+LANTERN_DECLARE_VARIANT(0) LANTERN_DECLARE_VARIANT(1) LANTERN_DECLARE_VARIANT(2) LANTERN_DECLARE_VARIANT(3)
+LANTERN_DECLARE_VARIANT(4) LANTERN_DECLARE_VARIANT(5) LANTERN_DECLARE_VARIANT(6) LANTERN_DECLARE_VARIANT(7)
+#undef LANTERN_DECLARE_VARIANT
+
+cudaError_t launch_context_kernel(const VerifyParams& P, int CH, bool bf16, bool uncond, bool tone, bool jsd, bool topk,
+                                  int grid, size_t smem_bytes, cudaStream_t st) {
+  switch ((tone ? 1 : 0) | (jsd ? 2 : 0) | (topk ? 4 : 0)) {
+    case 0: return launch_context_v0(P, CH, bf16, uncond, grid, smem_bytes, st);
+    case 1: return launch_context_v1(P, CH, bf16, uncond, grid, smem_bytes, st);
+    case 2: return launch_context_v2(P, CH, bf16, uncond, grid, smem_bytes, st);
+    case 3: return launch_context_v3(P, CH, bf16, uncond, grid, smem_bytes, st);
+    case 4: return launch_context_v4(P, CH, bf16, uncond, grid, smem_bytes, st);
+    case 5: return launch_context_v5(P, CH, bf16, uncond, grid, smem_bytes, st);
+    case 6: return launch_context_v6(P, CH, bf16, uncond, grid, smem_bytes, st);
+    default: return launch_context_v7(P, CH, bf16, uncond, grid, smem_bytes, st);
+  }
+}
+
+template <int CHB, bool BF16, bool UNC, bool TOPK>
+static cudaError_t launch_verify(const VerifyParams& P, int CH, bool tone, bool jsd, long long items, int sms,
+                                 int grid_ctx, int grid_bonus, size_t smem_bytes, cudaStream_t st) {
+  cudaError_t e;
   if (TOPK) {
-    e = launch_topk<BF16, UNC>(P, 0, items, sms, st);
+    e = launch_topk<BF16, UNC>(P, 0, 2 * items, sms, st);
     if (e != cudaSuccess) return e;
   }
   if (g_ev_before && g_ev_after) cudaEventRecord(g_ev_before, st);
-  kc<<<grid_ctx, CTX_THREADS, smem_bytes, st>>>(P);
-  e = cudaGetLastError();
+  e = launch_context_kernel(P, CH, BF16, UNC, tone, jsd, TOPK, grid_ctx, smem_bytes, st);
   if (e != cudaSuccess) return e;
   if (g_ev_before && g_ev_after) cudaEventRecord(g_ev_after, st);
   lantern_walk_kernel<<<(P.B + 127) / 128, 128, 0, st>>>(P);
@@ -530,7 +336,7 @@ static cudaError_t launch_verify(const VerifyParams& P, long long items, int sms
     e = launch_topk<BF16, UNC>(P, 1, P.B, sms, st);
     if (e != cudaSuccess) return e;
   }
-  lantern_bonus_kernel<CHB, BF16, UNC, TOPK><<<grid_bonus, NT, 0, st>>>(P);
+  lantern_bonus_kernel<CHB, BF16, UNC, TOPK><<<grid_bonus, NT, 0, st>>>(P);   // CHB: 1024 threads per row
   return cudaGetLastError();
 }
 
@@ -722,19 +528,15 @@ static lantern_status verify_impl(const void* target_logits, const void* draft_l
 #undef LANTERN_GREEDY
     return e == cudaSuccess ? LANTERN_OK : LANTERN_E_CUDA;
   }
-#define LANTERN_DISPATCH2(CHV, TV, JV, KV)                                                                        \
-  (bf ? (un ? launch_verify<CHV, true, true, TV, JV, KV>(P, items, sms, grid_ctx, grid_bonus, smem_bytes, st)     \
-            : launch_verify<CHV, true, false, TV, JV, KV>(P, items, sms, grid_ctx, grid_bonus, smem_bytes, st))   \
-      : (un ? launch_verify<CHV, false, true, TV, JV, KV>(P, items, sms, grid_ctx, grid_bonus, smem_bytes, st)    \
-            : launch_verify<CHV, false, false, TV, JV, KV>(P, items, sms, grid_ctx, grid_bonus, smem_bytes, st)))
-  // the JSD and top-k variants are built for the general-temperature code only (T = 1 runs through it unchanged)
-#define LANTERN_DISPATCH(CHV)                                                                                     \
-  (topk ? (divergence == LANTERN_DIV_JSD ? LANTERN_DISPATCH2(CHV, false, true, true)                              \
-                                         : LANTERN_DISPATCH2(CHV, false, false, true))                            \
-        : (divergence == LANTERN_DIV_JSD                                                                          \
-               ? LANTERN_DISPATCH2(CHV, false, true, false)                                                       \
-               : (T == 1.0f ? LANTERN_DISPATCH2(CHV, true, false, false) : LANTERN_DISPATCH2(CHV, false, false, false))))
-  e = CH == 8 ? LANTERN_DISPATCH(8) : (CH == 4 ? LANTERN_DISPATCH(4) : (CH == 2 ? LANTERN_DISPATCH(2) : LANTERN_DISPATCH(1)));
+  // every combination of the compile-time variants exists: T = 1 never meets the division code
+  const bool tone = T == 1.0f, jsd = divergence == LANTERN_DIV_JSD;
+#define LANTERN_DISPATCH2(CHB, KV)                                                                              \
+  (bf ? (un ? launch_verify<CHB, true, true, KV>(P, CH, tone, jsd, items, sms, grid_ctx, grid_bonus, smem_bytes, st)   \
+            : launch_verify<CHB, true, false, KV>(P, CH, tone, jsd, items, sms, grid_ctx, grid_bonus, smem_bytes, st)) \
+      : (un ? launch_verify<CHB, false, true, KV>(P, CH, tone, jsd, items, sms, grid_ctx, grid_bonus, smem_bytes, st)  \
+            : launch_verify<CHB, false, false, KV>(P, CH, tone, jsd, items, sms, grid_ctx, grid_bonus, smem_bytes, st)))
+#define LANTERN_DISPATCH(CHB) (topk ? LANTERN_DISPATCH2(CHB, true) : LANTERN_DISPATCH2(CHB, false))
+  e = CH == 8 ? LANTERN_DISPATCH(2) : LANTERN_DISPATCH(1);
 #undef LANTERN_DISPATCH2
 #undef LANTERN_DISPATCH
   return e == cudaSuccess ? LANTERN_OK : LANTERN_E_CUDA;

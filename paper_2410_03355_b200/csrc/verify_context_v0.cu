@@ -1,0 +1,6 @@
+// Fused context kernel, variant 0: temperature 1 compiled out = 0, JSD bound = 0, top-k thresholds = 0.
+#define LANTERN_VARIANT_TONE false
+#define LANTERN_VARIANT_JSD false
+#define LANTERN_VARIANT_TOPK false
+#define LANTERN_VARIANT_NAME launch_context_v0
+#include "verify_context_variant.cuh"

@@ -1,0 +1,6 @@
+// Fused context kernel, variant 3: temperature 1 compiled out = 1, JSD bound = 1, top-k thresholds = 0.
+#define LANTERN_VARIANT_TONE true
+#define LANTERN_VARIANT_JSD true
+#define LANTERN_VARIANT_TOPK false
+#define LANTERN_VARIANT_NAME launch_context_v3
+#include "verify_context_variant.cuh"

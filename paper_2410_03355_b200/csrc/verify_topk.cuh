@@ -2,8 +2,10 @@
 // value of the top_k-th largest processed logit; included by verify.cu.
 //
 // The verification kernels then treat every processed logit below that value as -inf (logits
-// equal to it are all kept).  One CTA of TKT threads per row job, the row's processed logits held
-// in registers as order-preserving 32-bit keys (64 per thread at V = 16384):
+// equal to it are all kept).  One CTA of TKT threads per row job; the raw row(s) arrive in shared
+// memory by bulk copy, and as soon as they have been turned into order-preserving 32-bit keys in
+// registers (64 per thread at V = 16384) the copy of the CTA's next job is started, so that it runs
+// under the selection:
 //   1. block statistics: number of keys above -inf, smallest such key, largest key;
 //   2. bisection on the key interval [lo, hi) with the invariant
 //        count(key >= lo) >= K > count(key >= hi),
@@ -22,15 +24,16 @@ namespace lantern {
 constexpr int TKT = 256;
 constexpr int TKW = TKT / 32;
 constexpr int TK_CH = 8;            // 8-token chunks per thread: 8 * 8 * 256 = 16384 tokens at most
-constexpr int TK_LIST = 256;
+constexpr int TK_LIST = 128;
 constexpr uint32_t TK_KEY_NINF = 0x007fffffu;
 
 struct TopkShared {
   int cnt[2][TKW];
   unsigned kmin[TKW], kmax[TKW];
-  unsigned list[TK_LIST];
+  __align__(16) unsigned list[TK_LIST];
   int list_n;
   unsigned result;
+  unsigned long long bar_full;
 };
 
 __device__ __forceinline__ uint32_t topk_key(float z) {
@@ -45,10 +48,15 @@ __device__ __forceinline__ float topk_value(uint32_t key) {
 
 // number of this thread's keys >= t, summed over the block (every thread gets the sum)
 __device__ __forceinline__ int topk_count(const uint32_t (&key)[TK_CH * 8], uint32_t t, TopkShared& S, int& flip) {
-  int c = 0;
+  int c0 = 0, c1 = 0, c2 = 0, c3 = 0;   // four chains: the adds do not wait for one another
 #pragma unroll
-  for (int i = 0; i < TK_CH * 8; ++i) c += key[i] >= t;
-  c = __reduce_add_sync(kFull, c);
+  for (int i = 0; i < TK_CH * 8; i += 4) {
+    c0 += key[i] >= t;
+    c1 += key[i + 1] >= t;
+    c2 += key[i + 2] >= t;
+    c3 += key[i + 3] >= t;
+  }
+  const int c = __reduce_add_sync(kFull, (c0 + c1) + (c2 + c3));
   if ((threadIdx.x & 31) == 0) S.cnt[flip][threadIdx.x >> 5] = c;
   __syncthreads();
   int tot = 0;
@@ -130,6 +138,7 @@ __device__ __forceinline__ float topk_select(const uint32_t (&key)[TK_CH * 8], i
     S.kmax[warp] = kmax;
   }
   if (tid == 0) S.list_n = 0;
+  if (tid < TK_LIST) S.list[tid] = 0u;   // unused slots: below every listed key
   __syncthreads();
 #pragma unroll
   for (int w = 0; w < TKW; ++w) {
@@ -175,11 +184,26 @@ __device__ __forceinline__ float topk_select(const uint32_t (&key)[TK_CH * 8], i
     if (ranked) {
       // the keys in [lo, hi): at most TK_LIST of them; wanted: the r-th largest, r = K - count(>= hi)
       if (tid == 0) S.result = lo;
+      // compaction without a chain of atomics: own count, warp scan, one atomic per warp, then the writes
+      int mine = 0;
 #pragma unroll
-      for (int i = 0; i < TK_CH * 8; ++i) {
-        if (key[i] >= lo && key[i] < hi) {
-          const int pos = atomicAdd(&S.list_n, 1);
-          if (pos < TK_LIST) S.list[pos] = key[i];
+      for (int i = 0; i < TK_CH * 8; ++i) mine += (key[i] >= lo) & (key[i] < hi);
+      int incl = mine;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(kFull, incl, o);
+        if (lane >= o) incl += v;
+      }
+      int base = 0;
+      if (lane == 31) base = atomicAdd(&S.list_n, incl);
+      int pos = __shfl_sync(kFull, base, 31) + incl - mine;
+      if (mine) {
+#pragma unroll
+        for (int i = 0; i < TK_CH * 8; ++i) {
+          if (key[i] >= lo && key[i] < hi) {
+            if (pos < TK_LIST) S.list[pos] = key[i];
+            ++pos;
+          }
         }
       }
       __syncthreads();
@@ -188,10 +212,11 @@ __device__ __forceinline__ float topk_select(const uint32_t (&key)[TK_CH * 8], i
       if (tid < n) {
         const uint32_t e = S.list[tid];
         int gt = 0, ge = 0;
-        for (int j = 0; j < n; ++j) {
-          const uint32_t o = S.list[j];
-          gt += o > e;
-          ge += o >= e;
+#pragma unroll 8
+        for (int j = 0; j < TK_LIST / 4; ++j) {                // slots past n hold key 0: below every listed key
+          const uint4 o = *reinterpret_cast<const uint4*>(&S.list[4 * j]);
+          gt += (o.x > e) + (o.y > e) + (o.z > e) + (o.w > e);
+          ge += (o.x >= e) + (o.y >= e) + (o.z >= e) + (o.w >= e);
         }
         if (gt < r && r <= ge) S.result = e;                   // equal keys write the same value
       }
@@ -204,39 +229,132 @@ __device__ __forceinline__ float topk_select(const uint32_t (&key)[TK_CH * 8], i
   return answer;
 }
 
-// mode 0: one job per context with children (target and drafter row of that context);
-// mode 1: one job per bonus row (target row only), after the walk has listed them.
+// raw row(s) of one job -> shared memory
+template <bool BF16, bool UNC>
+__device__ __forceinline__ void topk_issue(const VerifyParams& P, int item, bool drafter, unsigned char* stage,
+                                           uint32_t rowbytes, unsigned long long* bar) {
+  const size_t esize = BF16 ? 2 : 4;
+  const size_t row = static_cast<size_t>(item) * P.V * esize;
+  uint64_t* b = reinterpret_cast<uint64_t*>(bar);
+  if (drafter) {
+    mbar_expect_tx(b, rowbytes);
+    bulk_load(stage, static_cast<const unsigned char*>(P.draft) + row, rowbytes, b);
+  } else {
+    const unsigned char* base = static_cast<const unsigned char*>(P.target);
+    const size_t branch = static_cast<size_t>(P.B) * P.R * P.V * esize;
+    mbar_expect_tx(b, UNC ? 2 * rowbytes : rowbytes);
+    bulk_load(stage, base + row, rowbytes, b);
+    if (UNC) bulk_load(stage + rowbytes, base + branch + row, rowbytes, b);
+  }
+}
+
+// staged raw row(s) -> keys of the processed logits
+template <bool BF16>
+__device__ __forceinline__ void topk_keys_from_stage(const unsigned char* stage, uint32_t rowbytes, bool unc, int V,
+                                                     float s, float T, uint32_t (&key)[TK_CH * 8]) {
+  const int tid = threadIdx.x;
+#pragma unroll
+  for (int c = 0; c < TK_CH; ++c) {
+    const int g = c * TKT + tid;
+    float lc[8], lu[8];
+    if (g * 8 < V) {
+      if (BF16) {
+        const uint4 x = *reinterpret_cast<const uint4*>(stage + static_cast<size_t>(g) * 16);
+        const uint32_t xw[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          lc[2 * i] = __uint_as_float(xw[i] << 16);
+          lc[2 * i + 1] = __uint_as_float(xw[i] & 0xffff0000u);
+        }
+        if (unc) {
+          const uint4 y = *reinterpret_cast<const uint4*>(stage + rowbytes + static_cast<size_t>(g) * 16);
+          const uint32_t yw[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            lu[2 * i] = __uint_as_float(yw[i] << 16);
+            lu[2 * i + 1] = __uint_as_float(yw[i] & 0xffff0000u);
+          }
+        }
+      } else {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const float4 x = *reinterpret_cast<const float4*>(stage + static_cast<size_t>(g) * 32 + h * 16);
+          lc[4 * h] = x.x, lc[4 * h + 1] = x.y, lc[4 * h + 2] = x.z, lc[4 * h + 3] = x.w;
+          if (unc) {
+            const float4 y = *reinterpret_cast<const float4*>(stage + rowbytes + static_cast<size_t>(g) * 32 + h * 16);
+            lu[4 * h] = y.x, lu[4 * h + 1] = y.y, lu[4 * h + 2] = y.z, lu[4 * h + 3] = y.w;
+          }
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        float z = unc ? __fmaf_rn(s, __fsub_rn(lc[e], lu[e]), lu[e]) : lc[e];
+        if (T != 1.0f) z = __fdiv_rn(z, T);
+        key[c * 8 + e] = topk_key(z);
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) key[c * 8 + e] = 0u;   // padding: below everything
+    }
+  }
+}
+
+// mode 0 (after the plan): per context with children, its target rows and -- in sampling -- its
+// drafter row, as separate jobs; mode 1 (after the walk): the target rows of the bonus draws.
 template <bool BF16, bool UNC>
 __global__ void __launch_bounds__(TKT, 2) lantern_topk_kernel(VerifyParams P, int mode) {
+  extern __shared__ __align__(128) unsigned char tsm[];
   __shared__ TopkShared S;
+  const int tid = threadIdx.x;
   const int V = P.V, R = P.R, K = P.top_k;
   const float T = P.T == 0.0f ? 1.0f : P.T;   // greedy decoding works at temperature 1
-  const size_t branch = static_cast<size_t>(P.B) * R * V;
+  const uint32_t rowbytes = static_cast<uint32_t>(V) * (BF16 ? 2 : 4);
+  const bool sampling = P.T != 0.0f;
+  const int n_heavy = P.counters->n_heavy;
+  const int cap = P.B * P.N;
+  const int per = (mode == 0 && sampling) ? 2 : 1;
+  const long long njobs = mode == 0 ? static_cast<long long>(n_heavy + P.counters->n_light) * per : P.counters->n_bonus;
+  const long long G = gridDim.x;
+  auto job_item = [&](long long j) -> int {
+    if (mode == 0) {
+      const int w = static_cast<int>(j / per);
+      return P.work[w < n_heavy ? w : cap - 1 - (w - n_heavy)].item;
+    }
+    return P.bonus_seq[j] * R + P.bonus_ctx[j];
+  };
+  auto job_is_drafter = [&](long long j) { return per == 2 && (j & 1); };
+  uint64_t* bar = reinterpret_cast<uint64_t*>(&S.bar_full);
+
+  long long j = blockIdx.x;
+  if (tid == 0) {
+    mbar_init(bar, 1);
+    fence_mbar_init();
+    if (j < njobs) topk_issue<BF16, UNC>(P, job_item(j), job_is_drafter(j), tsm, rowbytes, &S.bar_full);
+  }
+  __syncthreads();
+  if (j >= njobs) return;
+  int item = job_item(j);
   uint32_t key[TK_CH * 8];
-  if (mode == 0) {
-    const int n_heavy = P.counters->n_heavy;
-    const int total = n_heavy + P.counters->n_light;
-    const int cap = P.B * P.N;
-    for (int w = blockIdx.x; w < total; w += gridDim.x) {
-      const int item = P.work[w < n_heavy ? w : cap - 1 - (w - n_heavy)].item;
-      const size_t row = static_cast<size_t>(item) * V;
-      topk_load_keys<BF16, UNC>(P.target, row, branch, V, P.cfg_scale, T, key);
-      const float tq = topk_select(key, K, S);
-      if (threadIdx.x == 0) P.thr_q[item] = tq;
-      if (P.T != 0.0f) {   // sampling: the drafter row of the same context
-        topk_load_keys<BF16, false>(P.draft, row, 0, V, 1.0f, T, key);
-        const float tp = topk_select(key, K, S);
-        if (threadIdx.x == 0) P.thr_p[item] = tp;
+  for (uint32_t it = 0; j < njobs; j += G, ++it) {
+    const long long jn = j + G < njobs ? j + G : j;
+    const int item_next = job_item(jn);   // consumed after the keys are out: no select on it before
+    const bool drafter = job_is_drafter(j);
+    const bool landed = __syncthreads_and(mbar_wait(bar, it & 1) ? 1 : 0) != 0;
+    if (!landed) {   // the copy did not complete within the wait limit: no filter for this row, reported
+      if (tid == 0) {
+        (drafter ? P.thr_p : P.thr_q)[item] = __int_as_float(0xff800000);
+        if (mode == 0) atomicOr(&P.seq_status[item / R], LANTERN_ST_INTERNAL);
+        else if (P.out_status) atomicOr(&P.out_status[item / R], LANTERN_ST_INTERNAL);
       }
+      break;
     }
-  } else {
-    const int count = P.counters->n_bonus;
-    for (int i = blockIdx.x; i < count; i += gridDim.x) {
-      const int item = P.bonus_seq[i] * R + P.bonus_ctx[i];
-      topk_load_keys<BF16, UNC>(P.target, static_cast<size_t>(item) * V, branch, V, P.cfg_scale, T, key);
-      const float tq = topk_select(key, K, S);
-      if (threadIdx.x == 0) P.thr_q[item] = tq;
-    }
+    topk_keys_from_stage<BF16>(tsm, rowbytes, UNC && !drafter, V, P.cfg_scale, T, key);
+    __syncthreads();   // the staging area is free
+    if (tid == 0 && j + G < njobs)
+      topk_issue<BF16, UNC>(P, item_next, job_is_drafter(j + G), tsm, rowbytes, &S.bar_full);
+    const float t = topk_select(key, K, S);
+    if (tid == 0) (drafter ? P.thr_p : P.thr_q)[item] = t;
+    item = item_next;
   }
 }
 

@@ -210,3 +210,22 @@ def verify_greedy(target_logits: np.ndarray, dtype: int, cfg_scale: float, has_u
     if rc != 0:
         raise ValueError(f"oracle_verify_greedy: bad arguments ({rc})")
     return res
+
+
+def aggregate_all(rows_c: np.ndarray, rows_u: Optional[np.ndarray], dtype: int, cfg_scale: float, T: float,
+                  neighbor_idx: np.ndarray, delta: float):
+    """agg[r, x] = sum of row r's distribution over A_{k,delta}(x), for every token x (a benchmark of the
+    V x k gather-sum; the paper's method needs it for the drafted tokens only).  Returns (agg, m, margin)."""
+    rc_ = np.ascontiguousarray(rows_c)
+    ru_ = None if rows_u is None else np.ascontiguousarray(rows_u)
+    rows, V = rc_.shape
+    nb = np.ascontiguousarray(neighbor_idx, dtype=np.int32)
+    agg = np.empty((rows, V), np.float64)
+    m = np.empty((rows, V), np.int32)
+    margin = np.empty((rows, V), np.float64)
+    rc = _load().oracle_aggregate_all(_p(rc_), _p(ru_), int(dtype), int(ru_ is not None), ctypes.c_float(cfg_scale),
+                                      ctypes.c_float(T), _p(nb), int(nb.shape[1]), ctypes.c_float(delta), rows, V,
+                                      _p(agg), _p(m), _p(margin))
+    if rc != 0:
+        raise ValueError(f"oracle_aggregate_all failed ({rc})")
+    return agg, m, margin

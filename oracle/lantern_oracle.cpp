@@ -686,4 +686,41 @@ int oracle_verify_greedy(const void* target_logits, int dtype, float cfg_scale, 
                                  out_accept_path, out_status, tr_tested, tr_qa, tr_m, tr_margin);
 }
 
+// ---------------------------------------------------------------------------------------
+// All-token aggregation (not part of the paper's method: a benchmark of the V x k gather-sum
+// that building A_{k,delta}(x) for EVERY token x of a row amounts to; the verification step
+// only ever needs it for the drafted tokens).  For one context row with distribution q:
+//     agg[x] = sum_{y in A_{k,delta}(x)} q(y),   m[x] = |A_{k,delta}(x)| - 1,
+// with A_{k,delta}(x) built exactly as in Algorithm 2's second block (oracle_a_set).
+// rows_c / rows_u: [rows, V] logits; agg [rows, V] double; m [rows, V] int32 (may be null);
+// margin [rows, V] double: distance of each cut to flipping (may be null).
+// ---------------------------------------------------------------------------------------
+int oracle_aggregate_all(const void* rows_c, const void* rows_u, int dtype, int has_uncond, float cfg_scale,
+                         float T, const int32_t* neighbor_idx, int k, float delta_f, int rows, int V, double* agg,
+                         int32_t* m_out, double* margin) {
+  if (rows < 0 || V < 1 || k < 1 || k > V || !(T > 0.0f) || !(delta_f >= 0.0f)) return -2;
+  if (rows == 0) return 0;
+  if (!rows_c || !neighbor_idx || !agg || (has_uncond && !rows_u)) return -1;
+  const double delta = static_cast<double>(delta_f);
+  std::vector<float> z(V);
+  std::vector<double> q;
+  for (int r = 0; r < rows; ++r) {
+    const size_t off = static_cast<size_t>(r) * V;
+    for (int x = 0; x < V; ++x) {
+      float lc = load_logit(rows_c, dtype, off + x);
+      float lu = has_uncond ? load_logit(rows_u, dtype, off + x) : 0.0f;
+      z[x] = target_z(lc, lu, has_uncond, cfg_scale, T);
+    }
+    if (!softmax(z, q, nullptr)) return -4;
+    for (int x = 0; x < V; ++x) {
+      double moved = 0.0, cm = 0.0;
+      const int m = oracle_a_set(q.data(), V, neighbor_idx + static_cast<size_t>(x) * k, k, delta, &moved, &cm, nullptr);
+      agg[off + x] = q[x] + moved;
+      if (m_out) m_out[off + x] = m;
+      if (margin) margin[off + x] = k > 1 ? cm : std::numeric_limits<double>::infinity();
+    }
+  }
+  return 0;
+}
+
 }  // extern "C"

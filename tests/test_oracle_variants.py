@@ -255,3 +255,37 @@ def test_top_k_plain_speculative_sampling_keeps_the_filtered_target():
     keep = q > 0
     chi2 = ((counts[keep] - trials * q[keep]) ** 2 / (trials * q[keep])).sum()
     assert chi2 < 30.0          # 4 degrees of freedom (5 kept tokens): P(chi2 > 30) < 1e-5
+
+
+# ------------------------------------------------------------------------------------ all-token aggregation
+def test_aggregate_all():
+    """agg[x] = sum_{A_{k,delta}(x)} q: delta >= 1 is a product with B_k's 0/1 matrix, delta = 0 and k = 1
+    give q itself, and every entry equals a numpy prefix sum cut at the bound."""
+    V, k, rows = 200, 12, 5
+    table = oracle.build_neighbors(li.codebook_gaussian(V, 4, seed=9), k)[0]
+    inp = li.verify_inputs(rows, 0, V, dtype=li.BF16, has_uncond=True, cfg_scale=2.0, sigma_target=1.0,
+                           sigma_draft=1.0, rho=0.5, seed=4)
+    rc, ru = inp.target_logits[0, :, 0], inp.target_logits[1, :, 0]
+    q = np.stack([oracle.row_distribution(rc[r], ru[r], li.BF16, 2.0, 1.0) for r in range(rows)])
+    adj = np.zeros((V, V))
+    adj[np.arange(V)[:, None], table] = 1.0
+    agg, m, _ = oracle.aggregate_all(rc, ru, li.BF16, 2.0, 1.0, table, 1.5)
+    assert np.abs(agg - q @ adj.T).max() < 1e-14 and np.all(m == k - 1)
+    agg0, m0, _ = oracle.aggregate_all(rc, ru, li.BF16, 2.0, 1.0, table, 0.0)
+    assert np.array_equal(agg0, q) and not m0.any()
+    agg1, _, _ = oracle.aggregate_all(rc, ru, li.BF16, 2.0, 1.0, table[:, :1], 0.3)
+    assert np.array_equal(agg1, q)
+    delta = 0.05
+    agg, m, margin = oracle.aggregate_all(rc, ru, li.BF16, 2.0, 1.0, table, delta)
+    cut = 0
+    for r in range(rows):
+        for x in range(V):
+            cs = np.cumsum(q[r, table[x, 1:]])
+            fits = cs < np.float32(delta)
+            want = k - 1 if fits.all() else int(np.argmin(fits))
+            if margin[r, x] > 1e-12:
+                assert m[r, x] == want
+                assert abs(agg[r, x] - (q[r, x] + (cs[want - 1] if want else 0.0))) < 1e-15
+            cut += want < k - 1
+    assert cut > rows * V // 10
+    assert np.all(oracle.aggregate_all(rc, ru, li.BF16, 2.0, 1.0, table, 0.2)[0] >= agg - 1e-15)

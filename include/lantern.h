@@ -196,6 +196,27 @@ lantern_status lantern_verify_ex(const void* target_logits, const void* draft_lo
                                  size_t workspace_bytes, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
+ * All-token aggregation: for every token x of every given context row,
+ *     out_agg[r, x] = sum_{y in A_{k,delta}(x)} q_r(y),   out_m[r, x] = |A_{k,delta}(x)| - 1,
+ * with q_r the row's target distribution (guidance and temperature as in lantern_verify) and
+ * A_{k,delta}(x) grown as in Algorithm 2's second block (TVD bound).  The paper's method never
+ * needs this for more than the drafted tokens -- lantern_verify does not use it; the entry point
+ * exists to measure the V x k gather-sum that the full aggregation amounts to.
+ *
+ *   logits        [C, rows, V], C = 2 (conditional, unconditional) if has_uncond else 1; 16-byte aligned
+ *   neighbor_idx  [V, k] int32 as written by lantern_build_neighbors; 16-byte aligned
+ *   rows, V, k    rows >= 0; V a multiple of 8, 8 <= V <= 16384; 1 <= k <= V
+ *   T, delta      T > 0; delta >= 0
+ *   out_agg       [rows, V] fp32 (NaN for a row with a NaN / +inf logit or no finite logit)
+ *   out_m         [rows, V] int32, may be NULL (-1 for such a row)
+ *   out_status    [rows] LANTERN_ST_NONFINITE / LANTERN_ST_BAD_TABLE bits, may be NULL
+ * No workspace.  Asynchronous on cuda_stream.
+ * ---------------------------------------------------------------------------------------- */
+lantern_status lantern_aggregate_all(const void* logits, int dtype, float cfg_scale, int has_uncond, float T,
+                                     const int32_t* neighbor_idx, int k, float delta, int rows, int V,
+                                     float* out_agg, int32_t* out_m, int32_t* out_status, void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
  * lantern_verify without a caller-supplied workspace.  (The paper has no counterpart: this
  * entry point exists for integration reasons only and computes exactly what lantern_verify
  * computes.)

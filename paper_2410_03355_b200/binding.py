@@ -57,6 +57,8 @@ def load_library():
     lib.lantern_build_neighbors_metric.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, sz, vp]
     lib.lantern_verify_workspace_bytes_ex.restype = sz
     lib.lantern_verify_workspace_bytes_ex.argtypes = [i32, i32, i32]
+    lib.lantern_aggregate_all.restype = i32
+    lib.lantern_aggregate_all.argtypes = [vp, i32, f32, i32, f32, vp, i32, f32, i32, i32, vp, vp, vp, vp]
     lib.lantern_verify_ex.restype = i32
     lib.lantern_verify_ex.argtypes = [vp, vp, i32, f32, i32, f32, vp, vp, vp, i32, f32, i32, i32, vp, i32, i32, i32,
                                       vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -198,6 +200,30 @@ def verify(target_logits: torch.Tensor, draft_logits: Optional[torch.Tensor], cf
     if rc != 0:
         raise LanternError(rc, "lantern_verify_ex")
     return out
+
+
+def aggregate_all(logits: torch.Tensor, cfg_scale: float, T: float, neighbor_idx: torch.Tensor, delta: float, *,
+                  with_m: bool = True, stream: Optional[torch.cuda.Stream] = None):
+    """lantern_aggregate_all: logits [C, rows, V] -> (agg [rows, V] fp32, m [rows, V] int32 or None, status [rows]).
+    A benchmark of the V x k gather-sum (the mass of A_{k,delta}(x) for every token x); verify() does not use it."""
+    lib = load_library()
+    C, rows, V = logits.shape
+    if C not in (1, 2):
+        raise ValueError("logits must have 1 or 2 guidance branches")
+    dtype = BF16 if logits.dtype == torch.bfloat16 else F32
+    if logits.dtype not in (torch.bfloat16, torch.float32):
+        raise ValueError("logits must be float32 or bfloat16")
+    dev = logits.device
+    with torch.cuda.device(dev):
+        agg = torch.empty((rows, V), dtype=torch.float32, device=dev)
+        m = torch.empty((rows, V), dtype=torch.int32, device=dev) if with_m else None
+        status = torch.empty(rows, dtype=torch.int32, device=dev)
+        rc = lib.lantern_aggregate_all(_ptr(logits, None, "logits"), dtype, float(cfg_scale), int(C == 2), float(T),
+                                       _ptr(neighbor_idx, torch.int32, "neighbor_idx"), int(neighbor_idx.shape[1]),
+                                       float(delta), rows, V, _ptr(agg), _ptr(m), _ptr(status), _stream_ptr(stream))
+    if rc != 0:
+        raise LanternError(rc, "lantern_aggregate_all")
+    return agg, m, status
 
 
 def verify_launch_count() -> int:

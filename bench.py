@@ -251,6 +251,57 @@ def run_reference(args, rank, world):
     print(json.dumps(line), flush=True)
 
 
+def run_aggregate(args):
+    """Side benchmark (not the headline metric): lantern_aggregate_all on `--aggregate-rows` root-context rows
+    of the workload.  Every row re-reads the whole neighbour table (V * k * 4 bytes), which lives in L2."""
+    import torch
+
+    import lantern_inputs as li
+    import lantern_inputs.device as lid
+    import oracle
+    import paper_2410_03355_b200 as lt
+    torch.cuda.set_device(0)
+    w = WORKLOADS[args.workload]
+    cfg = li.CONFIGS[w["config"]]
+    V, k, delta = cfg["V"], cfg["k"], cfg["delta"]
+    rows = args.aggregate_rows
+    cb = torch.from_numpy(li.config_codebook(w["config"])).cuda()
+    table, _ = lt.build_neighbors(cb, k, with_dist=False, metric=args.metric)
+    d = lid.config_verify_inputs_device(w["config"], B=rows, seed=li.BASE_SEED)
+    logits = d["target_logits"][:, :, 0].contiguous()            # [C, rows, V]: the root contexts
+    for _ in range(max(args.warmup, 3)):
+        lt.aggregate_all(logits, d["cfg_scale"], d["T"], table, delta, with_m=False)
+    torch.cuda.synchronize()
+    a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    steps = min(args.steps, 20)
+    a.record()
+    for _ in range(steps):
+        agg, _, status = lt.aggregate_all(logits, d["cfg_scale"], d["T"], table, delta, with_m=False)
+    b_.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b_) / steps
+    t0 = time.perf_counter()
+    host = logits[:, :1].cpu()
+    hl = host.view(torch.int16).numpy().view(np.uint16) if cfg["dtype"] == li.BF16 else host.numpy()
+    oracle.aggregate_all(hl[0], hl[1] if cfg["has_uncond"] else None, cfg["dtype"], d["cfg_scale"], d["T"],
+                         table.cpu().numpy(), delta)
+    cpu_s = time.perf_counter() - t0
+    table_bytes = rows * V * k * 4
+    print(json.dumps({
+        "metric": "all_token_aggregation_rows_per_s", "value": rows / (ms * 1e-3), "unit": "rows/s", "n_gpus": 1,
+        "steps": steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "data": "synthetic",
+        "dtype": "f32", "config": {"workload": args.workload, "rows": rows, "V": V, "k": k, "delta": delta,
+                                   "note": "side benchmark of the V x k gather-sum; not used by verification"},
+        "roofline": {"bound": "l2", "kernel": "lantern_aggregate_kernel", "achieved": table_bytes / (ms * 1e-3) / 1e9,
+                     "peak": None, "unit": "GB/s", "frac": None, "traffic": None,
+                     "note": "achieved = neighbour-table bytes read per second (from L2); no measured L2 peak on file",
+                     "gathers_per_s": rows * V * k / (ms * 1e-3)},
+        "cpu_baseline": {"value": 1.0 / cpu_s, "unit": "rows/s", "cores": 1, "kind": "oracle", "sample": "1 row"},
+        "gpu_launches": steps, "outputs": {"rows_with_status_bits": int((status != 0).sum().item()),
+                                           "mean_aggregated_mass": float(agg.mean().item() * V)},
+    }), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -268,6 +319,8 @@ def main():
     ap.add_argument("--metric", default="l2", choices=["l2", "cosine"], help="latent proximity of the table")
     ap.add_argument("--top-k", type=int, default=0, dest="top_k",
                     help="top-k logit filter of the generation settings (Appendix B.2); 0 = off")
+    ap.add_argument("--aggregate-rows", type=int, default=0, dest="aggregate_rows",
+                    help="run the all-token aggregation side benchmark on this many rows instead of verification")
     ap.add_argument("--greedy", action="store_true",
                     help="run the workload at T = 0 (greedy decoding: no drafter rows, no random numbers)")
     args = ap.parse_args()
@@ -279,6 +332,10 @@ def main():
 
     if args.impl == "reference":
         run_reference(args, rank, world)
+        return
+    if args.aggregate_rows > 0:
+        if rank == 0:
+            run_aggregate(args)
         return
 
     import torch

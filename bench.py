@@ -493,7 +493,8 @@ def main():
             "roofline": {"bound": "hbm", "kernel": "lantern_greedy_context_kernel" if args.greedy else "lantern_context_kernel",
                          "achieved": achieved, "peak": peak,
                          "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None if args.greedy else ncu_traffic(args.workload, cfg, alg_bytes),
+                         "traffic": None if (args.greedy or args.divergence != "tvd" or 0 < args.top_k < V) else
+                                    ncu_traffic(args.workload, cfg, alg_bytes),
                          "algorithmic_bytes_per_launch": int(alg_bytes), "kernel_ms": fused_ms},
             "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": (4 + (0 if not 0 < args.top_k < V else (1 if args.greedy else 2))) * args.steps, "clocks": clocks,

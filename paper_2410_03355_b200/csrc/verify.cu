@@ -161,7 +161,7 @@ __global__ void __launch_bounds__(128) lantern_walk_kernel(VerifyParams P) {
 // (Algorithm 1, line after the verification loop)
 // ---------------------------------------------------------------------------------------
 template <int CH, bool BF16, bool UNC, bool TOPK>
-__global__ void __launch_bounds__(NT, 1) lantern_bonus_kernel(VerifyParams P) {
+__global__ void __launch_bounds__(NT, 2) lantern_bonus_kernel(VerifyParams P) {
   __shared__ BlockScratch S;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int V = P.V, R = P.R, N = P.N;
@@ -517,7 +517,7 @@ static lantern_status verify_impl(const void* target_logits, const void* draft_l
   const long long items = static_cast<long long>(B) * (N > 0 ? N : 1);   // upper bound of contexts with children
   const long long ctas = (items + NGRP - 1) / NGRP;   // every CTA runs NGRP contexts at a time
   const int grid_ctx = static_cast<int>(ctas < sms ? ctas : sms);
-  const int grid_bonus = B < sms ? B : sms;
+  const int grid_bonus = B < 2 * sms ? B : 2 * sms;   // two 1024-thread CTAs fit an SM
   cudaError_t e;
   const bool bf = dtype == LANTERN_BF16, un = has_uncond != 0;
   if (greedy) {

@@ -73,3 +73,29 @@ def test_bench_sized_call_against_sampled_oracle(workload, sample):
     torch.cuda.synchronize()
     assert torch.equal(out.accept_len, out2.accept_len) and torch.equal(out.next_token, out2.next_token)
     assert torch.equal(out.accept_path, out2.accept_path)
+
+
+@pytest.mark.parametrize("workload,sample,divergence,top_k", [
+    ("batch_chain", 64, oracle.DIV_JSD, 0),
+    ("batch_chain", 64, oracle.DIV_TVD, 1000),       # Appendix B.2's text-conditional setting
+    ("stress", 48, oracle.DIV_JSD, 2000),
+])
+def test_bench_sized_variants_against_sampled_oracle(workload, sample, divergence, top_k):
+    """The calls `bench.py --divergence jsd` / `--top-k K` time, checked on a seeded sample of their sequences."""
+    import bench
+    from parity import DIV_NAME
+    w = bench.WORKLOADS[workload]
+    cfg = li.CONFIGS[w["config"]]
+    B, N, V, delta = w["B"], cfg["N"], cfg["V"], cfg["delta"]
+    table = _table(w["config"])
+    d = lid.config_verify_inputs_device(w["config"], B=B, seed=bench.rank_seed(li.BASE_SEED, 0))
+    out = lt.verify(d["target_logits"], d["draft_logits"], d["cfg_scale"], d["T"], d["draft_tokens"],
+                    d["tree_parents"], table, delta, d["uniforms"], trace=True, divergence=DIV_NAME[divergence],
+                    top_k=top_k)
+    torch.cuda.synchronize()
+    _properties(d, out, N, V)
+    rows = np.sort(np.random.default_rng(13).choice(B, size=min(sample, B), replace=False))
+    host = lid.to_host(d, rows=rows)
+    res = compare(host, table.cpu().numpy(), delta, _take(out, rows), divergence=divergence, top_k=top_k)
+    assert_parity(res)
+    assert res["nodes_tested"] >= len(rows)

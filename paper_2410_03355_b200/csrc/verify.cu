@@ -116,6 +116,7 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
 #include "verify_context.cuh"
 // greedy decoding (temperature 0)
 #include "verify_greedy.cuh"
+#include "verify_bonus.cuh"
 #include "verify_topk.cuh"
 
 namespace lantern {
@@ -154,100 +155,6 @@ __global__ void __launch_bounds__(128) lantern_walk_kernel(VerifyParams P) {
   P.out_len[b] = len;
   P.out_tok[b] = next;
   if (P.out_status) P.out_status[b] = status;
-}
-
-// ---------------------------------------------------------------------------------------
-// kernel 4: bonus token ~ q at the context where the walk ran out of drafts
-// (Algorithm 1, line after the verification loop)
-// ---------------------------------------------------------------------------------------
-template <int CH, bool BF16, bool UNC, bool TOPK>
-__global__ void __launch_bounds__(NT, 2) lantern_bonus_kernel(VerifyParams P) {
-  __shared__ BlockScratch S;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int V = P.V, R = P.R, N = P.N;
-  const int rowbytes = V * (BF16 ? 2 : 4);
-  const int count = P.counters->n_bonus;
-  for (int i = blockIdx.x; i < count; i += gridDim.x) {
-    const int b = P.bonus_seq[i], ctx = P.bonus_ctx[i];
-    const size_t row_off = (static_cast<size_t>(b) * R + ctx) * rowbytes;
-    const size_t branch = static_cast<size_t>(P.B) * R * rowbytes;
-    const unsigned char* rc = static_cast<const unsigned char*>(P.target) + row_off;
-    const unsigned char* ru = rc + branch;
-    float a[CH * 8];
-    const float ninf = __int_as_float(0xff800000);
-    float tq = ninf;   // top-k filter, if any
-    if (TOPK) tq = __ldg(P.thr_q + static_cast<size_t>(b) * R + ctx);
-#pragma unroll
-    for (int c = 0; c < CH; ++c) {
-      const int g = c * NT + tid;
-      float lc[8], lu[8];
-      if (g * 8 < V) {
-        if (BF16) {
-          const uint4 x = __ldg(reinterpret_cast<const uint4*>(rc + g * 16));
-          const uint32_t xw[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            lc[2 * j] = __uint_as_float(xw[j] << 16);
-            lc[2 * j + 1] = __uint_as_float(xw[j] & 0xffff0000u);
-          }
-          if (UNC) {
-            const uint4 y = __ldg(reinterpret_cast<const uint4*>(ru + g * 16));
-            const uint32_t yw[4] = {y.x, y.y, y.z, y.w};
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              lu[2 * j] = __uint_as_float(yw[j] << 16);
-              lu[2 * j + 1] = __uint_as_float(yw[j] & 0xffff0000u);
-            }
-          }
-        } else {
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            const float4 x = __ldg(reinterpret_cast<const float4*>(rc + g * 32 + h * 16));
-            lc[4 * h] = x.x, lc[4 * h + 1] = x.y, lc[4 * h + 2] = x.z, lc[4 * h + 3] = x.w;
-            if (UNC) {
-              const float4 y = __ldg(reinterpret_cast<const float4*>(ru + g * 32 + h * 16));
-              lu[4 * h] = y.x, lu[4 * h + 1] = y.y, lu[4 * h + 2] = y.z, lu[4 * h + 3] = y.w;
-            }
-          }
-        }
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          float l = lc[e];
-          if (UNC) l = __fmaf_rn(P.cfg_scale, __fsub_rn(lc[e], lu[e]), lu[e]);
-          if (P.T != 1.0f) l = __fdiv_rn(l, P.T);
-          a[c * 8 + e] = (TOPK && l < tq) ? ninf : l;
-        }
-      } else {
-#pragma unroll
-        for (int e = 0; e < 8; ++e) a[c * 8 + e] = ninf;
-      }
-    }
-    float mq = a[0], dummy = 0.0f;
-#pragma unroll
-    for (int j = 1; j < CH * 8; ++j) mq = fmaxf(mq, a[j]);
-    block_max2(mq, dummy, S, lane, warp);
-    double cs[CH], excl[CH];
-#pragma unroll
-    for (int c = 0; c < CH; ++c) {
-#pragma unroll
-      for (int e = 0; e < 8; ++e) a[c * 8 + e] = exp_nonpos(a[c * 8 + e] - mq);
-      cs[c] = static_cast<double>(sum8(&a[c * 8]));
-    }
-    block_scan_chunks<CH>(cs, excl, 0.0, S, lane, warp);
-    const double Z = S.total;
-    int tok = -1, st = 0;
-    if (Z > 0.0 && Z < 1e300) {
-      const double u = static_cast<double>(P.uniforms[static_cast<size_t>(b) * R + N]);
-      tok = block_draw<CH>(a, cs, excl, u * Z, V, S, tid);
-    } else {
-      st = LANTERN_ST_NONFINITE;
-    }
-    if (tid == 0) {
-      P.out_tok[b] = tok;
-      if (st && P.out_status) P.out_status[b] |= st;
-    }
-    __syncthreads();
-  }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -317,9 +224,25 @@ cudaError_t launch_context_kernel(const VerifyParams& P, int CH, bool bf16, bool
   }
 }
 
-template <int CHB, bool BF16, bool UNC, bool TOPK>
+template <bool BF16, bool UNC, bool TOPK>
+static cudaError_t launch_bonus(const VerifyParams& P, int sms, cudaStream_t st) {
+  auto kb = lantern_bonus_stream_kernel<BF16, UNC, TOPK>;
+  const size_t smem = static_cast<size_t>(P.V) * (UNC ? 2 : 1) * (BF16 ? 2 : 4);   // one context's raw target rows
+  cudaError_t e = cudaFuncSetAttribute(kb, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
+  int per_sm = 0;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kb, BNT, smem);
+  if (e != cudaSuccess) return e;
+  if (per_sm < 1) return cudaErrorInvalidConfiguration;
+  const long long slots = static_cast<long long>(sms) * per_sm;
+  const int grid = static_cast<int>(P.B < slots ? P.B : slots);
+  kb<<<grid, BNT, smem, st>>>(P);
+  return cudaGetLastError();
+}
+
+template <bool BF16, bool UNC, bool TOPK>
 static cudaError_t launch_verify(const VerifyParams& P, int CH, bool tone, bool jsd, long long items, int sms,
-                                 int grid_ctx, int grid_bonus, size_t smem_bytes, cudaStream_t st) {
+                                 int grid_ctx, size_t smem_bytes, cudaStream_t st) {
   cudaError_t e;
   if (TOPK) {
     e = launch_topk<BF16, UNC>(P, 0, 2 * items, sms, st);
@@ -336,8 +259,7 @@ static cudaError_t launch_verify(const VerifyParams& P, int CH, bool tone, bool 
     e = launch_topk<BF16, UNC>(P, 1, P.B, sms, st);
     if (e != cudaSuccess) return e;
   }
-  lantern_bonus_kernel<CHB, BF16, UNC, TOPK><<<grid_bonus, NT, 0, st>>>(P);   // CHB: 1024 threads per row
-  return cudaGetLastError();
+  return launch_bonus<BF16, UNC, TOPK>(P, sms, st);
 }
 
 template <bool BF16, bool UNC, bool TOPK>
@@ -517,7 +439,7 @@ static lantern_status verify_impl(const void* target_logits, const void* draft_l
   const long long items = static_cast<long long>(B) * (N > 0 ? N : 1);   // upper bound of contexts with children
   const long long ctas = (items + NGRP - 1) / NGRP;   // every CTA runs NGRP contexts at a time
   const int grid_ctx = static_cast<int>(ctas < sms ? ctas : sms);
-  const int grid_bonus = B < 2 * sms ? B : 2 * sms;   // two 1024-thread CTAs fit an SM
+  const int grid_bonus = B < 4 * sms ? B : 4 * sms;   // greedy bonus: 256-thread CTAs
   cudaError_t e;
   const bool bf = dtype == LANTERN_BF16, un = has_uncond != 0;
   if (greedy) {
@@ -530,15 +452,13 @@ static lantern_status verify_impl(const void* target_logits, const void* draft_l
   }
   // every combination of the compile-time variants exists: T = 1 never meets the division code
   const bool tone = T == 1.0f, jsd = divergence == LANTERN_DIV_JSD;
-#define LANTERN_DISPATCH2(CHB, KV)                                                                              \
-  (bf ? (un ? launch_verify<CHB, true, true, KV>(P, CH, tone, jsd, items, sms, grid_ctx, grid_bonus, smem_bytes, st)   \
-            : launch_verify<CHB, true, false, KV>(P, CH, tone, jsd, items, sms, grid_ctx, grid_bonus, smem_bytes, st)) \
-      : (un ? launch_verify<CHB, false, true, KV>(P, CH, tone, jsd, items, sms, grid_ctx, grid_bonus, smem_bytes, st)  \
-            : launch_verify<CHB, false, false, KV>(P, CH, tone, jsd, items, sms, grid_ctx, grid_bonus, smem_bytes, st)))
-#define LANTERN_DISPATCH(CHB) (topk ? LANTERN_DISPATCH2(CHB, true) : LANTERN_DISPATCH2(CHB, false))
-  e = CH == 8 ? LANTERN_DISPATCH(2) : LANTERN_DISPATCH(1);
+#define LANTERN_DISPATCH2(KV)                                                                        \
+  (bf ? (un ? launch_verify<true, true, KV>(P, CH, tone, jsd, items, sms, grid_ctx, smem_bytes, st)   \
+            : launch_verify<true, false, KV>(P, CH, tone, jsd, items, sms, grid_ctx, smem_bytes, st)) \
+      : (un ? launch_verify<false, true, KV>(P, CH, tone, jsd, items, sms, grid_ctx, smem_bytes, st)  \
+            : launch_verify<false, false, KV>(P, CH, tone, jsd, items, sms, grid_ctx, smem_bytes, st)))
+  e = topk ? LANTERN_DISPATCH2(true) : LANTERN_DISPATCH2(false);
 #undef LANTERN_DISPATCH2
-#undef LANTERN_DISPATCH
   return e == cudaSuccess ? LANTERN_OK : LANTERN_E_CUDA;
 }
 

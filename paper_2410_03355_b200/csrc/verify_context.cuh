@@ -25,7 +25,7 @@
 // inverse-CDF draw or the write-back for the next sibling.
 #pragma once
 
-#define LANTERN_CONTEXT_KERNEL_REVISION 12   // bump on every change to this file
+#define LANTERN_CONTEXT_KERNEL_REVISION 13   // bump on every change to this file
 
 namespace lantern {
 
@@ -563,8 +563,10 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
     if (!(Zq > 0.0 && Zq < 1e300 && Zp > 0.0 && Zp < 1e300)) {
       status |= LANTERN_ST_NONFINITE;
     } else {
-      double qscale = 1.0 / Zq;     // q'(x) = E(x) * fq[slice of x] * qscale
-      double pscale = 1.0 / Zp;     // p'(x) = ep(x) * fp[slice of x] * pscale
+      // current normalisers: q'(x) = E(x) * fq[slice of x] / Zq_c,  p'(x) = ep(x) * fp[slice of x] / Zp_c
+      // (Zp_c = 0 stands for a drafter distribution that has no mass left).  Comparisons are written on
+      // the unnormalised sums, so that no thread divides on the way to a decision.
+      double Zq_c = Zq, Zp_c = Zp;
       const double delta = static_cast<double>(P.delta);
       if (gt == 0) {   // the two single probabilities of the first child, in double precision
         float zq = raw_c;
@@ -602,11 +604,11 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
         }
 
         // ---- A_{k,delta}(x~): gather + prefix scan with the strict bound ----
-        double thr = delta / qscale;   // the bound in the units of the unnormalised sums
+        double thr = delta * Zq_c;   // the bound in the units of the unnormalised sums
         // Section 6.2.2: the mass whose JSD is delta; one thread, published by [scan 1] through the last
         // slot of wt[], which nothing else touches between the start of a child and its [scan 2]
         if (JSD && gt == GT - 32)
-          S.wt[8 * GW - 1] = jsd_mass_bound(delta, static_cast<double>(e_xt_bulk) * qscale) / qscale;
+          S.wt[8 * GW - 1] = jsd_mass_bound(delta, static_cast<double>(e_xt_bulk) / Zq_c) * Zq_c;
         double carry = 0.0, sm = 0.0;
         int m = k - 1;
         bool cut = false;
@@ -678,13 +680,13 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
         const bool acc = S.acc_valid != 0;
         const double e_xt = (acc && e_xt_bulk != 0.0f) ? S.acc_e : static_cast<double>(e_xt_bulk);
         const double p_xt = (acc && px_bulk != 0.0f) ? S.acc_p : static_cast<double>(px_bulk);
-        const double qa = (e_xt + sm) * qscale;
-        const double px = p_xt * pscale;
-        const bool accept = static_cast<double>(r) * px < qa;   // Section 4.3: min(1, sum_A q / p(x~))
-        if (gt == 0) {
+        // Section 4.3: accept iff r p(x~) < sum_A q, i.e. r p_xt / Zp_c < (e_xt + sm) / Zq_c, both sides times Zq_c Zp_c
+        const double qa_un = e_xt + sm;
+        const bool accept = Zp_c > 0.0 ? static_cast<double>(r) * p_xt * Zq_c < qa_un * Zp_c : 0.0 < qa_un;
+        if (gt == 0 && (P.out_qa || P.out_px || P.out_m)) {
           const size_t o = static_cast<size_t>(b) * N + node;
-          if (P.out_qa) P.out_qa[o] = static_cast<float>(qa);
-          if (P.out_px) P.out_px[o] = static_cast<float>(px);
+          if (P.out_qa) P.out_qa[o] = static_cast<float>(qa_un / Zq_c);
+          if (P.out_px) P.out_px[o] = Zp_c > 0.0 ? static_cast<float>(p_xt / Zp_c) : 0.0f;
           if (P.out_m) P.out_m[o] = m;
         }
         if (accept) {
@@ -729,7 +731,7 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
         gbar(grp);   // [flags]
         // w = E - (p'/q' scale ratio) * ep in common units, i.e. E - ratio * ep in the slice's own units
         // of E; the residual replaces E (it is the next sibling's target, or what the draw reads)
-        const float ratio_g = static_cast<float>(pscale / qscale);
+        const float ratio_g = Zp_c > 0.0 ? static_cast<float>(Zq_c / Zp_c) : 0.0f;
         float cs[CH];
         double wsum = 0.0, psum = 0.0;
 #pragma unroll
@@ -812,8 +814,8 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
               S.acc_valid = 0;
             }
           }
-          qscale = 1.0 / W;
-          pscale = Sp > 0.0 ? 1.0 / Sp : 0.0;
+          Zq_c = W;
+          Zp_c = Sp > 0.0 ? Sp : 0.0;
           continue;
         }
         // ---- last child rejected: draw the replacement token from the residual (Algorithm 1) ----

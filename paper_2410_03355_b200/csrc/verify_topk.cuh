@@ -25,12 +25,15 @@ constexpr int TKT = 256;
 constexpr int TKW = TKT / 32;
 constexpr int TK_CH = 8;            // 8-token chunks per thread: 8 * 8 * 256 = 16384 tokens at most
 constexpr int TK_LIST = 128;
+constexpr int TK_CE = 16;           // candidate keys per thread after the pre-filter
+constexpr int TK_CAND = TK_CE * 256;
 constexpr uint32_t TK_KEY_NINF = 0x007fffffu;
 
 struct TopkShared {
   int cnt[2][TKW];
   unsigned kmin[TKW], kmax[TKW];
   __align__(16) unsigned list[TK_LIST];
+  unsigned cand[TK_CAND];           // keys that passed the pre-filter
   int list_n;
   unsigned result;
   unsigned long long bar_full;
@@ -47,16 +50,15 @@ __device__ __forceinline__ float topk_value(uint32_t key) {
 }
 
 // number of this thread's keys >= t, summed over the block (every thread gets the sum)
-__device__ __forceinline__ int topk_count(const uint32_t (&key)[TK_CH * 8], uint32_t t, TopkShared& S, int& flip) {
-  int c0 = 0, c1 = 0, c2 = 0, c3 = 0;   // four chains: the adds do not wait for one another
+template <int NE>
+__device__ __forceinline__ int topk_count(const uint32_t (&key)[NE], uint32_t t, TopkShared& S, int& flip) {
+  int c0 = 0, c1 = 0;   // two chains: the adds do not wait for one another
 #pragma unroll
-  for (int i = 0; i < TK_CH * 8; i += 4) {
+  for (int i = 0; i < NE; i += 2) {
     c0 += key[i] >= t;
     c1 += key[i + 1] >= t;
-    c2 += key[i + 2] >= t;
-    c3 += key[i + 3] >= t;
   }
-  const int c = __reduce_add_sync(kFull, (c0 + c1) + (c2 + c3));
+  const int c = __reduce_add_sync(kFull, c0 + c1);
   if ((threadIdx.x & 31) == 0) S.cnt[flip][threadIdx.x >> 5] = c;
   __syncthreads();
   int tot = 0;
@@ -119,15 +121,16 @@ __device__ __forceinline__ void topk_load_keys(const void* logits, size_t row_el
   }
 }
 
-// value of the K-th largest key held by the block (-inf if fewer than K keys lie above -inf)
-__device__ __forceinline__ float topk_select(const uint32_t (&key)[TK_CH * 8], int K, TopkShared& S) {
+// K-th largest of the block's keys, NE per thread (the key of -inf if fewer than K keys lie above -inf)
+template <int NE>
+__device__ __forceinline__ uint32_t topk_select_keys(const uint32_t (&key)[NE], int K, TopkShared& S) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float NEG_INF = __int_as_float(0xff800000);
   int flip = 0;
   // block statistics
   uint32_t kmin = 0xffffffffu, kmax = 0u;
 #pragma unroll
-  for (int i = 0; i < TK_CH * 8; ++i) {
+  for (int i = 0; i < NE; ++i) {
     kmax = key[i] > kmax ? key[i] : kmax;
     kmin = (key[i] > TK_KEY_NINF && key[i] < kmin) ? key[i] : kmin;
   }
@@ -146,7 +149,7 @@ __device__ __forceinline__ float topk_select(const uint32_t (&key)[TK_CH * 8], i
     kmax = S.kmax[w] > kmax ? S.kmax[w] : kmax;
   }
   // every exit goes through the barrier at the end: the next row reuses S
-  float answer = NEG_INF;
+  uint32_t answer = TK_KEY_NINF;
   bool open = kmax > TK_KEY_NINF;                              // else: nothing above -inf
   uint32_t lo = kmin, hi = kmax;
   int c_lo = 0, c_hi = 0;
@@ -157,7 +160,7 @@ __device__ __forceinline__ float topk_select(const uint32_t (&key)[TK_CH * 8], i
   if (open) {
     c_hi = topk_count(key, hi, S, flip);
     if (c_hi >= K) {
-      answer = topk_value(hi);
+      answer = hi;
       open = false;
     }
   }
@@ -187,7 +190,7 @@ __device__ __forceinline__ float topk_select(const uint32_t (&key)[TK_CH * 8], i
       // compaction without a chain of atomics: own count, warp scan, one atomic per warp, then the writes
       int mine = 0;
 #pragma unroll
-      for (int i = 0; i < TK_CH * 8; ++i) mine += (key[i] >= lo) & (key[i] < hi);
+      for (int i = 0; i < NE; ++i) mine += (key[i] >= lo) & (key[i] < hi);
       int incl = mine;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
@@ -199,7 +202,7 @@ __device__ __forceinline__ float topk_select(const uint32_t (&key)[TK_CH * 8], i
       int pos = __shfl_sync(kFull, base, 31) + incl - mine;
       if (mine) {
 #pragma unroll
-        for (int i = 0; i < TK_CH * 8; ++i) {
+        for (int i = 0; i < NE; ++i) {
           if (key[i] >= lo && key[i] < hi) {
             if (pos < TK_LIST) S.list[pos] = key[i];
             ++pos;
@@ -223,10 +226,98 @@ __device__ __forceinline__ float topk_select(const uint32_t (&key)[TK_CH * 8], i
       __syncthreads();
       result = S.result;
     }
-    answer = topk_value(result);
+    answer = result;
   }
   __syncthreads();
   return answer;
+}
+
+// Value of the K-th largest of the row's keys (64 per thread).  Rows of at least 4096 tokens first
+// go through a pre-filter: a bisection on a 512-key sample (two keys per thread) finds a bound t0
+// that, by the sample's ranks, leaves somewhat more than K keys; one pass over all keys counts
+// and compacts those >= t0 into shared memory, and the exact selection then runs on at most
+// TK_CE keys per thread instead of 64.  If the bound turns out to keep fewer than K keys or more
+// than fit (a sample that misleads, many equal keys), the selection runs on all keys instead.
+__device__ __forceinline__ float topk_select(const uint32_t (&key)[TK_CH * 8], int K, int V, TopkShared& S) {
+  const int tid = threadIdx.x, lane = tid & 31;
+  const float mean = static_cast<float>(K) * 512.0f / static_cast<float>(V);   // expected sample rank of the answer
+  const int r_lo = static_cast<int>(mean + 3.5f * sqrtf(mean) + 3.0f);
+  const int r_hi = r_lo + (r_lo / 6 > 4 ? r_lo / 6 : 4);
+  const bool try_filter = V >= 4096 && static_cast<long long>(r_hi + r_lo / 2) * V / 512 < TK_CAND;
+  if (try_filter) {
+    int flip = 0;
+    const uint32_t smp[2] = {key[0], key[32]};
+    // the sample's own range (block minimum above -inf and maximum): the search is on values, so it must
+    // start from bounds that are as close together as the data are
+    uint32_t lo = 0xffffffffu, hi = 0u, t0 = 0u;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      hi = smp[i] > hi ? smp[i] : hi;
+      lo = (smp[i] > TK_KEY_NINF && smp[i] < lo) ? smp[i] : lo;
+    }
+    lo = __reduce_min_sync(kFull, lo);
+    hi = __reduce_max_sync(kFull, hi);
+    if (lane == 0) {
+      S.kmin[tid >> 5] = lo;
+      S.kmax[tid >> 5] = hi;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < TKW; ++w) {
+      lo = S.kmin[w] < lo ? S.kmin[w] : lo;
+      hi = S.kmax[w] > hi ? S.kmax[w] : hi;
+    }
+    bool found = false;
+    for (int pass = 0; pass < 40 && hi - lo > 1u; ++pass) {
+      uint32_t km = topk_key(0.5f * topk_value(lo) + 0.5f * topk_value(hi));
+      if (!(km > lo && km < hi)) km = lo + ((hi - lo) >> 1);
+      const int c = topk_count<2>(smp, km, S, flip);
+      if (c > r_hi) {
+        lo = km;
+      } else if (c < r_lo) {
+        hi = km;
+      } else {
+        t0 = km;
+        found = true;
+        break;
+      }
+    }
+    if (!found) t0 = lo;   // many equal sample keys: the bound that keeps more
+    // count and compact the keys >= t0
+    int mine = 0;
+#pragma unroll
+    for (int i = 0; i < TK_CH * 8; ++i) mine += key[i] >= t0;
+    int incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(kFull, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (tid == 0) S.list_n = 0;
+    __syncthreads();
+    int base = 0;
+    if (lane == 31) base = atomicAdd(&S.list_n, incl);
+    int pos = __shfl_sync(kFull, base, 31) + incl - mine;
+    __syncthreads();
+    const int total = S.list_n;   // uniform
+    if (t0 > 0u && total >= K && total <= TK_CAND) {
+#pragma unroll
+      for (int i = 0; i < TK_CH * 8; ++i) {
+        if (key[i] >= t0) S.cand[pos++] = key[i];
+      }
+      __syncthreads();
+      uint32_t ck[TK_CE];
+#pragma unroll
+      for (int j = 0; j < TK_CE; ++j) {
+        const int idx = tid + j * TKT;
+        ck[j] = idx < total ? S.cand[idx] : 0u;
+      }
+      __syncthreads();   // S.list_n is reused by the selection
+      return topk_value(topk_select_keys<TK_CE>(ck, K, S));
+    }
+    __syncthreads();
+  }
+  return topk_value(topk_select_keys<TK_CH * 8>(key, K, S));
 }
 
 // raw row(s) of one job -> shared memory
@@ -352,7 +443,7 @@ __global__ void __launch_bounds__(TKT, 2) lantern_topk_kernel(VerifyParams P, in
     __syncthreads();   // the staging area is free
     if (tid == 0 && j + G < njobs)
       topk_issue<BF16, UNC>(P, item_next, job_is_drafter(j + G), tsm, rowbytes, &S.bar_full);
-    const float t = topk_select(key, K, S);
+    const float t = topk_select(key, K, V, S);
     if (tid == 0) (drafter ? P.thr_p : P.thr_q)[item] = t;
     item = item_next;
   }

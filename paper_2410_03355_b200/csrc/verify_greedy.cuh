@@ -181,11 +181,11 @@ __device__ __forceinline__ float4 greedy_quad(const unsigned char* area, uint32_
     c = *reinterpret_cast<const float4*>(area + static_cast<size_t>(qd) * 16);
     if (UNC) u = *reinterpret_cast<const float4*>(area + rowbytes + static_cast<size_t>(qd) * 16);
   }
-  if (UNC) {
-    c.x = __fmaf_rn(s, __fsub_rn(c.x, u.x), u.x);
-    c.y = __fmaf_rn(s, __fsub_rn(c.y, u.y), u.y);
-    c.z = __fmaf_rn(s, __fsub_rn(c.z, u.z), u.z);
-    c.w = __fmaf_rn(s, __fsub_rn(c.w, u.w), u.w);
+  if (UNC) {   // l_u + s (l_c - l_u) on packed pairs: same roundings as the scalar form, half the instructions
+    const uint64_t s2 = pack2(s, s);
+    const uint64_t u01 = pack2(u.x, u.y), u23 = pack2(u.z, u.w);
+    unpack2(fma2(s2, sub2(pack2(c.x, c.y), u01), u01), c.x, c.y);
+    unpack2(fma2(s2, sub2(pack2(c.z, c.w), u23), u23), c.z, c.w);
   }
   return c;
 }
@@ -296,8 +296,13 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
       if (z.w > m) m = z.w, mi = 4 * qd + 3;
       if (m > old) ssum *= greedy_ex2((old - m) * L_hi);   // old = -inf: the factor is 0, and so was the sum
       const float mL = m > NEG_INF ? m * L_hi : 0.0f;       // all -inf so far: every numerator is 2^-inf = 0
-      ssum += (greedy_ex2(__fmaf_rn(z.x, L_hi, -mL)) + greedy_ex2(__fmaf_rn(z.y, L_hi, -mL))) +
-              (greedy_ex2(__fmaf_rn(z.z, L_hi, -mL)) + greedy_ex2(__fmaf_rn(z.w, L_hi, -mL)));
+      float a0, a1, a2_, a3;
+      {
+        const uint64_t L2 = pack2(L_hi, L_hi), n2 = pack2(-mL, -mL);
+        unpack2(fma2(pack2(z.x, z.y), L2, n2), a0, a1);
+        unpack2(fma2(pack2(z.z, z.w), L2, n2), a2_, a3);
+      }
+      ssum += (greedy_ex2(a0) + greedy_ex2(a1)) + (greedy_ex2(a2_) + greedy_ex2(a3));
     }
     // A NaN logit (or +inf, through inf - inf) makes the thread's sum NaN: no per-element test is needed.
     const int bad = ssum != ssum;

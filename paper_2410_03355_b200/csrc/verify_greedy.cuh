@@ -279,9 +279,8 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
 
     // ---- the sweep: maximum, smallest arg max, numerators summed against the running maximum ----
     float m = NEG_INF, ssum = 0.0f;
-    int mi = 0x7fffffff;
-#pragma unroll 4
-    for (int qd = tid; qd < quads; qd += GCT) {
+    int mq = -1;   // the quad that first reached the thread's maximum; the position inside it is found afterwards
+    auto quad_of = [&](int qd) {
       float4 z = greedy_quad<BF16, UNC>(raw, rowbytes, qd, P.cfg_scale);
       if (TOPK) {   // a NaN stays, to be reported
         z.x = z.x < tq ? NEG_INF : z.x;
@@ -289,11 +288,14 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
         z.z = z.z < tq ? NEG_INF : z.z;
         z.w = z.w < tq ? NEG_INF : z.w;
       }
+      return z;
+    };
+#pragma unroll 4
+    for (int qd = tid; qd < quads; qd += GCT) {
+      const float4 z = quad_of(qd);
       const float old = m;
-      if (z.x > m) m = z.x, mi = 4 * qd;          // ascending index within a thread: strict > keeps
-      if (z.y > m) m = z.y, mi = 4 * qd + 1;      // the smallest index
-      if (z.z > m) m = z.z, mi = 4 * qd + 2;
-      if (z.w > m) m = z.w, mi = 4 * qd + 3;
+      const float qm = max3(z.x, z.y, fmaxf(z.z, z.w));
+      if (qm > m) m = qm, mq = qd;                 // ascending quads: strict > keeps the first one
       if (m > old) ssum *= greedy_ex2((old - m) * L_hi);   // old = -inf: the factor is 0, and so was the sum
       const float mL = m > NEG_INF ? m * L_hi : 0.0f;       // all -inf so far: every numerator is 2^-inf = 0
       float a0, a1, a2_, a3;
@@ -306,6 +308,11 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
     }
     // A NaN logit (or +inf, through inf - inf) makes the thread's sum NaN: no per-element test is needed.
     const int bad = ssum != ssum;
+    int mi = 0x7fffffff;   // smallest index at which the thread's maximum sits: one quad read again
+    if (mq >= 0) {
+      const float4 z = quad_of(mq);
+      mi = 4 * mq + (z.x == m ? 0 : (z.y == m ? 1 : (z.z == m ? 2 : 3)));
+    }
     {
       const float wmx = warp_max(m);
       const int wix = __reduce_min_sync(kFull, (m == wmx) ? mi : 0x7fffffff);

@@ -279,6 +279,7 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
 
     // ---- the sweep: maximum, smallest arg max, numerators summed against the running maximum ----
     float m = NEG_INF, ssum = 0.0f;
+    float mL = 0.0f;   // m * log2(e) once a finite maximum exists (before that every numerator is 2^-inf = 0)
     int mq = -1;   // the quad that first reached the thread's maximum; the position inside it is found afterwards
     auto quad_of = [&](int qd) {
       float4 z = greedy_quad<BF16, UNC>(raw, rowbytes, qd, P.cfg_scale);
@@ -295,9 +296,10 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
       const float4 z = quad_of(qd);
       const float old = m;
       const float qm = max3(z.x, z.y, fmaxf(z.z, z.w));
-      if (qm > m) m = qm, mq = qd;                 // ascending quads: strict > keeps the first one
-      if (m > old) ssum *= greedy_ex2((old - m) * L_hi);   // old = -inf: the factor is 0, and so was the sum
-      const float mL = m > NEG_INF ? m * L_hi : 0.0f;       // all -inf so far: every numerator is 2^-inf = 0
+      if (qm > m) {                                // ascending quads: strict > keeps the first one
+        m = qm, mq = qd, mL = qm * L_hi;
+        ssum *= greedy_ex2((old - m) * L_hi);      // old = -inf: the factor is 0, and so was the sum
+      }
       float a0, a1, a2_, a3;
       {
         const uint64_t L2 = pack2(L_hi, L_hi), n2 = pack2(-mL, -mL);

@@ -108,6 +108,19 @@ __device__ __forceinline__ void ctx_issue_rows(const VerifyParams& P, int item, 
   }
 }
 
+// Ask L2 for the rows of a context ahead of time: the bulk copy that later brings them into shared
+// memory (it cannot start before the group has released its staging area) then finds them on chip.
+template <bool BF16, bool UNC>
+__device__ __forceinline__ void ctx_prefetch_rows(const VerifyParams& P, int item, int rowbytes) {
+  const size_t row_off = static_cast<size_t>(item) * rowbytes;
+  const size_t branch = static_cast<size_t>(P.B) * P.R * rowbytes;
+  const unsigned char* t = static_cast<const unsigned char*>(P.target) + row_off;
+  const unsigned char* d = static_cast<const unsigned char*>(P.draft) + row_off;
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(t), "r"(rowbytes) : "memory");
+  if (UNC) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(t + branch), "r"(rowbytes) : "memory");
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(d), "r"(rowbytes) : "memory");
+}
+
 // one logit of a row in global memory, widened to fp32
 template <bool BF16>
 __device__ __forceinline__ float ctx_raw_logit(const void* base, size_t elem) {
@@ -264,6 +277,7 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
         }
         fence_proxy_async();
         ctx_issue_rows<BF16, UNC>(P, it_cur.item, smem + grp * stage_bytes, rowbytes, &bar_full[grp]);
+        if (it_next.item >= 0) ctx_prefetch_rows<BF16, UNC>(P, it_next.item, rowbytes);
         it_cur = it_next;
         tq_cur = tq_next, tp_cur = tp_next;
         it_next = load_item(w_next2);

@@ -25,7 +25,7 @@
 // inverse-CDF draw or the write-back for the next sibling.
 #pragma once
 
-#define LANTERN_CONTEXT_KERNEL_REVISION 13   // bump on every change to this file
+#define LANTERN_CONTEXT_KERNEL_REVISION 14   // bump on every change to this file
 
 namespace lantern {
 

@@ -260,7 +260,9 @@ lantern_status lantern_verify_static(const void* target_logits, const void* draf
  * stored profiler counters can be matched to the code they were taken on. */
 int lantern_kernel_revision(void);
 
-/* Number of kernels (and memsets) one lantern_verify call enqueues; for launch accounting. */
+/* Number of kernels (and memsets) one lantern_verify call enqueues (memset, plan, fused pass or greedy
+ * pass, walk, bonus); a call with a top-k filter enqueues one threshold kernel more in greedy decoding
+ * and two more in sampling.  For launch accounting. */
 int lantern_verify_launch_count(void);
 
 /* Measurement hook (not part of the method): when both arguments are non-NULL cudaEvent_t

@@ -109,7 +109,16 @@ __global__ void __launch_bounds__(BNT, 3) lantern_bonus_stream_kernel(VerifyPara
       st = LANTERN_ST_NONFINITE;
       __syncthreads();   // every thread has read S.wm and is done with the rows
     } else {
-      // ---- sweep 2: numerators, one partial sum per iteration ----
+      // ---- sweep 2: numerators 2^((z - M) log2 e) through the ex2 unit (as in the fused pass), one partial
+      // sum per iteration ----
+      const float L_hi = 1.44269502162933349609375f;
+      const uint64_t L2 = pack2(L_hi, L_hi), nM2 = pack2(-(M * L_hi), -(M * L_hi));
+      auto numer4 = [&](const float4& z) {
+        float a0, a1, a2_, a3;
+        unpack2(fma2(pack2(z.x, z.y), L2, nM2), a0, a1);
+        unpack2(fma2(pack2(z.z, z.w), L2, nM2), a2_, a3);
+        return make_float4(greedy_ex2(a0), greedy_ex2(a1), greedy_ex2(a2_), greedy_ex2(a3));
+      };
       float s[BN_ITERS];
 #pragma unroll
       for (int j = 0; j < BN_ITERS; ++j) {
@@ -117,7 +126,8 @@ __global__ void __launch_bounds__(BNT, 3) lantern_bonus_stream_kernel(VerifyPara
         s[j] = 0.0f;
         if (qd < quads) {
           const float4 z = quad(qd, tq);
-          s[j] = (exp_nonpos(z.x - M) + exp_nonpos(z.y - M)) + (exp_nonpos(z.z - M) + exp_nonpos(z.w - M));
+          const float4 e = numer4(z);
+          s[j] = (e.x + e.y) + (e.z + e.w);
         }
       }
 #pragma unroll
@@ -170,7 +180,8 @@ __global__ void __launch_bounds__(BNT, 3) lantern_bonus_stream_kernel(VerifyPara
         if (excl + md > target && !(excl > target)) {   // the first thread whose inclusive sum exceeds the target
           const int qd = tid + jstar * BNT;
           const float4 z = quad(qd, tq);
-          const float e[4] = {exp_nonpos(z.x - M), exp_nonpos(z.y - M), exp_nonpos(z.z - M), exp_nonpos(z.w - M)};
+          const float4 e4 = numer4(z);
+          const float e[4] = {e4.x, e4.y, e4.z, e4.w};
           double cum = excl;
           int pick = -1, lastpos = -1;
 #pragma unroll

@@ -1,5 +1,4 @@
-// Device-side helpers shared by the LANTERN kernels: accurate exponential, warp/block
-// reductions and scans, mbarrier + bulk-copy (TMA) wrappers for sm_100a.
+// Device-side helpers shared by the LANTERN kernels: warp reductions and scans, the JSD mass bound, mbarrier + bulk-copy (TMA) wrappers for sm_100a.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -9,25 +8,6 @@ namespace lantern {
 
 constexpr int kWarp = 32;
 constexpr unsigned kFull = 0xffffffffu;
-
-// ---------------------------------------------------------------------------------------
-// exp(t) for t <= 0 (softmax numerators) with about 2.5e-7 relative error.
-// 2^(t*log2e) is evaluated by the hardware ex2 unit on x = fl(t*L_hi); the rounding error
-// of that product and the low part of log2(e) are folded back in to first order:
-// 2^(x+e) = 2^x * (1 + e ln2 + ...).  NaN propagates; t = -inf gives 0.
-// ---------------------------------------------------------------------------------------
-__device__ __forceinline__ float exp_nonpos(float t) {
-  const float L_hi = 1.44269502162933349609375f;     // fl32(log2 e)
-  const float L_lo = 1.925963033500011e-08f;         // log2 e - L_hi
-  const float LN2 = 0.693147182464599609375f;
-  t = (t < -104.0f) ? -104.0f : t;                   // keeps NaN, maps -inf to a flushed-to-zero result
-  float x = t * L_hi;
-  float e = __fmaf_rn(t, L_hi, -x);
-  e = __fmaf_rn(t, L_lo, e);
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return __fmaf_rn(y, e * LN2, y);
-}
 
 // ---------------------------------------------------------------------------------------
 // warp primitives

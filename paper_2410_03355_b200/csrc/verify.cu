@@ -17,7 +17,7 @@
 // context without children (Algorithm 1, line after the loop).
 //
 // Precision: processed logits are fp32 (difference, fused multiply-add, division, each
-// rounded once); exponentials are fp32 with ~2.5e-7 relative error; every sum over more
+// rounded once); exponentials come from the fp32 ex2 unit (about 3e-7 relative); every sum over more
 // than eight terms and every threshold comparison is done in double precision.
 #include "verify_common.cuh"
 

@@ -82,7 +82,7 @@ def check_outputs(inp, host, delta, gpu, divergence=oracle.DIV_TVD, top_k=0):
     far = t & (ora.margin >= WINDOW)
     assert np.array_equal(m[far], ora.m[far])
     agree = t & (m == ora.m)
-    assert agree.sum() > 0
+    assert agree.sum() > 0 or not t.any()         # (no node tested at all: N = 0, or every sequence flagged)
     assert (np.abs(qa[agree] - ora.qa[agree]) <= REL * ora.qa[agree]).all()
     assert not gpu.node_px.cpu().numpy()[t].any()       # trace entries of untested nodes are not written
     return ora, near

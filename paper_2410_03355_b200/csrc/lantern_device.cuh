@@ -95,17 +95,20 @@ __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, 
                "l"(src_gmem), "r"(bytes), "r"(smem_addr(bar))
                : "memory");
 }
-// Bounded wait for phase `parity` of `bar`.  Returns false if the limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t max_tries = (1u << 22)) {
+// Bounded wait for phase `parity` of `bar`.  Returns false if the limit ran out.  Each try may suspend
+// the thread in hardware for up to `suspend_ns` (it wakes when the phase completes), so a long wait costs
+// few issue slots; the hint is an upper limit, the loop bound is what ends a wait that never completes.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t max_tries = (1u << 21),
+                                          uint32_t suspend_ns = 4000) {
   const uint32_t a = smem_addr(bar);
   for (uint32_t i = 0; i < max_tries; ++i) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(a), "r"(parity)
+        : "r"(a), "r"(parity), "r"(suspend_ns)
         : "memory");
     if (ok) return true;
   }

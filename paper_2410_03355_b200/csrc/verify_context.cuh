@@ -25,7 +25,7 @@
 // inverse-CDF draw or the write-back for the next sibling.
 #pragma once
 
-#define LANTERN_CONTEXT_KERNEL_REVISION 14   // bump on every change to this file
+#define LANTERN_CONTEXT_KERNEL_REVISION 15   // bump on every change to this file
 
 namespace lantern {
 
@@ -67,7 +67,9 @@ struct GroupShared {
   int acc_valid;                // acc_e / acc_p are usable for the current child
   int tok;
   int status;                   // OR of status bits seen by single threads
-  WorkItem work;
+  int fail;                     // a bounded wait for the target rows ran out (sticky)
+  float thr[2][2];              // top-k thresholds (target, drafter) of the context in work[i]
+  WorkItem work[2];             // descriptor of context i in work[i & 1]: the next one is published while the current one runs
 };
 
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -87,25 +89,29 @@ __device__ __forceinline__ double exp2_single(float z, float shift) {
   return static_cast<double>(__fmaf_rn(y, xl * 0.693147182464599609375f, y));
 }
 
-template <bool BF16, bool UNC>
-__device__ __forceinline__ void ctx_issue_rows(const VerifyParams& P, int item, unsigned char* stage, int rowbytes,
-                                               uint64_t* bar) {
-  const int nrows = UNC ? 3 : 2;
-  mbar_expect_tx(bar, static_cast<uint32_t>(nrows * rowbytes));
-  const size_t row_off = static_cast<size_t>(item) * rowbytes;
-  const size_t branch = static_cast<size_t>(P.B) * P.R * rowbytes;
-  const unsigned char* src[3];
-  src[0] = static_cast<const unsigned char*>(P.target) + row_off;
-  src[1] = UNC ? static_cast<const unsigned char*>(P.target) + branch + row_off
-               : static_cast<const unsigned char*>(P.draft) + row_off;
-  src[2] = static_cast<const unsigned char*>(P.draft) + row_off;
-  for (int r = 0; r < nrows; ++r) {
-    const int dst_row = (r == nrows - 1) ? 2 : r;   // the drafter row always goes to row slot 2
-    for (int off = 0; off < rowbytes; off += 16384) {
-      const int n = min(16384, rowbytes - off);
-      bulk_load(stage + dst_row * rowbytes + off, src[r] + off, static_cast<uint32_t>(n), bar);
-    }
+// one row of a context into one row slot of a staging area, in bulk copies of at most 16 KB
+__device__ __forceinline__ void ctx_issue_row(unsigned char* dst, const unsigned char* src, int rowbytes, uint64_t* bar) {
+  for (int off = 0; off < rowbytes; off += 16384) {
+    const int n = min(16384, rowbytes - off);
+    bulk_load(dst + off, src + off, static_cast<uint32_t>(n), bar);
   }
+}
+// the drafter row of a context, into row slot 2
+__device__ __forceinline__ void ctx_issue_drafter(const VerifyParams& P, int item, unsigned char* stage, int rowbytes,
+                                                  uint64_t* bar) {
+  mbar_expect_tx(bar, static_cast<uint32_t>(rowbytes));
+  ctx_issue_row(stage + 2 * rowbytes, static_cast<const unsigned char*>(P.draft) + static_cast<size_t>(item) * rowbytes,
+                rowbytes, bar);
+}
+// the target rows of a context (conditional, and unconditional if there is one), into row slots 0 and 1
+template <bool UNC>
+__device__ __forceinline__ void ctx_issue_target(const VerifyParams& P, int item, unsigned char* stage, int rowbytes,
+                                                 uint64_t* bar) {
+  mbar_expect_tx(bar, static_cast<uint32_t>((UNC ? 2 : 1) * rowbytes));
+  const size_t row_off = static_cast<size_t>(item) * rowbytes;
+  const unsigned char* t = static_cast<const unsigned char*>(P.target) + row_off;
+  ctx_issue_row(stage, t, rowbytes, bar);
+  if (UNC) ctx_issue_row(stage + rowbytes, t + static_cast<size_t>(P.B) * P.R * rowbytes, rowbytes, bar);
 }
 
 // Ask L2 for the rows of a context ahead of time: the bulk copy that later brings them into shared
@@ -196,7 +202,8 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
   constexpr int LOG_CP = CP == 4 ? 2 : (CP == 2 ? 1 : 0);
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ GroupShared SG[NGRP];
-  __shared__ __align__(8) uint64_t bar_full[NGRP], bar_empty[NGRP];
+  // per group: drafter row landed / target rows landed / drafter slot free / target slots (E) free
+  __shared__ __align__(8) uint64_t bar_full_d[NGRP], bar_full_t[NGRP], bar_empty_d[NGRP], bar_empty_t[NGRP];
 
   const int tid = threadIdx.x, lane = tid & 31;
   const int V = P.V, N = P.N, R = P.R, k = P.k;
@@ -209,9 +216,12 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
 
   if (tid == 0) {
     for (int g = 0; g < NGRP; ++g) {
-      mbar_init(&bar_full[g], 1);
-      mbar_init(&bar_empty[g], GW);
+      mbar_init(&bar_full_d[g], 1);
+      mbar_init(&bar_full_t[g], 1);
+      mbar_init(&bar_empty_d[g], GW);
+      mbar_init(&bar_empty_t[g], GW);
       SG[g].status = 0;
+      SG[g].fail = 0;
     }
     fence_mbar_init();
     fence_proxy_async();
@@ -261,22 +271,28 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       load_thr(it_next, tq_next, tp_next);
       int w_next2 = me + 2 * G;
       for (int i = 0;; ++i) {
-        // the staging area is free once every warp of the group has finished the previous context
-        if (i >= 1 && !mbar_wait(&bar_empty[grp], (i - 1) & 1)) {
+        // The drafter slot is free once every warp of the group has streamed the previous context's
+        // drafter row (nothing reads it afterwards), i.e. while that context is still being decided:
+        // the next drafter row travels early, and the group streams it while its target rows are copied.
+        if (i >= 1 && !mbar_wait(&bar_empty_d[grp], (i - 1) & 1)) {
           it_cur.item = -1;
-          it_cur.pad = LANTERN_ST_INTERNAL;   // the group never released its area: stop handing out work
+          it_cur.pad = LANTERN_ST_INTERNAL;   // the group never released its slot: stop handing out work
         }
-        S.work = it_cur;                      // published by the mbarrier operation below
-        if (TOPK) {   // the group is between contexts: its scratch is free; these two slots stay untouched until read
-          S.wt[8 * GW - 2] = static_cast<double>(tq_cur);
-          S.wt[8 * GW - 3] = static_cast<double>(tp_cur);
+        S.work[i & 1] = it_cur;               // published by the mbarrier operation below
+        if (TOPK) {
+          S.thr[i & 1][0] = tq_cur;
+          S.thr[i & 1][1] = tp_cur;
         }
         if (it_cur.item < 0) {
-          mbar_arrive(&bar_full[grp]);        // wake the group; it sees the terminator
+          mbar_arrive(&bar_full_d[grp]);      // wake the group; it sees the terminator
           break;
         }
         fence_proxy_async();
-        ctx_issue_rows<BF16, UNC>(P, it_cur.item, smem + grp * stage_bytes, rowbytes, &bar_full[grp]);
+        ctx_issue_drafter(P, it_cur.item, smem + grp * stage_bytes, rowbytes, &bar_full_d[grp]);
+        // the target slots (later E) are free once every warp of the group has finished the previous context
+        if (i >= 1 && !mbar_wait(&bar_empty_t[grp], (i - 1) & 1)) break;   // the group's own wait runs out too
+        fence_proxy_async();
+        ctx_issue_target<UNC>(P, it_cur.item, smem + grp * stage_bytes, rowbytes, &bar_full_t[grp]);
         if (it_next.item >= 0) ctx_prefetch_rows<BF16, UNC>(P, it_next.item, rowbytes);
         it_cur = it_next;
         tq_cur = tq_next, tp_cur = tp_next;
@@ -300,22 +316,35 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
   const unsigned char* ru = stage + rowbytes;
   unsigned char* rd = stage + 2 * rowbytes;
   constexpr bool T_is_one = TONE;
-  // eight processed drafter logits of 16-byte group g (z_p = l_d / T)
-  auto draft_chunk = [&](int g, float (&out)[8]) {
+  // The eight raw drafter logits of 16-byte group g of a row in global memory (a rejection reads the
+  // drafter row again from there -- normally from L2 -- because its slot already belongs to the next context)
+  struct DraftRaw {
+    uint4 a, b;   // b: second half of an fp32 group
+  };
+  auto draft_fetch = [&](const unsigned char* row, int g) {
+    DraftRaw d;
+    d.b = make_uint4(0, 0, 0, 0);
     if (BF16) {
-      const uint4 d = *reinterpret_cast<const uint4*>(rd + g * 16);
-      const uint32_t dw[4] = {d.x, d.y, d.z, d.w};
+      d.a = __ldg(reinterpret_cast<const uint4*>(row + static_cast<size_t>(g) * 16));
+    } else {
+      d.a = __ldg(reinterpret_cast<const uint4*>(row + static_cast<size_t>(g) * 32));
+      d.b = __ldg(reinterpret_cast<const uint4*>(row + static_cast<size_t>(g) * 32 + 16));
+    }
+    return d;
+  };
+  // the same eight as processed logits (z_p = l_d / T)
+  auto draft_chunk = [&](const DraftRaw& d, float (&out)[8]) {
+    if (BF16) {
+      const uint32_t dw[4] = {d.a.x, d.a.y, d.a.z, d.a.w};
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         out[2 * i] = __uint_as_float(dw[i] << 16);
         out[2 * i + 1] = __uint_as_float(dw[i] & 0xffff0000u);
       }
     } else {
+      const uint32_t dw[8] = {d.a.x, d.a.y, d.a.z, d.a.w, d.b.x, d.b.y, d.b.z, d.b.w};
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const float4 d = *reinterpret_cast<const float4*>(rd + g * 32 + h * 16);
-        out[4 * h] = d.x, out[4 * h + 1] = d.y, out[4 * h + 2] = d.z, out[4 * h + 3] = d.w;
-      }
+      for (int e = 0; e < 8; ++e) out[e] = __uint_as_float(dw[e]);
     }
     if (!T_is_one) {
 #pragma unroll
@@ -326,16 +355,16 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
     // One warp watches the copy's mbarrier (bounded wait); the group barrier then releases everybody
     // at once and tells every thread alike whether the rows have landed.
     bool landed = true;
-    if (gw == 0) landed = mbar_wait(&bar_full[grp], iter & 1);
+    if (gw == 0) landed = mbar_wait(&bar_full_d[grp], iter & 1);
     const bool arrived = gbar_and(grp, landed);
     if (!arrived) break;   // the copy did not land within the limit; the walk reports the missing record
-    const WorkItem cur = S.work;
+    const WorkItem cur = S.work[iter & 1];
     const int item = cur.item;
     if (item < 0) break;
     float tq = 0.0f, tp = 0.0f;   // top-k thresholds of this context's target and drafter rows
     if (TOPK) {
-      tq = static_cast<float>(S.wt[8 * GW - 2]);
-      tp = static_cast<float>(S.wt[8 * GW - 3]);
+      tq = S.thr[iter & 1][0];
+      tp = S.thr[iter & 1][1];
     }
     const int b = item / R;
     const ChildInfo* kids = P.children + cur.cbase;
@@ -355,12 +384,13 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       const int j = 4 * gt + 1 + i;
       nb[i] = (j < k) ? ld_nc_here(P.nbr + static_cast<size_t>(xt) * k + j) : -1;
     }
-    float raw_c = 0.0f, raw_u = 0.0f, raw_d = 0.0f;
+    // (the drafter logit of x~ goes to every thread: the drafter row does not stay in shared memory)
+    float raw_c = 0.0f, raw_u = 0.0f;
+    float raw_d = ctx_raw_logit<BF16>(P.draft, static_cast<size_t>(item) * V + xt);
     if (gt == 0) {
       const size_t e = static_cast<size_t>(item) * V + xt;
       raw_c = ctx_raw_logit<BF16>(P.target, e);
       if (UNC) raw_u = ctx_raw_logit<BF16>(P.target, static_cast<size_t>(P.B) * R * V + e);
-      raw_d = ctx_raw_logit<BF16>(P.draft, e);
     }
 
     // ---------------- streaming part, thread-local, NP passes of CP chunks ----------------
@@ -390,6 +420,63 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       unpack2(v, lo, hi);
       return pack2(__fdiv_rn(lo, P.T), __fdiv_rn(hi, P.T));
     };
+    // --- drafter first (its row came early): slice maximum and partial sum of numerators ---
+#pragma unroll
+    for (int p = 0; p < NP; ++p) {
+      float mp = ninf;
+#pragma unroll
+      for (int c = 0; c < CP; ++c) {
+        const int g = (p * CP + c) * GT + gt;
+        if (g * 8 < V) {
+          uint64_t d2[4];
+          pairs_of(rd, g, d2);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            uint64_t l2 = d2[i];
+            if (!T_is_one) l2 = divide_T(l2);
+            float lo, hi;
+            unpack2(l2, lo, hi);
+            if (TOPK) {   // below the row's top-k threshold: -inf
+              lo = lo < tp ? ninf : lo, hi = hi < tp ? ninf : hi;
+              l2 = pack2(lo, hi);
+            }
+            a2[c * 4 + i] = l2;
+            mp = max3(mp, lo, hi);
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) a2[c * 4 + i] = pack2(ninf, ninf);
+        }
+      }
+      mp = fmaxf(mp, -1.0e37f);
+      const float mlp_w = mp * L_hi;
+      mlp_mine[p] = mlp_w;
+      const uint64_t nml2 = pack2(-mlp_w, -mlp_w);
+      uint64_t t2 = pack2(0.0f, 0.0f);
+#pragma unroll
+      for (int c = 0; c < CP; ++c) {
+        uint64_t e2[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          float lo, hi;
+          unpack2(fma2(a2[c * 4 + i], L2, nml2), lo, hi);
+          e2[i] = pack2(ex2_approx(lo), ex2_approx(hi));
+        }
+        t2 = add2(t2, add2(add2(e2[0], e2[1]), add2(e2[2], e2[3])));
+      }
+      float tlo, thi;
+      unpack2(t2, tlo, thi);
+      tp_mine[p] = tlo + thi;
+    }
+
+    // The drafter slot is not read again for this context (a rejection fetches the drafter logits from
+    // global memory): hand it back, so that the next context's drafter row is copied while this one is decided.
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&bar_empty_d[grp]);
+    // The target rows were issued when the previous context was released; they arrive while the drafter
+    // row is streamed.  Every thread waits for itself (bounded); a wait that runs out is reported after
+    // the next group barrier, where every thread sees it alike.
+    if (!mbar_wait(&bar_full_t[grp], iter & 1)) S.fail = 1;
     // --- target: guidance combine, slice maximum, numerators, partial sum; E replaces the raw rows ---
 #pragma unroll
     for (int p = 0; p < NP; ++p) {
@@ -449,77 +536,6 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       unpack2(t2, tlo, thi);
       tq_mine[p] = tlo + thi;
     }
-    // --- drafter: slice maximum and partial sum of numerators; the raw row stays in shared memory ---
-#pragma unroll
-    for (int p = 0; p < NP; ++p) {
-      float mp = ninf;
-#pragma unroll
-      for (int c = 0; c < CP; ++c) {
-        const int g = (p * CP + c) * GT + gt;
-        if (g * 8 < V) {
-          uint64_t d2[4];
-          pairs_of(rd, g, d2);
-          bool cut = false;
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            uint64_t l2 = d2[i];
-            if (!T_is_one) l2 = divide_T(l2);
-            float lo, hi;
-            unpack2(l2, lo, hi);
-            if (TOPK) {   // the filtered tokens are also struck from the raw row, which later steps re-read
-              const bool clo = lo < tp, chi = hi < tp;
-              float rlo, rhi;
-              unpack2(d2[i], rlo, rhi);
-              d2[i] = pack2(clo ? ninf : rlo, chi ? ninf : rhi);
-              lo = clo ? ninf : lo, hi = chi ? ninf : hi;
-              l2 = pack2(lo, hi);
-              cut |= clo | chi;
-            }
-            a2[c * 4 + i] = l2;
-            mp = max3(mp, lo, hi);
-          }
-          if (TOPK && cut) {
-            float v[8];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) unpack2(d2[i], v[2 * i], v[2 * i + 1]);
-            if (BF16) {
-              uint4 w;
-              w.x = (__float_as_uint(v[0]) >> 16) | (__float_as_uint(v[1]) & 0xffff0000u);
-              w.y = (__float_as_uint(v[2]) >> 16) | (__float_as_uint(v[3]) & 0xffff0000u);
-              w.z = (__float_as_uint(v[4]) >> 16) | (__float_as_uint(v[5]) & 0xffff0000u);
-              w.w = (__float_as_uint(v[6]) >> 16) | (__float_as_uint(v[7]) & 0xffff0000u);
-              *reinterpret_cast<uint4*>(rd + g * 16) = w;
-            } else {
-              *reinterpret_cast<float4*>(rd + g * 32) = make_float4(v[0], v[1], v[2], v[3]);
-              *reinterpret_cast<float4*>(rd + g * 32 + 16) = make_float4(v[4], v[5], v[6], v[7]);
-            }
-          }
-        } else {
-#pragma unroll
-          for (int i = 0; i < 4; ++i) a2[c * 4 + i] = pack2(ninf, ninf);
-        }
-      }
-      mp = fmaxf(mp, -1.0e37f);
-      const float mlp_w = mp * L_hi;
-      mlp_mine[p] = mlp_w;
-      const uint64_t nml2 = pack2(-mlp_w, -mlp_w);
-      uint64_t t2 = pack2(0.0f, 0.0f);
-#pragma unroll
-      for (int c = 0; c < CP; ++c) {
-        uint64_t e2[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          float lo, hi;
-          unpack2(fma2(a2[c * 4 + i], L2, nml2), lo, hi);
-          e2[i] = pack2(ex2_approx(lo), ex2_approx(hi));
-        }
-        t2 = add2(t2, add2(add2(e2[0], e2[1]), add2(e2[2], e2[3])));
-      }
-      float tlo, thi;
-      unpack2(t2, tlo, thi);
-      tp_mine[p] = tlo + thi;
-    }
-
     // ---------------- group statistics ----------------
     // common maxima first (one warp reduction, then eight values read by everybody), then the slices'
     // factors and the normalisers
@@ -539,6 +555,7 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       }
     }
     gbar(grp);   // [stats 1] per-warp maxima, and E, are visible
+    if (S.fail) break;   // the target rows did not land within the limit; the walk reports the missing record
     mlq_g = S.wmq[0];
     mlp_g = S.wmp[0];
 #pragma unroll
@@ -607,12 +624,15 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
           const int4 v = __ldg(reinterpret_cast<const int4*>(kids + ci + 1));
           sib.node = v.x, sib.token = v.y, sib.r = __int_as_float(v.z);
         }
-        // bulk numerators of x~ itself, common units (drafter: from the raw row, -inf once x~ was rejected)
+        // bulk numerators of x~ itself, common units (drafter: from its raw logit; no mass is left once x~
+        // was rejected as an earlier sibling of this context, or where the top-k filter cut it)
         float px_bulk, e_xt_bulk;
         {
-          float dz = BF16 ? __uint_as_float(static_cast<uint32_t>(reinterpret_cast<const unsigned short*>(rd)[xt]) << 16)
-                          : reinterpret_cast<const float*>(rd)[xt];
+          float dz = raw_d;
           if (!T_is_one) dz = __fdiv_rn(dz, P.T);
+          if (TOPK) dz = dz < tp ? ninf : dz;
+          for (int j = 0; j < ci; ++j)
+            if (__ldg(&kids[j].token) == xt) dz = ninf;
           px_bulk = ex2_approx(__fmaf_rn(dz, L_hi, -mlp_g));
           e_xt_bulk = E[EI(xt)] * S.fqt[owner_slice<LOG_CP>(xt)];
         }
@@ -719,11 +739,14 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
             }
           }
         }
-        if (gt == 0) {
-          E[EI(xt)] = -fabsf(E[EI(xt)]);
-          // x~ leaves the drafter distribution for the following siblings
-          if (BF16) reinterpret_cast<unsigned short*>(rd)[xt] = 0xff80;   // -inf
-          else reinterpret_cast<float*>(rd)[xt] = ninf;
+        if (gt == 0) E[EI(xt)] = -fabsf(E[EI(xt)]);
+        // x~ leaves the drafter distribution for the following siblings: the residual pass below strikes
+        // every token rejected so far (children 0..ci) from the drafter logits it fetches.  Which of this
+        // thread's chunks hold one:
+        uint32_t struck = 0;
+        for (int j = 0; j <= ci; ++j) {
+          const int t = j == ci ? xt : __ldg(&kids[j].token);
+          if (((t >> 3) & (GT - 1)) == gt) struck |= 1u << (t >> (3 + LOG_GT));
         }
         const bool last = (ci + 1 == nchild);
         if (!last) {   // next sibling's neighbour row, in flight during the residual pass
@@ -735,12 +758,20 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
             const int j = 4 * gt + 1 + i;
             nb[i] = (j < k) ? ld_nc_here(P.nbr + static_cast<size_t>(xt) * k + j) : -1;
           }
-          if (gt == 0) {   // its raw logits, for the double-precision replay below
+          raw_d = ctx_raw_logit<BF16>(P.draft, static_cast<size_t>(item) * V + xt);
+          if (gt == 0) {   // its raw target logits, for the double-precision replay below
             const size_t e = static_cast<size_t>(item) * V + xt;
             raw_c = ctx_raw_logit<BF16>(P.target, e);
             if (UNC) raw_u = ctx_raw_logit<BF16>(P.target, static_cast<size_t>(P.B) * R * V + e);
-            raw_d = ctx_raw_logit<BF16>(P.draft, e);
           }
+        }
+        // the drafter logits of the first pass, in flight across the barrier
+        const unsigned char* drow = static_cast<const unsigned char*>(P.draft) + static_cast<size_t>(item) * rowbytes;
+        DraftRaw dnext[CP];
+#pragma unroll
+        for (int c = 0; c < CP; ++c) {
+          const int g = c * GT + gt;
+          dnext[c] = draft_fetch(drow, g * 8 < V ? g : gt);
         }
         gbar(grp);   // [flags]
         // w = E - (p'/q' scale ratio) * ep in common units, i.e. E - ratio * ep in the slice's own units
@@ -753,6 +784,15 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
           // (a slice whose numerators are all negligible has factor 0; nothing of it survives anyway)
           const float ratio = fq_mine[p] > 0.0f ? ratio_g * (fp_mine[p] / fq_mine[p]) : 0.0f;
           float wp_ = 0.0f, pp_ = 0.0f;
+          DraftRaw dcur[CP];
+#pragma unroll
+          for (int c = 0; c < CP; ++c) {
+            dcur[c] = dnext[c];
+            if (p + 1 < NP) {   // the next pass's logits travel during this pass
+              const int g = ((p + 1) * CP + c) * GT + gt;
+              dnext[c] = draft_fetch(drow, g * 8 < V ? g : gt);
+            }
+          }
 #pragma unroll
           for (int c = 0; c < CP; ++c) {
             const int g = (p * CP + c) * GT + gt;
@@ -762,7 +802,20 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
               const float4 hi = *reinterpret_cast<const float4*>(E + EI(g * 8 + 4));
               const float e8[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
               float ep8[8];
-              draft_chunk(g, ep8);
+              draft_chunk(dcur[c], ep8);
+              if (TOPK) {   // below the row's top-k threshold: -inf
+#pragma unroll
+                for (int e = 0; e < 8; ++e) ep8[e] = ep8[e] < tp ? ninf : ep8[e];
+              }
+              if ((struck >> (p * CP + c)) & 1u) {   // a token rejected in this context sits in this chunk
+                for (int j = 0; j <= ci; ++j) {
+                  const int t = __ldg(&kids[j].token);
+                  if ((t >> 3) == g) {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) ep8[e] = (t & 7) == e ? ninf : ep8[e];
+                  }
+                }
+              }
 #pragma unroll
               for (int e = 0; e < 8; ++e) {
                 ep8[e] = ex2_approx(__fmaf_rn(ep8[e], L_hi, -mlp_mine[p]));
@@ -921,7 +974,7 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
     }
     // this context's staging area (rows and E) is no longer needed by this warp
     __syncwarp();
-    if (lane == 0) mbar_arrive(&bar_empty[grp]);
+    if (lane == 0) mbar_arrive(&bar_empty_t[grp]);
   }
 }
 

@@ -78,7 +78,7 @@ def algorithmic_bytes(cfg: dict, B: int, parents, greedy: bool = False) -> int:
 # of a 512-sequence call of the chain workload, as a ratio to that call's algorithmic bytes; traffic
 # grows in proportion to the contexts processed, so a full launch is scaled by its algorithmic bytes.
 # Tied to the kernel revision the capture was taken on: any other revision reports null.
-NCU_TRAFFIC = {"kernel_revision": 14, "workload": "batch_chain", "traffic_over_algorithmic": 374759424 / 366657536}
+NCU_TRAFFIC = {"kernel_revision": 15, "workload": "batch_chain", "traffic_over_algorithmic": 377546752 / 366657536}
 
 
 def ncu_traffic(workload, cfg, alg_bytes):

@@ -315,7 +315,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--divergence", default="tvd", choices=["tvd", "jsd"],
-                    help="what delta bounds (Section 6.2.2); the JSD run uses the workload's delta as it is")
+                    help="what delta bounds (Section 5.3.2); the JSD run uses the workload's delta as it is")
     ap.add_argument("--metric", default="l2", choices=["l2", "cosine"], help="latent proximity of the table")
     ap.add_argument("--top-k", type=int, default=0, dest="top_k",
                     help="top-k logit filter of the generation settings (Appendix B.2); 0 = off")
@@ -377,7 +377,7 @@ def main():
     torch.cuda.synchronize()
     alg_bytes = algorithmic_bytes(cfg, B, d["tree_parents"], args.greedy)
     T = 0.0 if args.greedy else d["T"]
-    ws = torch.empty(lt.verify_workspace_bytes(B, N, args.top_k), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(lt.verify_workspace_bytes(B, N, V, k, cfg["dtype"], args.top_k), dtype=torch.uint8, device="cuda")
     i32 = dict(dtype=torch.int32, device="cuda")
     out = lt.VerifyOutputs(accept_len=torch.empty(B, **i32), next_token=torch.empty(B, **i32),
                            accept_path=torch.empty((B, N), **i32), status=torch.empty(B, **i32),

@@ -21,7 +21,10 @@
  *   - Return value: LANTERN_OK, or a negative code found on the host before anything is
  *     launched (outputs untouched).  Faults that live in the data (a token out of range, a
  *     NaN logit ...) never trap: they set bits in out_status[b] and give that sequence the
- *     fallback result accept_len = number of drafts accepted before the fault, next_token = -1.
+ *     fallback result accept_len = number of drafts accepted before the fault, next_token = -1
+ *     (a token no vocabulary holds, so that a caller who does not look at out_status cannot
+ *     mistake it for a result).  lantern_last_status() tells in one word whether any sequence
+ *     of a call carried such a bit.
  */
 #ifndef LANTERN_H_
 #define LANTERN_H_
@@ -42,8 +45,9 @@ enum {
   LANTERN_E_PARAM = -3,         /* a scalar parameter is invalid (T <= 0, delta < 0, NaN ...) */
   LANTERN_E_WORKSPACE = -4,     /* workspace missing, too small or misaligned */
   LANTERN_E_CUDA = -5,          /* a CUDA runtime call failed (no device, launch error) */
-  LANTERN_E_ALIGN = -6,         /* a pointer is not 16-byte aligned */
-  LANTERN_E_UNIMPLEMENTED = -7  /* valid request this build does not cover (none at present) */
+  LANTERN_E_DATA = -6,          /* lantern_last_status: some sequence of the call carries a status bit */
+  LANTERN_E_UNIMPLEMENTED = -7, /* valid request this build does not cover (none at present) */
+  LANTERN_E_ALIGN = -8          /* a pointer is not 16-byte aligned */
 };
 
 /* storage type of logits */
@@ -55,9 +59,9 @@ enum {
   LANTERN_ST_BAD_PARENT = 2,    /* a parent index outside [-1, own index) */
   LANTERN_ST_BAD_UNIFORM = 4,   /* a uniform outside [0, 1) */
   LANTERN_ST_NONFINITE = 8,     /* NaN / +inf logit, or a row with no finite logit, on the walked path */
-  LANTERN_ST_DEGENERATE = 16,   /* a residual of zero total weight (rounding only) */
-  LANTERN_ST_BAD_TABLE = 32,    /* a neighbour entry outside [0, V) was met (it carries no mass) */
-  LANTERN_ST_INTERNAL = 64      /* an on-chip copy did not complete within its wait limit */
+  LANTERN_ST_DEGENERATE = 16,   /* a residual without weight was met; next_token was drawn from q instead (see lantern_verify) */
+  LANTERN_ST_BAD_TABLE = 32,    /* a neighbour entry outside [0, V) was met while a set A was grown (it carries no mass) */
+  LANTERN_ST_INTERNAL = 64      /* an on-chip copy did not complete within its wait limit: the sequence was not finished */
 };
 
 /* Human-readable name of a return code (static storage). */
@@ -83,7 +87,7 @@ lantern_status lantern_build_neighbors(const float* codebook, int V, int D, int 
                                        void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
- * Neighbour table under a named latent proximity (Section 6.2.1 compares the l2 distance with
+ * Neighbour table under a named latent proximity (Section 5.3.1 compares the l2 distance with
  * cosine similarity).  LANTERN_METRIC_L2 is lantern_build_neighbors.  LANTERN_METRIC_COSINE
  * scales every code to unit length first -- squared norm accumulated in fp32 in dimension order
  * by one fused multiply-add per dimension, one square root, one division per component; a zero
@@ -122,6 +126,18 @@ lantern_status lantern_build_neighbors_metric(const float* codebook, int V, int 
  * last residual, and where the walk reaches a node without children it is drawn from that
  * row's q, both by inverse CDF at uniforms[b, N].
  *
+ * A residual whose total weight is at most 1e-5 of the mass of the distribution it was taken
+ * from defines nothing to draw from (Algorithm 1's else-branch presumes a positive weight; the
+ * case needs a drafted token outside the drafter's own support, or two distributions that agree
+ * to single precision): the walk stops at that context, LANTERN_ST_DEGENERATE is set, and the
+ * next token is drawn from the context's own q at uniforms[b, N] -- a valid token.
+ *
+ * A neighbour entry outside [0, V) carries no mass; LANTERN_ST_BAD_TABLE is set when Algorithm 2's
+ * loop meets one, i.e. in a slot ahead of the one that ends the set (entries behind it are not read).
+ *
+ * Only contexts that the walk can reach need evaluating, and with many sequences per call the
+ * library leaves out most of the others (see out_node_* below); the results never depend on it.
+ *
  *   target_logits  [C, B, N+1, V], C = 2 (conditional, unconditional) if has_uncond else 1
  *   draft_logits   [B, N+1, V] (already guided); rows of contexts without children are not read;
  *                  may be NULL when N == 0
@@ -147,12 +163,15 @@ lantern_status lantern_build_neighbors_metric(const float* codebook, int V, int 
  *   out_accept_path [B, N] node ids of the accepted path in order, -1 padded; may be NULL
  *   out_status      [B] LANTERN_ST_* bits; may be NULL
  *   out_node_qa, out_node_px  [B, N] fp32: sum_A q and p(x~) as used in each node's test;
- *   out_node_m                [B, N] int32: |A_{k,delta}(x~)| - 1.  Every node whose parent
- *                  context has a child is evaluated up to and including the first accepted
- *                  sibling; other nodes get NaN / -1.  Each may be NULL.
- *   workspace       lantern_verify_workspace_bytes(B, N) bytes, 256-byte aligned
+ *   out_node_m                [B, N] int32: |A_{k,delta}(x~)| - 1.  Written for every node the
+ *                  walk tests (the children of each context on the accepted path, up to and
+ *                  including the first accepted one).  Other nodes hold either NaN / -1 or the
+ *                  values of a test made ahead of time that the walk did not need.  Each may be NULL.
+ *   workspace       lantern_verify_workspace_bytes(B, N, V, k, dtype) bytes, 256-byte aligned
+ *
+ * lantern_verify_workspace_bytes returns 0 for sizes lantern_verify would refuse.
  * ---------------------------------------------------------------------------------------- */
-size_t lantern_verify_workspace_bytes(int B, int N);
+size_t lantern_verify_workspace_bytes(int B, int N, int V, int k, int dtype);
 
 lantern_status lantern_verify(const void* target_logits, const void* draft_logits, int dtype, float cfg_scale,
                               int has_uncond, float T, const int32_t* draft_tokens, const int32_t* tree_parents,
@@ -165,7 +184,7 @@ lantern_status lantern_verify(const void* target_logits, const void* draft_logit
 /* ------------------------------------------------------------------------------------------
  * lantern_verify with the variants of the paper's ablations and generation settings.
  *
- *   divergence  what delta bounds when A_{k,delta}(x~) is grown (Section 6.2.2):
+ *   divergence  what delta bounds when A_{k,delta}(x~) is grown (Section 5.3.2):
  *               LANTERN_DIV_TVD  the total variation distance between q and q_{k,delta}(.|D = x~),
  *                                i.e. the mass moved onto x~ (Section 4.3; lantern_verify);
  *               LANTERN_DIV_JSD  their Jensen-Shannon divergence with the natural logarithm,
@@ -178,14 +197,14 @@ lantern_status lantern_verify(const void* target_logits, const void* draft_logit
  *               processed logits below the top_k-th largest of their row count as -inf, for the
  *               target and for the drafter alike, before the softmax; logits equal to the
  *               top_k-th largest are all kept.  0, or any value >= V, switches the filter off.
- *   workspace   lantern_verify_workspace_bytes_ex(B, N, top_k) bytes, 256-byte aligned
+ *   workspace   lantern_verify_workspace_bytes_ex(B, N, V, k, dtype, top_k) bytes, 256-byte aligned
  *
  * Everything else, and every return code, is as for lantern_verify; an unknown divergence or a
  * negative top_k returns LANTERN_E_PARAM.
  * ---------------------------------------------------------------------------------------- */
 enum { LANTERN_DIV_TVD = 0, LANTERN_DIV_JSD = 1 };
 
-size_t lantern_verify_workspace_bytes_ex(int B, int N, int top_k);
+size_t lantern_verify_workspace_bytes_ex(int B, int N, int V, int k, int dtype, int top_k);
 
 lantern_status lantern_verify_ex(const void* target_logits, const void* draft_logits, int dtype, float cfg_scale,
                                  int has_uncond, float T, const int32_t* draft_tokens, const int32_t* tree_parents,
@@ -229,24 +248,26 @@ lantern_status lantern_aggregate_all(const void* logits, int dtype, float cfg_sc
  * outputs; only the scratch that lantern_verify asks for is taken off their hands.
  *
  * The scratch lives in a fixed array inside the library's device image,
- * LANTERN_STATIC_WORKSPACE_BYTES (4 MiB) large: every GPU on which the library is loaded
- * holds those 4 MiB until the process exits.  The call makes no cudaMalloc / cudaFree and
+ * LANTERN_STATIC_WORKSPACE_BYTES (6 MiB) large: every GPU on which the library is loaded
+ * holds those 6 MiB until the process exits.  The call makes no cudaMalloc / cudaFree and
  * calls nothing that allocates.
  *
- *   - Sizes: lantern_verify_workspace_bytes(B, N) must not exceed
+ *   - Sizes: lantern_verify_workspace_bytes(B, N, V, k, dtype) must not exceed
  *     LANTERN_STATIC_WORKSPACE_BYTES (e.g. B = 8192, N = 7 or B = 1024, N = 60 fit);
  *     otherwise the call returns LANTERN_E_WORKSPACE and does nothing.  All other argument
  *     rules and return codes are those of lantern_verify.
  *   - First call on a device: the library looks up the device address of its array (once per
- *     device, with that device current, no allocation).  Make that first call outside any
- *     stream capture.
+ *     device, with that device current, no allocation) and keeps it for the life of the process.
+ *     Make that first call outside any stream capture.  The address does not survive a
+ *     cudaDeviceReset of that device: do not reset a device between calls.  Device ordinals
+ *     0..63 are served; a higher ordinal returns LANTERN_E_SHAPE.
  *   - The array is shared by every call on that device and keeps the previous call's contents;
  *     the call itself resets the few words that must start at zero.  Two such calls that may
  *     run on the GPU at the same time (different streams, different host threads) would write
  *     the same scratch and corrupt each other: serialise them, or use lantern_verify with
  *     separate workspaces.
  * ---------------------------------------------------------------------------------------- */
-#define LANTERN_STATIC_WORKSPACE_BYTES (4u << 20)
+#define LANTERN_STATIC_WORKSPACE_BYTES (6u << 20)
 
 lantern_status lantern_verify_static(const void* target_logits, const void* draft_logits, int dtype,
                                      float cfg_scale, int has_uncond, float T, const int32_t* draft_tokens,
@@ -260,10 +281,38 @@ lantern_status lantern_verify_static(const void* target_logits, const void* draf
  * stored profiler counters can be matched to the code they were taken on. */
 int lantern_kernel_revision(void);
 
-/* Number of kernels (and memsets) one lantern_verify call enqueues (memset, plan, fused pass or greedy
- * pass, walk, bonus); a call with a top-k filter enqueues one threshold kernel more in greedy decoding
- * and two more in sampling.  For launch accounting. */
-int lantern_verify_launch_count(void);
+/* Number of kernels (and memsets) one verification call enqueues: memset, plan, fused pass or greedy
+ * pass, walk, bonus; a call whose top-k filter is active (0 < top_k < V) enqueues one threshold kernel
+ * more in greedy decoding (greedy != 0) and two more in sampling.  For launch accounting. */
+int lantern_verify_launch_count(int greedy, int top_k_active);
+
+/* ------------------------------------------------------------------------------------------
+ * Summary of the data faults of the last verification call that used `workspace` (the per-sequence
+ * detail is in that call's out_status).  Waits for `cuda_stream`, on which that call was enqueued.
+ *
+ *   out_bits   receives the OR of the LANTERN_ST_* bits of all sequences of the call; may be NULL
+ *   returns    LANTERN_OK if no sequence carried a bit, LANTERN_E_DATA if one did,
+ *              LANTERN_E_NULL / LANTERN_E_CUDA otherwise
+ * ---------------------------------------------------------------------------------------- */
+lantern_status lantern_last_status(const void* workspace, void* cuda_stream, int32_t* out_bits);
+
+/* Work accounting of the last verification call that used `workspace` (waits for `cuda_stream`):
+ *   out_counts[0]  contexts with at least one drafted child
+ *   out_counts[1]  of those, the ones the fused pass evaluated
+ *   out_counts[2]  the ones it left out because the walk could not reach them (Algorithm 1 stops
+ *                  at the first rejection)
+ *   out_counts[3]  next tokens drawn from a context's own q (bonus draws and degenerate residuals)
+ * Greedy decoding evaluates every context: [1] and [2] stay 0 there. */
+lantern_status lantern_verify_counts(const void* workspace, void* cuda_stream, int64_t* out_counts);
+
+/* Self-test of the kernels' bounded waits (not part of the method).  Every wait for an on-chip copy
+ * gives up after a number of tries (2^21 by default, each suspended for up to 4 us); a sequence whose
+ * copy never completes ends with LANTERN_ST_INTERNAL instead of hanging the GPU.  This call sets, for
+ * the calling host thread's later sampling calls, the number of tries (0 = the default) and the index
+ * b * (N + 1) + c of one context whose copies the fused pass deliberately never starts (-1 = none), so
+ * that the path can be exercised without any fault: nothing is left in flight, the affected group
+ * gives up, the rest of the call is abandoned cleanly, and the device stays usable. */
+lantern_status lantern_debug_wait_test(int max_tries, int withhold_context);
 
 /* Measurement hook (not part of the method): when both arguments are non-NULL cudaEvent_t
  * handles, every later lantern_verify call made by the calling host thread records

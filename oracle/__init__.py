@@ -19,6 +19,7 @@ _LIB = os.path.join(_HERE, "liblantern_oracle.so")
 
 ST_BAD_TOKEN, ST_BAD_PARENT, ST_BAD_UNIFORM, ST_NONFINITE, ST_DEGENERATE, ST_BAD_TABLE = 1, 2, 4, 8, 16, 32
 DIV_TVD, DIV_JSD = 0, 1
+DEGENERATE_EPS = 1e-5      # reading R10: a residual of total weight <= this defines no distribution
 
 
 def build(force: bool = False) -> str:
@@ -46,7 +47,7 @@ def _p(a: Optional[np.ndarray]):
 
 
 def normalize_rows(codebook: np.ndarray) -> np.ndarray:
-    """Codes scaled to unit length in the canonical fp32 sequence (cosine variant, Section 6.2.1)."""
+    """Codes scaled to unit length in the canonical fp32 sequence (cosine variant, Section 5.3.1)."""
     cb = np.ascontiguousarray(codebook, dtype=np.float32)
     out = np.empty_like(cb)
     rc = _load().oracle_normalize_rows(_p(cb), cb.shape[0], cb.shape[1], _p(out))
@@ -57,7 +58,7 @@ def normalize_rows(codebook: np.ndarray) -> np.ndarray:
 
 def build_neighbors(codebook: np.ndarray, k: int, rows: Optional[np.ndarray] = None, metric: str = "l2"):
     """B_k for every code, or for the codes listed in `rows` (Algorithm 2, precompute block).
-    metric "l2" (the paper's choice) or "cosine" (Section 6.2.1: the same routine on unit-length codes).
+    metric "l2" (the paper's choice) or "cosine" (Section 5.3.1: the same routine on unit-length codes).
     Returns idx [n, k] int32, dist [n, k] fp32 with n = V or len(rows)."""
     assert metric in ("l2", "cosine")
     cb = np.ascontiguousarray(codebook, dtype=np.float32)
@@ -103,7 +104,7 @@ def jsd_collapsed(q0: float, S: float) -> float:
 
 def a_set(q: np.ndarray, nbr_row: np.ndarray, delta: float, divergence: int = DIV_TVD):
     """Size (beyond x~) and moved mass of A_{k,delta}(x~) on distribution q (Algorithm 2, second block);
-    the bound is on the TVD (Section 4.3) or on the JSD (Section 6.2.2).  nbr_row[0] is x~."""
+    the bound is on the TVD (Section 4.3) or on the JSD (Section 5.3.2).  nbr_row[0] is x~."""
     q_ = np.ascontiguousarray(q, dtype=np.float64)
     nb = np.ascontiguousarray(nbr_row, dtype=np.int32)
     moved = ctypes.c_double(0.0)
@@ -133,8 +134,10 @@ class VerifyResult:
 
 def verify(target_logits: np.ndarray, draft_logits: np.ndarray, dtype: int, cfg_scale: float, has_uncond: int,
            T: float, draft_tokens: np.ndarray, tree_parents: Optional[np.ndarray], neighbor_idx: np.ndarray,
-           delta: float, uniforms: np.ndarray, divergence: int = DIV_TVD, top_k: int = 0) -> VerifyResult:
-    """One verification call on host arrays (same layouts as the library's lantern_verify)."""
+           delta: float, uniforms: np.ndarray, divergence: int = DIV_TVD, top_k: int = 0,
+           degenerate_eps: float = DEGENERATE_EPS) -> VerifyResult:
+    """One verification call on host arrays (same layouts as the library's lantern_verify).
+    degenerate_eps: total weight at or below which a residual counts as undefined (reading R10)."""
     tl = np.ascontiguousarray(target_logits)
     dl = np.ascontiguousarray(draft_logits)
     C, B, R, V = tl.shape
@@ -160,17 +163,18 @@ def verify(target_logits: np.ndarray, draft_logits: np.ndarray, dtype: int, cfg_
         _p(par), _p(nb), int(k), ctypes.c_float(delta), int(divergence), int(top_k), _p(un), B, N, V,
         _p(res.accept_len),
         _p(res.next_token), _p(res.accept_path), _p(res.status), _p(res.tested), _p(res.qa), _p(res.px),
-        _p(res.m), _p(res.margin), _p(res.w), _p(res.draw_margin), _p(res.qa_mag))
+        _p(res.m), _p(res.margin), _p(res.w), _p(res.draw_margin), _p(res.qa_mag), ctypes.c_double(degenerate_eps))
     if rc != 0:
         raise ValueError(f"oracle_verify: bad arguments ({rc})")
     return res
 
 
 def verify_inputs(inp, neighbor_idx: np.ndarray, delta: float, divergence: int = DIV_TVD,
-                  top_k: int = 0) -> VerifyResult:
+                  top_k: int = 0, degenerate_eps: float = DEGENERATE_EPS) -> VerifyResult:
     """Convenience: run `verify` on a lantern_inputs.VerifyInputs bundle."""
     return verify(inp.target_logits, inp.draft_logits, inp.dtype, inp.cfg_scale, inp.has_uncond, inp.T,
-                  inp.draft_tokens, inp.tree_parents, neighbor_idx, delta, inp.uniforms, divergence, top_k)
+                  inp.draft_tokens, inp.tree_parents, neighbor_idx, delta, inp.uniforms, divergence, top_k,
+                  degenerate_eps)
 
 
 @dataclasses.dataclass

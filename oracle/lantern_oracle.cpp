@@ -33,6 +33,11 @@
 //   R7  the uniform r lies in [0,1); accept iff r * p(x~) < sum_A q  (no division).
 //   R8  inverse CDF: the smallest token whose inclusive cumulative weight exceeds
 //       u * (total weight); if rounding leaves none, the largest token of positive weight.
+//   R10 a residual whose total weight does not exceed `degenerate_eps` (1e-5 of the unit mass
+//       unless the caller says otherwise) defines no distribution to draw from: the relaxed
+//       target and the drafter coincide there.  The walk stops at that context, the status
+//       bit is set, and the next token is drawn from the context's own target q -- the one
+//       distribution Algorithm 1 does define for a context (its line after the loop).
 //
 // Parity pins: every exported function is pinned by tests/test_oracle_*.py against closed
 // forms, brute force, a separately written textbook speculative sampler, and Monte-Carlo
@@ -56,7 +61,7 @@ enum {
   ST_BAD_PARENT = 2,       // a parent index not in [-1, own index)
   ST_BAD_UNIFORM = 4,      // a uniform outside [0, 1) or NaN
   ST_NONFINITE = 8,        // NaN / +inf logit or empty softmax in a visited context
-  ST_DEGENERATE = 16,      // residual with zero total weight
+  ST_DEGENERATE = 16,      // residual of (near) zero total weight: next token drawn from q (R10)
   ST_BAD_TABLE = 32        // a neighbour entry outside [0, V)
 };
 
@@ -183,7 +188,7 @@ int oracle_build_neighbors_rows(const float* codebook, int V, int D, int k, cons
 }
 
 // ---------------------------------------------------------------------------------------
-// Cosine variant of the latent proximity (Section 6.2.1): every code is scaled to unit length
+// Cosine variant of the latent proximity (Section 5.3.1): every code is scaled to unit length
 // and B_k is then built on the scaled codes with the same distance routine -- on unit vectors
 // the squared distance is 2 - 2 cos, so the order is that of decreasing cosine similarity.
 // Canonical fp32 sequence: squared norm accumulated in dimension order with one fused
@@ -274,7 +279,7 @@ int oracle_a_set(const double* q, int V, const int32_t* nbr_row, int k, double d
 
 // ---------------------------------------------------------------------------------------
 // Jensen-Shannon divergence (natural logarithm) between q and q_{k,delta}(.|D = x~) when A
-// holds x~ with q(x~) = q0 and further tokens of total mass S (Section 6.2.2 names the
+// holds x~ with q(x~) = q0 and further tokens of total mass S (Section 5.3.2 names the
 // divergence; the formula is its definition written out on the only tokens where the two
 // distributions differ).  With mid = (q + q')/2:
 //   a token y of A other than x~ has q' = 0, mid = q(y)/2: it adds q(y) ln 2;
@@ -354,7 +359,8 @@ static void top_k_filter(std::vector<float>& z, int K) {
 //   tr_qa      sum of the current target over A_{k,delta}(x~)
 //   tr_px      current drafter probability of x~
 //   tr_m       |A_{k,delta}(x~)| - 1
-//   tr_margin  min(|r - qa/px|, cut margin)      (distance of the node's decisions to flipping)
+//   tr_margin  min(|r - qa/px|, cut margin, |W - degenerate_eps| after a rejection)
+//              (distance of the node's decisions to flipping)
 //   tr_qa_mag  magnitude of the terms qa was formed from: equal to qa for the first child of a
 //              context; after sibling rejections the target is a difference (q' - p')/W, and this
 //              is the sum over A of the minuend-plus-subtrahend magnitudes carried through the
@@ -365,16 +371,17 @@ static void top_k_filter(std::vector<float>& z, int K) {
 // Returns 0 or a negative code for bad arguments.
 // ---------------------------------------------------------------------------------------
 // oracle_verify_ex adds the variants: `divergence` (DIV_TVD: Section 4.3 as written; DIV_JSD:
-// Section 6.2.2's alternative bound) and `top_k` (Appendix B.2's logit filter; 0 = none).
+// Section 5.3.2's alternative bound), `top_k` (Appendix B.2's logit filter; 0 = none) and
+// `degenerate_eps` (R10's threshold on a residual's total weight, in units of the unit mass).
 int oracle_verify_ex(const void* target_logits, const void* draft_logits, int dtype, float cfg_scale,
                      int has_uncond, float T, const int32_t* draft_tokens, const int32_t* tree_parents,
                      const int32_t* neighbor_idx, int k, float delta_f, int divergence, int top_k,
                      const float* uniforms, int B, int N, int V, int32_t* out_accept_len,
                      int32_t* out_next_token, int32_t* out_accept_path, int32_t* out_status, uint8_t* tr_tested,
                      double* tr_qa, double* tr_px, int32_t* tr_m, double* tr_margin, double* tr_w,
-                     double* tr_draw_margin, double* tr_qa_mag) {
+                     double* tr_draw_margin, double* tr_qa_mag, double degenerate_eps) {
   if (B < 0 || N < 0 || V < 1 || k < 1 || k > V) return -2;
-  if (!(T > 0.0f) || !(delta_f >= 0.0f)) return -3;
+  if (!(T > 0.0f) || !(delta_f >= 0.0f) || !(degenerate_eps >= 0.0)) return -3;
   if ((divergence != DIV_TVD && divergence != DIV_JSD) || top_k < 0) return -3;
   if (B == 0) return 0;
   if (!target_logits || !neighbor_idx || !uniforms || !out_accept_len || !out_next_token) return -1;
@@ -387,7 +394,7 @@ int oracle_verify_ex(const void* target_logits, const void* draft_logits, int dt
   const size_t branch = static_cast<size_t>(B) * R * rowsz;  // elements per guidance branch
 
   std::vector<float> z(V);
-  std::vector<double> q, p, w(V), mag(V);
+  std::vector<double> q, q_ctx, p, w(V), mag(V);
   std::vector<std::vector<int>> kids(R);
 
   for (int b = 0; b < B; ++b) {
@@ -460,6 +467,7 @@ int oracle_verify_ex(const void* target_logits, const void* draft_logits, int dt
 
       int accepted = -1;
       bool degenerate = false;
+      q_ctx = q;  // the context's own target, kept for R10
       if (tr_qa_mag) mag.assign(q.begin(), q.end());
       for (int c : kids[cur]) {
         const int32_t xt = draft_tokens[static_cast<size_t>(b) * N + c];
@@ -505,9 +513,12 @@ int oracle_verify_ex(const void* target_logits, const void* draft_logits, int dt
           W += w[x];
         }
         if (tr_w) tr_w[b] = W;
-        if (!(W > 0.0)) {
-          // Cannot occur in exact arithmetic (a rejection leaves at least p(x~) - sum_A q of
-          // residual mass); if rounding produces it, the step ends here with no token.
+        if (tr_margin) tr_margin[o] = std::min(tr_margin[o], std::fabs(W - degenerate_eps));
+        if (!(W > degenerate_eps)) {
+          // R10.  A rejection of a token the drafter could have produced leaves at least
+          // p(x~) - sum_A q of residual mass, so this is reached only through a drafted token
+          // outside the drafter's support with target and drafter equal elsewhere, or through
+          // two distributions that agree to within the threshold.
           status |= ST_DEGENERATE;
           degenerate = true;
           break;
@@ -525,7 +536,12 @@ int oracle_verify_ex(const void* target_logits, const void* draft_logits, int dt
           std::fill(p.begin(), p.end(), 0.0);
         }
       }
-      if (degenerate) break;  // next_token stays -1
+      if (degenerate) {  // R10: no residual to draw from; the context's own target serves
+        double mg;
+        next_token = inverse_cdf(q_ctx, u_final, &mg);
+        if (tr_draw_margin) tr_draw_margin[b] = mg;
+        break;
+      }
       if (accepted >= 0) {
         if (path) path[accept_len] = accepted;
         ++accept_len;
@@ -673,7 +689,7 @@ int oracle_verify(const void* target_logits, const void* draft_logits, int dtype
   return oracle_verify_ex(target_logits, draft_logits, dtype, cfg_scale, has_uncond, T, draft_tokens, tree_parents,
                           neighbor_idx, k, delta_f, DIV_TVD, 0, uniforms, B, N, V, out_accept_len, out_next_token,
                           out_accept_path, out_status, tr_tested, tr_qa, tr_px, tr_m, tr_margin, tr_w,
-                          tr_draw_margin, tr_qa_mag);
+                          tr_draw_margin, tr_qa_mag, 1e-5);
 }
 
 int oracle_verify_greedy(const void* target_logits, int dtype, float cfg_scale, int has_uncond,

@@ -17,8 +17,7 @@ ST_BAD_TOKEN, ST_BAD_PARENT, ST_BAD_UNIFORM, ST_NONFINITE, ST_DEGENERATE, ST_BAD
     1, 2, 4, 8, 16, 32, 64
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-# LANTERN_LIBRARY may point at another build of the same library (e.g. an instrumented one)
-_LIB_PATH = os.environ.get("LANTERN_LIBRARY", os.path.join(_HERE, "liblantern.so"))
+_LIB_PATH = os.path.join(_HERE, "liblantern.so")
 _lib = None
 
 
@@ -50,13 +49,19 @@ def load_library():
     lib.lantern_build_neighbors.restype = i32
     lib.lantern_build_neighbors.argtypes = [vp, i32, i32, i32, vp, vp, vp, sz, vp]
     lib.lantern_verify_workspace_bytes.restype = sz
-    lib.lantern_verify_workspace_bytes.argtypes = [i32, i32]
+    lib.lantern_verify_workspace_bytes.argtypes = [i32, i32, i32, i32, i32]
+    lib.lantern_last_status.restype = i32
+    lib.lantern_last_status.argtypes = [vp, vp, vp]
+    lib.lantern_verify_counts.restype = i32
+    lib.lantern_verify_counts.argtypes = [vp, vp, vp]
+    lib.lantern_debug_wait_test.restype = i32
+    lib.lantern_debug_wait_test.argtypes = [i32, i32]
     lib.lantern_build_workspace_bytes_metric.restype = sz
     lib.lantern_build_workspace_bytes_metric.argtypes = [i32, i32, i32, i32]
     lib.lantern_build_neighbors_metric.restype = i32
     lib.lantern_build_neighbors_metric.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, sz, vp]
     lib.lantern_verify_workspace_bytes_ex.restype = sz
-    lib.lantern_verify_workspace_bytes_ex.argtypes = [i32, i32, i32]
+    lib.lantern_verify_workspace_bytes_ex.argtypes = [i32, i32, i32, i32, i32, i32]
     lib.lantern_aggregate_all.restype = i32
     lib.lantern_aggregate_all.argtypes = [vp, i32, f32, i32, f32, vp, i32, f32, i32, i32, vp, vp, vp, vp]
     lib.lantern_verify_ex.restype = i32
@@ -65,7 +70,7 @@ def load_library():
     lib.lantern_kernel_revision.restype = i32
     lib.lantern_kernel_revision.argtypes = []
     lib.lantern_verify_launch_count.restype = i32
-    lib.lantern_verify_launch_count.argtypes = []
+    lib.lantern_verify_launch_count.argtypes = [i32, i32]
     lib.lantern_verify_static.restype = i32
     lib.lantern_verify_static.argtypes = [vp, vp, i32, f32, i32, f32, vp, vp, vp, i32, f32, vp, i32, i32, i32,
                                           vp, vp, vp, vp, vp, vp, vp, vp]
@@ -129,8 +134,40 @@ def build_neighbors(codebook: torch.Tensor, k: int, *, with_dist: bool = True, m
     return idx, dist
 
 
-def verify_workspace_bytes(B: int, N: int, top_k: int = 0) -> int:
-    return int(load_library().lantern_verify_workspace_bytes_ex(B, N, int(top_k)))
+def verify_workspace_bytes(B: int, N: int, V: int = 16384, k: int = 1, dtype: int = BF16, top_k: int = 0) -> int:
+    """lantern_verify_workspace_bytes_ex: scratch bytes of one verify() call (0 for a refused shape)."""
+    return int(load_library().lantern_verify_workspace_bytes_ex(B, N, V, k, dtype, int(top_k)))
+
+
+E_DATA = -6
+
+
+def last_status(workspace: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> int:
+    """lantern_last_status: OR of the status bits of every sequence of the last verify() call that used
+    `workspace` (0 = none); waits for the stream."""
+    bits = ctypes.c_int32(0)
+    with torch.cuda.device(workspace.device):
+        rc = load_library().lantern_last_status(_ptr(workspace), _stream_ptr(stream), ctypes.byref(bits))
+    if rc not in (0, E_DATA):
+        raise LanternError(rc, "lantern_last_status")
+    return int(bits.value)
+
+
+def verify_counts(workspace: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> dict:
+    """lantern_verify_counts: work accounting of the last verify() call that used `workspace`."""
+    out = (ctypes.c_int64 * 4)()
+    with torch.cuda.device(workspace.device):
+        rc = load_library().lantern_verify_counts(_ptr(workspace), _stream_ptr(stream), out)
+    if rc != 0:
+        raise LanternError(rc, "lantern_verify_counts")
+    return dict(contexts=int(out[0]), evaluated=int(out[1]), skipped=int(out[2]), from_q=int(out[3]))
+
+
+def debug_wait_test(max_tries: int = 0, withhold_context: int = -1) -> None:
+    """lantern_debug_wait_test: self-test hook of the bounded waits (0, -1 restores the defaults)."""
+    rc = load_library().lantern_debug_wait_test(int(max_tries), int(withhold_context))
+    if rc != 0:
+        raise LanternError(rc, "lantern_debug_wait_test")
 
 
 @dataclasses.dataclass
@@ -155,7 +192,7 @@ def verify(target_logits: torch.Tensor, draft_logits: Optional[torch.Tensor], cf
     draft_logits [B, N+1, V]; draft_tokens / tree_parents [B, N] int32 (tree_parents None = chain);
     neighbor_idx [V, k] int32; uniforms [B, N+1] fp32.  Outputs are allocated unless `out` is given.
     T == 0 selects greedy decoding: draft_logits and uniforms are not read and may be None.
-    divergence "tvd" | "jsd": what delta bounds (Section 6.2.2); top_k: logit filter, 0 = off (Appendix B.2).
+    divergence "tvd" | "jsd": what delta bounds (Section 5.3.2); top_k: logit filter, 0 = off (Appendix B.2).
     """
     if divergence not in DIVERGENCES:
         raise ValueError(f"divergence must be one of {sorted(DIVERGENCES)}")
@@ -185,7 +222,7 @@ def verify(target_logits: torch.Tensor, draft_logits: Optional[torch.Tensor], cf
                 node_qa=torch.empty((B, N), dtype=torch.float32, device=dev) if trace else None,
                 node_px=torch.empty((B, N), dtype=torch.float32, device=dev) if trace else None,
                 node_m=torch.empty((B, N), **i32) if trace else None)
-        need = verify_workspace_bytes(B, N, top_k)
+        need = verify_workspace_bytes(B, N, V, int(k), dtype, top_k)
         if workspace is None:
             workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
         rc = lib.lantern_verify_ex(
@@ -226,9 +263,9 @@ def aggregate_all(logits: torch.Tensor, cfg_scale: float, T: float, neighbor_idx
     return agg, m, status
 
 
-def verify_launch_count() -> int:
-    """Stream operations (4 kernels + 1 memset) enqueued by one verify() call."""
-    return int(load_library().lantern_verify_launch_count())
+def verify_launch_count(greedy: bool = False, top_k_active: bool = False) -> int:
+    """Stream operations (kernels + 1 memset) enqueued by one verify() call."""
+    return int(load_library().lantern_verify_launch_count(int(greedy), int(top_k_active)))
 
 
 def profile_events(before: Optional[torch.cuda.Event], after: Optional[torch.cuda.Event]) -> None:
@@ -244,18 +281,18 @@ def profile_events(before: Optional[torch.cuda.Event], after: Optional[torch.cud
         raise LanternError(rc, "lantern_verify_profile_events")
 
 
-STATIC_WORKSPACE_BYTES = 4 << 20
+STATIC_WORKSPACE_BYTES = 6 << 20
 
 
 def verify_static(target_logits: torch.Tensor, draft_logits: Optional[torch.Tensor], cfg_scale: float, T: float,
                   draft_tokens: Optional[torch.Tensor], tree_parents: Optional[torch.Tensor],
-                  neighbor_idx: torch.Tensor, delta: float, uniforms: torch.Tensor, *, out: VerifyOutputs,
+                  neighbor_idx: torch.Tensor, delta: float, uniforms: Optional[torch.Tensor], *, out: VerifyOutputs,
                   stream: Optional[torch.cuda.Stream] = None) -> VerifyOutputs:
     """lantern_verify_static: verify() for callers that must not allocate device memory.
 
-    The library's scratch comes from a fixed 4 MiB array inside its device image, so nothing is
+    The library's scratch comes from a fixed 6 MiB array inside its device image, so nothing is
     allocated here either: the caller passes every output tensor in `out` (allocated whenever it was
-    still allowed to).  The call is refused (LanternError, code -4) if verify_workspace_bytes(B, N)
+    still allowed to).  The call is refused (LanternError, code -4) if verify_workspace_bytes(B, N, V, k)
     exceeds STATIC_WORKSPACE_BYTES.  Calls on one device share the array: do not let two of them run
     on the GPU at the same time.  Make the first call on a device outside stream capture."""
     lib = load_library()

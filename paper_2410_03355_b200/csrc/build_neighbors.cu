@@ -329,7 +329,7 @@ extern "C" lantern_status lantern_build_neighbors(const float* codebook, int V, 
 }
 
 // ---------------------------------------------------------------------------------------
-// Cosine variant of the latent proximity (Section 6.2.1): codes scaled to unit length, then the
+// Cosine variant of the latent proximity (Section 5.3.1): codes scaled to unit length, then the
 // same neighbour build -- on unit vectors the squared distance is 2 - 2 cos, so increasing
 // distance is decreasing cosine similarity.  One thread per code runs the canonical fp32
 // sequence: squared norm by one fused multiply-add per dimension in dimension order, one square

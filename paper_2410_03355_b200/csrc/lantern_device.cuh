@@ -32,7 +32,7 @@ __device__ __forceinline__ double warp_incl_scan(double v, int lane) {
 }
 
 // ---------------------------------------------------------------------------------------
-// JSD bound (Section 6.2.2).  Moving mass S onto a token of probability q0 changes the
+// JSD bound (Section 5.3.2).  Moving mass S onto a token of probability q0 changes the
 // distribution by JSD (natural logarithm; only the collapsed tokens contribute)
 //   f(S) = 1/2 [ S ln 2 + q0 ln(1 - x) + (q0 + S) ln(1 + x) ],   x = S / (2 q0 + S),
 // since (q0 + S) / mid = 1 + x and q0 / mid = 1 - x for mid = q0 + S/2.  f is increasing and

@@ -21,12 +21,22 @@
 // than eight terms and every threshold comparison is done in double precision.
 #include "verify_common.cuh"
 
+#include <stddef.h>
+
 namespace lantern {
 
 // ---------------------------------------------------------------------------------------
 // kernel 1: plan.  One warp per sequence: validate tokens / parents / uniforms, bucket the
-// nodes by parent context (children in node order), initialise the per-node outputs, mark
-// childless contexts, and append one self-contained work item per context with children.
+// nodes by parent context (children in node order), initialise the per-node outputs, and write
+// one self-contained work item per context with children.
+//
+// Work items are laid out so that the fused pass meets a sequence's contexts in the order
+// Algorithm 1's loop can reach them: slot r * B + b holds the r-th context with children of
+// sequence b in breadth-first order (by depth, then by index).  A context whose parent node has
+// already been rejected when its turn comes is never evaluated (see verify_context.cuh); the
+// order only decides how often that is known in time, never the result.
+// Every context with children starts with a record that says "not evaluated" (INTERNAL), which
+// the fused pass overwrites; contexts without children are marked as leaves.
 // ---------------------------------------------------------------------------------------
 constexpr int PLAN_WARPS = 4;
 
@@ -35,10 +45,12 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b = blockIdx.x * PLAN_WARPS + warp;
   if (b >= P.B) return;
-  const int N = P.N, R = P.R;
-  int* cnt = plan_smem + warp * 2 * (R + 1);   // cnt[c]: number of children of context c
+  const int N = P.N, R = P.R, B = P.B;
+  int* cnt = plan_smem + warp * 4 * (R + 1);   // cnt[c]: number of children of context c
   int* cur = cnt + (R + 1);                    // fill cursor, ends as the end offset of context c
-  for (int i = lane; i <= R; i += 32) cnt[i] = 0;
+  int* dep = cur + (R + 1);                    // depth of context c (root = 0)
+  int* dst = dep + (R + 1);                    // per depth: next breadth-first rank
+  for (int i = lane; i <= R; i += 32) cnt[i] = 0, dst[i] = 0;
   __syncwarp();
   int status = 0;
   const float qnan = __int_as_float(0x7fc00000);
@@ -60,28 +72,47 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
       if (!(r >= 0.0f && r < 1.0f)) status |= LANTERN_ST_BAD_UNIFORM;
     }
   }
+  for (int c = lane; c < R; c += 32) P.dead[static_cast<size_t>(b) * R + c] = 0;
   status = __reduce_or_sync(kFull, status);
   __syncwarp();
   if (lane == 0) P.seq_status[b] = status;
-  if (status) return;   // the walk reports the fault; no work is queued for this sequence
+  if (status) {   // the walk reports the fault; no work is queued for this sequence
+    for (int r = lane; r < N; r += 32) P.work[static_cast<size_t>(r) * B + b].item = -1;
+    return;
+  }
 
   ChildInfo* kids = P.children + static_cast<size_t>(b) * N;
-  if (lane == 0) {      // children of each context, in node order
+  int n_ctx = 0;
+  if (lane == 0) {      // children of each context in node order; depths; breadth-first ranks
     int run = 0;
     for (int c = 0; c < R; ++c) {
       cur[c] = run;
       run += cnt[c];
     }
+    dep[0] = 0;
     for (int i = 0; i < N; ++i) {
       const size_t o = static_cast<size_t>(b) * N + i;
       const int par = P.parents ? P.parents[o] : i - 1;
       ChildInfo ci = {i, P.tokens[o], P.uniforms ? P.uniforms[static_cast<size_t>(b) * R + i] : 0.0f, 0};
       kids[cur[par + 1]++] = ci;
+      dep[i + 1] = dep[par + 1] + 1;
     }
+    for (int c = 0; c < R; ++c)
+      if (cnt[c] > 0) ++dst[dep[c]];          // contexts with children per depth
+    for (int d = 0; d < R; ++d) {             // exclusive prefix: first rank of each depth
+      const int n = dst[d];
+      dst[d] = n_ctx;
+      n_ctx += n;
+    }
+    for (int c = 0; c < R; ++c)
+      if (cnt[c] > 0) dep[c] = dst[dep[c]]++; // dep[c] becomes the context's rank
+    if (n_ctx > 0) atomicMax(&P.counters->n_rank, n_ctx);
   }
-  __syncwarp();         // lane 0's writes to cur[] and kids[] are visible to the warp
+  n_ctx = __shfl_sync(kFull, n_ctx, 0);
+  __syncwarp();         // lane 0's writes to cur[], dep[] and kids[] are visible to the warp
+  for (int r = n_ctx + lane; r < N; r += 32) P.work[static_cast<size_t>(r) * B + b].item = -1;
   const float u_final = P.uniforms ? P.uniforms[static_cast<size_t>(b) * R + N] : 0.0f;
-  const int cap = P.B * N;
+  const int cap = B * N;
   for (int base = 0; base < R; base += 32) {
     const int c = base + lane;
     const int n = c < R ? cnt[c] : 0;
@@ -100,11 +131,14 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
         Record leaf = {kLeaf, -1, 0, 0};
         P.records[static_cast<size_t>(b) * R + c] = leaf;
       } else {
+        Record pending = {-1, -1, LANTERN_ST_INTERNAL, 0};   // stands until the fused pass has evaluated the context
+        P.records[static_cast<size_t>(b) * R + c] = pending;
         const int start = cur[c] - n;
         const ChildInfo f = kids[start];
         WorkItem w = {b * R + c, b * N + start, n, f.node, f.token, f.r, u_final, 0};
-        const int slot = n >= 2 ? hb + __popc(heavy & below) : cap - 1 - (lb + __popc(light & below));
+        const int slot = dep[c] * B + b;
         P.work[slot] = w;
+        P.ctx_slots[n >= 2 ? hb + __popc(heavy & below) : cap - 1 - (lb + __popc(light & below))] = slot;
       }
     }
   }
@@ -134,15 +168,26 @@ __global__ void __launch_bounds__(128) lantern_walk_kernel(VerifyParams P) {
     int cur = 0;
     for (int step = 0; step <= N; ++step) {
       const Record rec = P.records[static_cast<size_t>(b) * R + cur];
-      if (rec.accepted == kLeaf) {   // no drafts left on this path: bonus token from q
+      bool from_q = rec.accepted == kLeaf;   // no drafts left on this path: bonus token from q
+      if (!from_q) {
+        status |= rec.status;
+        // a residual without weight: the next token comes from the context's own target as well
+        from_q = (rec.status & LANTERN_ST_DEGENERATE) && !(rec.status & (LANTERN_ST_NONFINITE | LANTERN_ST_INTERNAL));
+      }
+      if (from_q) {
         const int slot = atomicAdd(&P.counters->n_bonus, 1);
         P.bonus_seq[slot] = b;
         P.bonus_ctx[slot] = cur;
         break;
       }
-      status |= rec.status;
-      if (rec.status & (LANTERN_ST_NONFINITE | LANTERN_ST_DEGENERATE | LANTERN_ST_INTERNAL)) break;
+      if (rec.status & (LANTERN_ST_NONFINITE | LANTERN_ST_INTERNAL)) break;
       if (rec.accepted >= 0) {
+        // an accepted node is a child of this context: its index is at least the context's, and the path
+        // holds at most N nodes; anything else is not a record the fused pass wrote
+        if (rec.accepted < cur || rec.accepted >= N || len >= N) {
+          status |= LANTERN_ST_INTERNAL;
+          break;
+        }
         if (P.out_path) P.out_path[static_cast<size_t>(b) * N + len] = rec.accepted;
         ++len;
         cur = rec.accepted + 1;
@@ -155,6 +200,7 @@ __global__ void __launch_bounds__(128) lantern_walk_kernel(VerifyParams P) {
   P.out_len[b] = len;
   P.out_tok[b] = next;
   if (P.out_status) P.out_status[b] = status;
+  if (status) atomicOr(&P.counters->status_or, status);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -163,17 +209,20 @@ __global__ void __launch_bounds__(128) lantern_walk_kernel(VerifyParams P) {
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WsLayout {
-  size_t counters, work, children, records, seqst, bseq, bctx, thrq, thrp, total;
+  size_t counters, work, slots, children, records, dead, seqst, bseq, bctx, thrq, thrp, total;
 };
 
 static WsLayout ws_layout(int B, int N, bool topk = false) {
   const size_t R = static_cast<size_t>(N) + 1, b = static_cast<size_t>(B);
+  const size_t n1 = N > 0 ? N : 1;
   WsLayout L;
   size_t o = 0;
   L.counters = o; o += 256;
-  L.work = o;     o += align_up(b * (N > 0 ? N : 1) * sizeof(WorkItem), 256);
-  L.children = o; o += align_up(b * (N > 0 ? N : 1) * sizeof(ChildInfo), 256);
+  L.work = o;     o += align_up(b * n1 * sizeof(WorkItem), 256);
+  L.slots = o;    o += align_up(b * n1 * 4, 256);
+  L.children = o; o += align_up(b * n1 * sizeof(ChildInfo), 256);
   L.records = o;  o += align_up(b * R * sizeof(Record), 256);
+  L.dead = o;     o += align_up(b * R, 256);
   L.seqst = o;    o += align_up(b * 4, 256);
   L.bseq = o;     o += align_up(b * 4, 256);
   L.bctx = o;     o += align_up(b * 4, 256);
@@ -184,6 +233,11 @@ static WsLayout ws_layout(int B, int N, bool topk = false) {
 }
 
 static thread_local cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
+
+// limit of the kernels' bounded waits and the self-test's withheld context (lantern_debug_wait_test)
+constexpr uint32_t kDefaultWaitTries = 1u << 21;
+static thread_local uint32_t g_wait_tries = kDefaultWaitTries;
+static thread_local int g_withhold_item = -1;
 
 // thresholds of the top-k filter: mode 0 = rows of the contexts with children (after the plan),
 // mode 1 = rows of the bonus draws (after the walk)
@@ -299,12 +353,53 @@ static cudaError_t launch_greedy(const VerifyParams& P, long long items, int sms
 
 using namespace lantern;
 
-extern "C" size_t lantern_verify_workspace_bytes(int B, int N) {
-  if (B < 0 || N < 0 || N > MAX_N) return 0;
+static bool shape_ok(int B, int N, int V, int k, int dtype) {
+  if (dtype != LANTERN_F32 && dtype != LANTERN_BF16) return false;
+  if (B < 0 || N < 0 || N > MAX_N || V < 8 || V > 16384 || (V % 8) != 0 || k < 1 || k > V) return false;
+  return static_cast<long long>(B) * (N + 1) < (1ll << 31);
+}
+
+extern "C" size_t lantern_verify_workspace_bytes(int B, int N, int V, int k, int dtype) {
+  if (!shape_ok(B, N, V, k, dtype)) return 0;
   return ws_layout(B > 0 ? B : 1, N).total;
 }
 
-extern "C" int lantern_verify_launch_count(void) { return 5; }
+extern "C" int lantern_verify_launch_count(int greedy, int top_k_active) {
+  // memset, plan, fused pass (or greedy pass), walk, bonus; with the filter one threshold kernel ahead of
+  // the pass and, in sampling, one more ahead of the bonus draw
+  return 5 + (top_k_active ? (greedy ? 1 : 2) : 0);
+}
+
+extern "C" lantern_status lantern_last_status(const void* workspace, void* cuda_stream, int32_t* out_bits) {
+  if (!workspace) return LANTERN_E_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int32_t bits = 0;
+  const unsigned char* c = static_cast<const unsigned char*>(workspace) + offsetof(Counters, status_or);
+  if (cudaMemcpyAsync(&bits, c, sizeof(bits), cudaMemcpyDeviceToHost, st) != cudaSuccess) return LANTERN_E_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return LANTERN_E_CUDA;
+  if (out_bits) *out_bits = bits;
+  return bits ? LANTERN_E_DATA : LANTERN_OK;
+}
+
+extern "C" lantern_status lantern_verify_counts(const void* workspace, void* cuda_stream, int64_t* out_counts) {
+  if (!workspace || !out_counts) return LANTERN_E_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  Counters c;
+  if (cudaMemcpyAsync(&c, workspace, sizeof(c), cudaMemcpyDeviceToHost, st) != cudaSuccess) return LANTERN_E_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return LANTERN_E_CUDA;
+  out_counts[0] = static_cast<int64_t>(c.n_heavy) + c.n_light;
+  out_counts[1] = c.n_evaluated;
+  out_counts[2] = c.n_skipped;
+  out_counts[3] = c.n_bonus;
+  return LANTERN_OK;
+}
+
+extern "C" lantern_status lantern_debug_wait_test(int max_tries, int withhold_context) {
+  if (max_tries < 0) return LANTERN_E_PARAM;
+  g_wait_tries = max_tries == 0 ? kDefaultWaitTries : static_cast<uint32_t>(max_tries);
+  g_withhold_item = withhold_context;
+  return LANTERN_OK;
+}
 
 extern "C" int lantern_kernel_revision(void) { return LANTERN_CONTEXT_KERNEL_REVISION; }
 
@@ -337,8 +432,8 @@ extern "C" lantern_status lantern_verify(const void* target_logits, const void* 
                            workspace, workspace_bytes, cuda_stream);
 }
 
-extern "C" size_t lantern_verify_workspace_bytes_ex(int B, int N, int top_k) {
-  if (B < 0 || N < 0 || N > MAX_N || top_k < 0) return 0;
+extern "C" size_t lantern_verify_workspace_bytes_ex(int B, int N, int V, int k, int dtype, int top_k) {
+  if (!shape_ok(B, N, V, k, dtype) || top_k < 0) return 0;
   return ws_layout(B > 0 ? B : 1, N, top_k > 0).total;
 }
 
@@ -425,6 +520,10 @@ static lantern_status verify_impl(const void* target_logits, const void* draft_l
   P.top_k = topk ? top_k : 0;
   P.thr_q = topk ? reinterpret_cast<float*>(ws + L.thrq) : nullptr;
   P.thr_p = topk ? reinterpret_cast<float*>(ws + L.thrp) : nullptr;
+  P.ctx_slots = reinterpret_cast<int32_t*>(ws + L.slots);
+  P.dead = ws + L.dead;
+  P.wait_tries = g_wait_tries;
+  P.withhold_item = g_withhold_item;
 
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return LANTERN_E_CUDA;
@@ -432,7 +531,11 @@ static lantern_status verify_impl(const void* target_logits, const void* draft_l
   if (sms < 1) return LANTERN_E_CUDA;
 
   if (cudaMemsetAsync(P.counters, 0, 256, st) != cudaSuccess) return LANTERN_E_CUDA;
-  const size_t plan_smem = static_cast<size_t>(PLAN_WARPS) * 2 * (N + 2) * sizeof(int);
+  const size_t plan_smem = static_cast<size_t>(PLAN_WARPS) * 4 * (N + 2) * sizeof(int);
+  if (plan_smem > 48 * 1024 &&
+      cudaFuncSetAttribute(lantern_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           static_cast<int>(plan_smem)) != cudaSuccess)
+    return LANTERN_E_CUDA;
   lantern_plan_kernel<<<(B + PLAN_WARPS - 1) / PLAN_WARPS, PLAN_WARPS * 32, plan_smem, st>>>(P);
   if (cudaGetLastError() != cudaSuccess) return LANTERN_E_CUDA;
 
@@ -474,7 +577,8 @@ static void* g_static_workspace_ptr[64] = {};
 
 static lantern_status static_workspace_address(void** out) {
   int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return LANTERN_E_CUDA;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) return LANTERN_E_CUDA;
+  if (dev >= 64) return LANTERN_E_SHAPE;   // the table of addresses below serves ordinals 0..63
   void* p = __atomic_load_n(&g_static_workspace_ptr[dev], __ATOMIC_ACQUIRE);
   if (!p) {
     if (cudaGetSymbolAddress(&p, g_static_workspace) != cudaSuccess || !p) return LANTERN_E_CUDA;
@@ -514,6 +618,7 @@ extern "C" const char* lantern_status_string(lantern_status s) {
     case LANTERN_E_PARAM: return "a scalar parameter is invalid";
     case LANTERN_E_WORKSPACE: return "workspace missing, too small or misaligned";
     case LANTERN_E_CUDA: return "a CUDA runtime call failed";
+    case LANTERN_E_DATA: return "a fault in the data was found on the device (see out_status)";
     case LANTERN_E_ALIGN: return "a pointer is not 16-byte aligned";
     case LANTERN_E_UNIMPLEMENTED: return "not implemented in this build";
     default: return "unknown status";

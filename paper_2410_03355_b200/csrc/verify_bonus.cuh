@@ -78,7 +78,7 @@ __global__ void __launch_bounds__(BNT, 3) lantern_bonus_stream_kernel(VerifyPara
     float tq = 0.0f;
     if (TOPK) tq = __ldg(P.thr_q + item);
     const double u = static_cast<double>(P.uniforms[static_cast<size_t>(b) * R + N]);
-    const bool ok = mbar_wait(bar, it & 1);
+    const bool ok = mbar_wait(bar, it & 1, P.wait_tries);
 
     // ---- sweep 1: maximum ----
     float m = NEG_INF;
@@ -92,10 +92,17 @@ __global__ void __launch_bounds__(BNT, 3) lantern_bonus_stream_kernel(VerifyPara
     if (lane == 0) S.wm[warp] = m;
     const bool any_bad = __syncthreads_or(bad) != 0;
     const bool timeout = __syncthreads_or(ok ? 0 : 1) != 0;
-    if (timeout) {   // the copy did not complete within the wait limit: reported, and the kernel stops
+    if (timeout) {
+      // the copy did not complete within the wait limit: this draw and the CTA's remaining ones are
+      // reported instead of made; the late copy gets one more bounded wait before the CTA leaves
       if (tid == 0) {
-        P.out_tok[b] = -1;
-        if (P.out_status) P.out_status[b] |= LANTERN_ST_INTERNAL;
+        for (int j = i; j < count; j += G) {
+          const int bj = P.bonus_seq[j];
+          P.out_tok[bj] = -1;
+          if (P.out_status) P.out_status[bj] |= LANTERN_ST_INTERNAL;
+        }
+        atomicOr(&P.counters->status_or, LANTERN_ST_INTERNAL);
+        mbar_wait(bar, it & 1, P.wait_tries);
       }
       break;
     }
@@ -215,7 +222,10 @@ __global__ void __launch_bounds__(BNT, 3) lantern_bonus_stream_kernel(VerifyPara
     if (tid == 0) {
       if (i + G < count) greedy_issue_rows<BF16, UNC>(P, item_next, bsm, rowbytes, &S.bar_full);
       P.out_tok[b] = tok;
-      if (st && P.out_status) P.out_status[b] |= st;
+      if (st) {
+        if (P.out_status) P.out_status[b] |= st;
+        atomicOr(&P.counters->status_or, st);
+      }
     }
   }
 }

@@ -16,9 +16,15 @@ constexpr int MAX_N = 1024;
 
 struct Counters {               // first 256 bytes of the workspace, zeroed per call
   int work_next;                // dynamic part of the work counter
-  int n_heavy;                  // contexts with >= 2 children (handed out first)
+  int n_heavy;                  // contexts with >= 2 children (first in the compact list)
   int n_light;                  // contexts with exactly 1 child
-  int n_bonus;                  // sequences whose walk ended on a childless context
+  int n_bonus;                  // sequences whose next token is drawn from a context's own target
+  int n_rank;                   // largest number of contexts with children in one sequence
+  int n_evaluated;              // contexts the fused pass evaluated
+  int n_skipped;                // contexts it left out because the walk cannot reach them
+  int n_tested;                 // drafted nodes it tested
+  int status_or;                // OR of every sequence's status bits (written by the walk and later kernels)
+  int abort;                    // a bounded wait ran out somewhere: no further work is handed out
 };
 
 struct Record {                 // result of one context
@@ -63,7 +69,10 @@ struct VerifyParams {
   int32_t* out_m;
   // workspace pieces
   Counters* counters;
-  WorkItem* work;               // [B*N]: heavy items from the front, light items from the back
+  WorkItem* work;               // [N, B]: slot r * B + b holds the r-th context with children of sequence b in
+                                //         breadth-first order (by depth, then by index); item = -1 where there is none
+  int32_t* ctx_slots;           // [B*N]: the occupied slots, heavy ones from the front, light ones from the back
+  unsigned char* dead;          // [B, R]: 1 once the walk is known not to reach the context
   ChildInfo* children;          // [B, N]
   Record* records;              // [B, R]
   int32_t* seq_status;          // [B]
@@ -75,6 +84,8 @@ struct VerifyParams {
   int top_k;                    // logit filter; 0 = off (then thr_q, thr_p are null)
   float* thr_q;                 // [B, R] top_k-th largest processed target logit of a context row
   float* thr_p;                 // [B, R] the same for the drafter row
+  uint32_t wait_tries;          // limit of every bounded mbarrier wait, in tries
+  int withhold_item;            // self-test only: the copies of this context are never issued (-1 = none)
 };
 
 __device__ __forceinline__ float sum8(const float* v) {

@@ -25,7 +25,15 @@
 // inverse-CDF draw or the write-back for the next sibling.
 #pragma once
 
-#define LANTERN_CONTEXT_KERNEL_REVISION 15   // bump on every change to this file
+// Which contexts are evaluated.  Algorithm 1 stops at the first rejection, so a context behind a
+// rejected node is never tested by the method.  Work items come in breadth-first order per sequence
+// (see the plan kernel); when a context has been decided, its group marks the contexts behind every
+// child it did not accept as dead, and a producer that meets a dead context leaves it out (and marks
+// that context's children in turn).  A context whose parent is still undecided when its turn comes is
+// evaluated anyway: with few sequences per call that keeps every SM busy (all contexts of a tree run
+// side by side), with many sequences it is rare, and the walk kernel reads only records on the
+// accepted path either way, so the result never depends on what was speculated.
+#define LANTERN_CONTEXT_KERNEL_REVISION 16   // bump on every change to this file
 
 namespace lantern {
 
@@ -35,6 +43,10 @@ constexpr int LOG_GT = 8;
 constexpr int NGRP = 2;         // consumer groups per CTA
 constexpr int MAXU = 16;        // (pass, warp) slices of a context, at most
 constexpr int kNone = 0x7fffffff;
+// A residual whose total weight is at most this fraction of the current target's mass defines no
+// distribution to draw from (the single-precision residual pass resolves totals to a few 1e-7 of that
+// mass): the walk stops there and the next token comes from the context's own target.
+constexpr double kDegenerate = 1e-5;
 constexpr int CTX_THREADS = NGRP * GT + NGRP * 32;   // consumers, then one producer warp per group
 
 // Thread t of a group owns, for chunk c, the eight consecutive tokens [(c*GT + t)*8, +8), i.e. 16-byte
@@ -63,10 +75,10 @@ struct GroupShared {
   float fqt[2 * GT];            // factor of every (pass, thread) slice: its units -> common units
   float wmq[GW], wmp[GW];       // per-warp maxima of the slices' shift constants
   int first[GW];                // a warp's first failing neighbour slot
+  int badslot[GW];              // a warp's first neighbour slot with an entry outside [0, V)
   int cand[GW];
   int acc_valid;                // acc_e / acc_p are usable for the current child
   int tok;
-  int status;                   // OR of status bits seen by single threads
   int fail;                     // a bounded wait for the target rows ran out (sticky)
   float thr[2][2];              // top-k thresholds (target, drafter) of the context in work[i]
   WorkItem work[2];             // descriptor of context i in work[i & 1]: the next one is published while the current one runs
@@ -192,7 +204,7 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 
 // CH = 8-token chunks per thread (1, 2, 4 or 8); a thread streams them in NP passes of CP chunks.
 // TONE = the temperature is exactly 1 (the paper's sampling setting): no division is compiled in.
-// JSD selects the Section 6.2.2 bound at compile time, so that the default path carries none of its code.
+// JSD selects the Section 5.3.2 bound at compile time, so that the default path carries none of its code.
 // TOPK applies the per-row thresholds of the top-k logit filter (Appendix B.2; written by
 // lantern_topk_kernel): processed logits below a row's threshold count as -inf.
 template <int CH, bool BF16, bool UNC, bool TONE, bool JSD, bool TOPK>
@@ -220,7 +232,6 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       mbar_init(&bar_full_t[g], 1);
       mbar_init(&bar_empty_d[g], GW);
       mbar_init(&bar_empty_t[g], GW);
-      SG[g].status = 0;
       SG[g].fail = 0;
     }
     fence_mbar_init();
@@ -229,77 +240,167 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
   __syncthreads();
 
   // ======================= producer warps =======================
-  // One thread per consumer group hands out work and keeps that group's copies going.  The first
-  // three items of every producer are dealt statically; from then on a global counter hands them out.
-  // A look-ahead pipeline keeps the global round trips of the work queue off the critical path: while
-  // the group processes context i, the descriptor of i+1 is in registers, that of i+2 is being loaded
-  // and the index of i+3 is being fetched.  The rows of i+1 are copied as soon as the group releases
-  // its staging area.
+  // One warp per consumer group hands out work and keeps that group's copies going.  Its 32 lanes look
+  // at up to 32 consecutive work slots at a time (a batch: the first one dealt statically, later ones
+  // from a global counter, in sizes that shrink towards the end of the list so that the groups finish
+  // together), drop the empty and the dead ones, and lane 0 feeds the rest to the group one by one:
+  // the drafter row as soon as the group has streamed the previous one, the target rows as soon as the
+  // group releases its staging area.  The next batch is loaded while the current one is being worked
+  // on, so that no round trip to the work list is on the critical path.
   if (tid >= NGRP * GT) {
     const int grp = (tid - NGRP * GT) >> 5;
-    if (lane == 0) {
-      GroupShared& S = SG[grp];
-      const int n_heavy = P.counters->n_heavy;
-      const int total = n_heavy + P.counters->n_light;
-      const int cap = P.B * N;
-      const int G = gridDim.x * NGRP;              // producers in the grid
-      const int me = blockIdx.x * NGRP + grp;
-      auto load_item = [&](int w) -> WorkItem {
-        WorkItem it;
-        it.item = -1;
-        it.pad = 0;
-        if (w < total) {
-          const int slot = w < n_heavy ? w : cap - 1 - (w - n_heavy);
-          const int4 lo = __ldg(reinterpret_cast<const int4*>(P.work + slot));
-          const int4 hi = __ldg(reinterpret_cast<const int4*>(P.work + slot) + 1);
-          it.item = lo.x, it.cbase = lo.y, it.nchild = lo.z, it.node0 = lo.w;
-          it.tok0 = hi.x, it.r0 = __int_as_float(hi.y), it.u_final = __int_as_float(hi.z);
+    GroupShared& S = SG[grp];
+    const int total = P.counters->n_rank * P.B;  // occupied part of the slot array
+    const int G = gridDim.x * NGRP;              // producers in the grid
+    const int me = blockIdx.x * NGRP + grp;
+    const uint32_t tries = P.wait_tries;
+    auto batch_size = [&](int at) {
+      const int s = (total - at) / (4 * G);
+      return s < 1 ? 1 : (s > 32 ? 32 : s);
+    };
+    struct Cand {
+      int item, cbase, nchild, node0, tok0;
+      float r0, u_final, tq, tp;
+    };
+    auto load_cand = [&](int start, int size) -> Cand {
+      Cand c;
+      c.item = -1;
+      c.cbase = c.nchild = c.node0 = c.tok0 = 0;
+      c.r0 = c.u_final = c.tq = c.tp = 0.0f;
+      const int w = start + lane;
+      if (lane < size && w < total) {
+        const int4 lo = __ldg(reinterpret_cast<const int4*>(P.work + w));
+        const int4 hi = __ldg(reinterpret_cast<const int4*>(P.work + w) + 1);
+        c.item = lo.x, c.cbase = lo.y, c.nchild = lo.z, c.node0 = lo.w;
+        c.tok0 = hi.x, c.r0 = __int_as_float(hi.y), c.u_final = __int_as_float(hi.z);
+        if (TOPK && c.item >= 0) {   // the context's thresholds travel with its descriptor: (target, drafter)
+          c.tq = __ldg(P.thr_q + c.item);
+          c.tp = __ldg(P.thr_p + c.item);
         }
-        return it;
-      };
-      // top-k thresholds of a context travel with its descriptor: (target, drafter)
-      auto load_thr = [&](const WorkItem& it, float& tq, float& tp) {
-        if (TOPK && it.item >= 0) {
-          tq = __ldg(P.thr_q + it.item);
-          tp = __ldg(P.thr_p + it.item);
+      }
+      return c;
+    };
+    auto is_dead = [&](int item) -> bool {
+      return *reinterpret_cast<const volatile unsigned char*>(P.dead + item) != 0;
+    };
+    // the walk cannot reach a dead context, hence none of the contexts behind its children either
+    auto bury = [&](const Cand& c) {
+      const size_t row0 = static_cast<size_t>(c.item / R) * R;
+      for (int j = 0; j < c.nchild; ++j) {
+        const int node = j == 0 ? c.node0 : __ldg(&P.children[c.cbase + j].node);
+        P.dead[row0 + node + 1] = 1;
+      }
+    };
+    int n_eval = 0, n_skip = 0;
+    // live candidates of a batch, as a lane mask
+    auto filter = [&](const Cand& c) -> unsigned {
+      const bool has = c.item >= 0;
+      const bool dead = has && is_dead(c.item);
+      if (dead) bury(c);
+      n_skip += __popc(__ballot_sync(kFull, dead));
+      return __ballot_sync(kFull, has && !dead);
+    };
+    const int b0 = batch_size(0);
+    Cand cur = load_cand(me * b0, b0);
+    bool cur_end = me * b0 >= total;
+    int seen = G * b0;
+    // start of the next dynamic batch (lane 0 asks, everybody hears)
+    auto grab = [&](int& size) -> int {
+      size = batch_size(seen < total ? seen : total);
+      int st = 0;
+      if (lane == 0) st = G * b0 + atomicAdd(&P.counters->work_next, size);
+      st = __shfl_sync(kFull, st, 0);
+      seen = st;
+      return st;
+    };
+    int nsize = 0;
+    int nstart = grab(nsize);
+    Cand nxt = load_cand(nstart, nsize);
+    bool nxt_end = nstart >= total;
+    unsigned mask = filter(cur);
+    int i = 0;        // contexts handed to the group so far
+    bool clean = true;
+    for (;;) {
+      while (mask == 0 && !cur_end) {
+        cur = nxt;
+        cur_end = nxt_end;
+        if (!cur_end) {
+          nstart = grab(nsize);
+          nxt = load_cand(nstart, nsize);
+          nxt_end = nstart >= total;
         }
-      };
-      float tq_cur = 0.0f, tp_cur = 0.0f, tq_next = 0.0f, tp_next = 0.0f;
-      WorkItem it_cur = load_item(me);
-      WorkItem it_next = load_item(me + G);
-      load_thr(it_cur, tq_cur, tp_cur);
-      load_thr(it_next, tq_next, tp_next);
-      int w_next2 = me + 2 * G;
-      for (int i = 0;; ++i) {
-        // The drafter slot is free once every warp of the group has streamed the previous context's
-        // drafter row (nothing reads it afterwards), i.e. while that context is still being decided:
-        // the next drafter row travels early, and the group streams it while its target rows are copied.
-        if (i >= 1 && !mbar_wait(&bar_empty_d[grp], (i - 1) & 1)) {
-          it_cur.item = -1;
-          it_cur.pad = LANTERN_ST_INTERNAL;   // the group never released its slot: stop handing out work
-        }
-        S.work[i & 1] = it_cur;               // published by the mbarrier operation below
+        mask = filter(cur);
+      }
+      if (mask == 0) break;
+      const int l = __ffs(mask) - 1;
+      mask &= mask - 1;
+      // The drafter slot is free once every warp of the group has streamed the previous context's
+      // drafter row (nothing reads it afterwards), i.e. while that context is still being decided:
+      // the next drafter row travels early, and the group streams it while its target rows are copied.
+      if (i >= 1 && !mbar_wait(&bar_empty_d[grp], (i - 1) & 1, tries)) {
+        clean = false;   // the group never released its slot: it has given up, and so does its producer
+        break;
+      }
+      // as late as possible: has the context died meanwhile, has the call been given up?
+      const int gone = (lane == l && is_dead(cur.item)) ? 1 : 0;
+      const int stop = *reinterpret_cast<const volatile int*>(&P.counters->abort);
+      if (__any_sync(kFull, stop != 0)) break;
+      if (__any_sync(kFull, gone)) {
+        if (lane == l) bury(cur);
+        ++n_skip;
+        continue;
+      }
+      WorkItem it;
+      it.item = __shfl_sync(kFull, cur.item, l);
+      it.cbase = __shfl_sync(kFull, cur.cbase, l);
+      it.nchild = __shfl_sync(kFull, cur.nchild, l);
+      it.node0 = __shfl_sync(kFull, cur.node0, l);
+      it.tok0 = __shfl_sync(kFull, cur.tok0, l);
+      it.r0 = __shfl_sync(kFull, cur.r0, l);
+      it.u_final = __shfl_sync(kFull, cur.u_final, l);
+      it.pad = 0;
+      const float tq_cur = TOPK ? __shfl_sync(kFull, cur.tq, l) : 0.0f;
+      const float tp_cur = TOPK ? __shfl_sync(kFull, cur.tp, l) : 0.0f;
+      // the rows of the context after this one, for the L2 prefetch below
+      const unsigned nraw = __ballot_sync(kFull, nxt.item >= 0);
+      const int item_ahead = mask ? __shfl_sync(kFull, cur.item, __ffs(mask) - 1)
+                                  : (nraw && !cur_end ? __shfl_sync(kFull, nxt.item, __ffs(nraw) - 1) : -1);
+      bool ok = true;
+      if (lane == 0) {
+        S.work[i & 1] = it;                   // published by the mbarrier operation of the copy below
         if (TOPK) {
           S.thr[i & 1][0] = tq_cur;
           S.thr[i & 1][1] = tp_cur;
         }
-        if (it_cur.item < 0) {
-          mbar_arrive(&bar_full_d[grp]);      // wake the group; it sees the terminator
-          break;
-        }
+        const bool withheld = it.item == P.withhold_item;   // self-test of the bounded waits: nothing is copied
         fence_proxy_async();
-        ctx_issue_drafter(P, it_cur.item, smem + grp * stage_bytes, rowbytes, &bar_full_d[grp]);
+        if (!withheld) ctx_issue_drafter(P, it.item, smem + grp * stage_bytes, rowbytes, &bar_full_d[grp]);
         // the target slots (later E) are free once every warp of the group has finished the previous context
-        if (i >= 1 && !mbar_wait(&bar_empty_t[grp], (i - 1) & 1)) break;   // the group's own wait runs out too
-        fence_proxy_async();
-        ctx_issue_target<UNC>(P, it_cur.item, smem + grp * stage_bytes, rowbytes, &bar_full_t[grp]);
-        if (it_next.item >= 0) ctx_prefetch_rows<BF16, UNC>(P, it_next.item, rowbytes);
-        it_cur = it_next;
-        tq_cur = tq_next, tp_cur = tp_next;
-        it_next = load_item(w_next2);
-        load_thr(it_next, tq_next, tp_next);
-        w_next2 = 3 * G + atomicAdd(&P.counters->work_next, 1);
+        if (i >= 1 && !mbar_wait(&bar_empty_t[grp], (i - 1) & 1, tries)) ok = false;
+        if (ok && !withheld) {
+          fence_proxy_async();
+          ctx_issue_target<UNC>(P, it.item, smem + grp * stage_bytes, rowbytes, &bar_full_t[grp]);
+          if (item_ahead >= 0) ctx_prefetch_rows<BF16, UNC>(P, item_ahead, rowbytes);
+        }
       }
+      ok = __shfl_sync(kFull, ok ? 1 : 0, 0) != 0;
+      ++n_eval;
+      ++i;
+      if (!ok) {
+        clean = false;
+        break;
+      }
+    }
+    if (lane == 0) {
+      if (clean) {   // the group is waiting for its next context: hand it the terminator
+        if (i == 0 || mbar_wait(&bar_empty_d[grp], (i - 1) & 1, tries)) {
+          S.work[i & 1].item = -1;
+          __threadfence_block();
+          mbar_arrive(&bar_full_d[grp]);
+        }
+      }
+      if (n_eval) atomicAdd(&P.counters->n_evaluated, n_eval);
+      if (n_skip) atomicAdd(&P.counters->n_skipped, n_skip);
     }
     return;
   }
@@ -351,13 +452,29 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       for (int e = 0; e < 8; ++e) out[e] = __fdiv_rn(out[e], P.T);
     }
   };
+  const uint32_t tries = P.wait_tries;
+  // A bounded wait that runs out ends the group: the context keeps the "not evaluated" record the plan
+  // gave it (the walk reports INTERNAL for a sequence that reaches it), the call is given up (no producer
+  // hands out further work), and one thread gives the copies that may still be on their way into this
+  // group's staging area the same bounded wait before the group leaves.
+  auto give_up = [&](int iter, bool drafter_too) {
+    if (gt == 0) {
+      *reinterpret_cast<volatile int*>(&P.counters->abort) = 1;
+      if (drafter_too) mbar_wait(&bar_full_d[grp], iter & 1, tries);
+      mbar_wait(&bar_full_t[grp], iter & 1, tries);
+      if (!drafter_too) mbar_wait(&bar_full_d[grp], (iter + 1) & 1, tries);   // the next drafter row may be under way
+    }
+  };
   for (int iter = 0;; ++iter) {
     // One warp watches the copy's mbarrier (bounded wait); the group barrier then releases everybody
     // at once and tells every thread alike whether the rows have landed.
     bool landed = true;
-    if (gw == 0) landed = mbar_wait(&bar_full_d[grp], iter & 1);
+    if (gw == 0) landed = mbar_wait(&bar_full_d[grp], iter & 1, tries);
     const bool arrived = gbar_and(grp, landed);
-    if (!arrived) break;   // the copy did not land within the limit; the walk reports the missing record
+    if (!arrived) {   // the drafter row did not land within the limit
+      give_up(iter, true);
+      break;
+    }
     const WorkItem cur = S.work[iter & 1];
     const int item = cur.item;
     if (item < 0) break;
@@ -369,9 +486,6 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
     const int b = item / R;
     const ChildInfo* kids = P.children + cur.cbase;
     const int nchild = cur.nchild;
-    // every thread of the group is past the previous context (its record included): clear the shared
-    // status word; nobody sets it again before the [stats] barrier below
-    if (gt == 0) S.status = 0;
 
     // first child: its neighbour row (four slots per thread) and, for thread 0, its raw logits; issued
     // now, used after the streaming part
@@ -476,7 +590,7 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
     // The target rows were issued when the previous context was released; they arrive while the drafter
     // row is streamed.  Every thread waits for itself (bounded); a wait that runs out is reported after
     // the next group barrier, where every thread sees it alike.
-    if (!mbar_wait(&bar_full_t[grp], iter & 1)) S.fail = 1;
+    if (!mbar_wait(&bar_full_t[grp], iter & 1, tries)) S.fail = 1;
     // --- target: guidance combine, slice maximum, numerators, partial sum; E replaces the raw rows ---
 #pragma unroll
     for (int p = 0; p < NP; ++p) {
@@ -555,7 +669,10 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       }
     }
     gbar(grp);   // [stats 1] per-warp maxima, and E, are visible
-    if (S.fail) break;   // the target rows did not land within the limit; the walk reports the missing record
+    if (S.fail) {   // the target rows did not land within the limit
+      give_up(iter, false);
+      break;
+    }
     mlq_g = S.wmq[0];
     mlp_g = S.wmp[0];
 #pragma unroll
@@ -639,7 +756,7 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
 
         // ---- A_{k,delta}(x~): gather + prefix scan with the strict bound ----
         double thr = delta * Zq_c;   // the bound in the units of the unnormalised sums
-        // Section 6.2.2: the mass whose JSD is delta; one thread, published by [scan 1] through the last
+        // Section 5.3.2: the mass whose JSD is delta; one thread, published by [scan 1] through the last
         // slot of wt[], which nothing else touches between the start of a child and its [scan 2]
         if (JSD && gt == GT - 32)
           S.wt[8 * GW - 1] = jsd_mass_bound(delta, static_cast<double>(e_xt_bulk) / Zq_c) * Zq_c;
@@ -650,13 +767,14 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
           double pre4[4];       // inclusive prefix over this thread's four slots
           bool val4[4];
           double run = 0.0;
+          int my_bad = kNone;   // first of this thread's slots whose entry lies outside [0, V): it carries no mass
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const int j = base + 4 * gt + 1 + i;
             val4[i] = j < k;
             const int n = base == 0 ? nb[i] : (val4[i] ? __ldg(nrow + j) : -1);
             const bool inr = val4[i] && static_cast<unsigned>(n) < static_cast<unsigned>(V);
-            if (val4[i] && !inr) atomicOr(&S.status, LANTERN_ST_BAD_TABLE);   // carries no mass
+            if (val4[i] && !inr && my_bad == kNone) my_bad = j;
             run += inr ? static_cast<double>(E[EI(n)] * S.fqt[owner_slice<LOG_CP>(n)]) : 0.0;
             pre4[i] = run;
           }
@@ -689,8 +807,10 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
           } else if (wfirst == kNone && lane == 0) {
             S.first[gw] = kNone;
           }
+          const int wbad = __reduce_min_sync(kFull, my_bad);
+          if (lane == 0) S.badslot[gw] = wbad;
           gbar(grp);   // [scan 2]
-          int gfirst = kNone, src = 0;
+          int gfirst = kNone, src = 0, gbad = kNone;
 #pragma unroll
           for (int w = GW - 1; w >= 0; --w) {
             const int f = S.first[w];
@@ -698,7 +818,10 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
               gfirst = f;
               src = w;
             }
+            gbad = min(gbad, S.badslot[w]);
           }
+          // a bad entry is reported where Algorithm 2's loop meets it, i.e. ahead of the slot that ends the set
+          if (gbad < gfirst) status |= LANTERN_ST_BAD_TABLE;
           if (gfirst != kNone) {
             m = gfirst - 1;
             sm = S.sbefore[src];
@@ -850,7 +973,7 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
             W += S.wt[w];
             Sp += S.wt[GW + w];
           }
-          if (!(W > 0.0)) {
+          if (!(W > kDegenerate * Zq_c)) {
             status |= LANTERN_ST_DEGENERATE;
             break;
           }
@@ -913,7 +1036,7 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
           }
           W = carry2;
         }
-        if (!(W > 0.0)) {
+        if (!(W > kDegenerate * Zq_c)) {
           status |= LANTERN_ST_DEGENERATE;
           break;
         }
@@ -939,7 +1062,7 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
           if (lastp >= 0) atomicMax(&S.tok, lastp);
           gbar(grp);
           if (gt == 0) {
-            Record rec = {-1, S.tok, status | S.status | (S.tok < 0 ? LANTERN_ST_DEGENERATE : 0), 0};
+            Record rec = {-1, S.tok, status | (S.tok < 0 ? LANTERN_ST_DEGENERATE : 0), 0};
             P.records[item] = rec;
           }
         } else if ((win & (GT - 1)) == gt) {
@@ -961,16 +1084,20 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
             if (tok < 0 && cum > target) tok = e;
           }
           if (tok < 0) tok = lastpos;
-          Record rec = {-1, g * 8 + tok, status | S.status, 0};
+          Record rec = {-1, g * 8 + tok, status, 0};
           P.records[item] = rec;
         }
         record_written = true;
       }
     }
     if (!record_written && gt == 0) {
-      // S.status was last written before a barrier every thread of the group has passed
-      Record rec = {accepted, -1, status | S.status, 0};
+      Record rec = {accepted, -1, status, 0};
       P.records[item] = rec;
+    }
+    // Algorithm 1 goes on from the accepted child only: the contexts behind the other children are dead
+    for (int j = gt; j < nchild; j += GT) {
+      const int nd = j == 0 ? cur.node0 : __ldg(&kids[j].node);
+      if (nd != accepted) P.dead[static_cast<size_t>(b) * R + nd + 1] = 1;
     }
     // this context's staging area (rows and E) is no longer needed by this warp
     __syncwarp();

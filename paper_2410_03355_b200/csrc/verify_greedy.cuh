@@ -141,6 +141,7 @@ struct GreedyCtxShared {
   float wm[GCW];
   int wi[GCW];
   int first[GGW];
+  int badslot[GGW];                 // per warp: first neighbour slot with an entry outside [0, V)
   double Z;
   float M;
   int arg;
@@ -234,7 +235,7 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
   const int cap = P.B * N;
   const int quads = V >> 2;
   const int G = gridDim.x;
-  auto slot = [&](int w) { return w < n_heavy ? w : cap - 1 - (w - n_heavy); };
+  auto slot = [&](int w) { return __ldg(P.ctx_slots + (w < n_heavy ? w : cap - 1 - (w - n_heavy))); };   // compact list -> work slot
 
   if (tid == 0) {
     for (int r = 0; r < ring; ++r) mbar_init(reinterpret_cast<uint64_t*>(&S.bar_full[r]), 1);
@@ -275,7 +276,7 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
       }
     }
     unsigned char* raw = gsm + static_cast<size_t>(buf) * area_bytes;
-    const bool ok = mbar_wait(reinterpret_cast<uint64_t*>(&S.bar_full[buf]), phase);
+    const bool ok = mbar_wait(reinterpret_cast<uint64_t*>(&S.bar_full[buf]), phase, P.wait_tries);
 
     // ---- the sweep: maximum, smallest arg max, numerators summed against the running maximum ----
     float m = NEG_INF, ssum = 0.0f;
@@ -359,7 +360,7 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
         for (int d = 1; d < ring; ++d) {
           const long long wj = w + static_cast<long long>(d) * G;
           const uint32_t j = it + d;
-          if (wj < total) mbar_wait(reinterpret_cast<uint64_t*>(&S.bar_full[j % ring]), (j / ring) & 1);
+          if (wj < total) mbar_wait(reinterpret_cast<uint64_t*>(&S.bar_full[j % ring]), (j / ring) & 1, P.wait_tries);
         }
       }
       __syncthreads();
@@ -388,7 +389,7 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
         // A_{k,delta}(x~): gather + prefix scan with the strict bound (Algorithm 2, second block)
         double thr = thr_tvd;
         const bool jsd = P.divergence == LANTERN_DIV_JSD;
-        if (jsd && tid == GGT)   // Section 6.2.2: the mass whose JSD is delta, from a thread that does not gather
+        if (jsd && tid == GGT)   // Section 5.3.2: the mass whose JSD is delta, from a thread that does not gather
           S.thr = jsd_mass_bound(static_cast<double>(P.delta), static_cast<double>(numer(xt)) / Z) * Z;
         double carry = 0.0;
         for (int base = 0;; base += 4 * GGT) {
@@ -396,6 +397,7 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
           bool val4[4];
           if (tid < GGT) {
             int nn[4];
+            int my_bad = kNone;   // first of this thread's slots whose entry lies outside [0, V)
             if (ci == 0 && base == 0) {   // a real branch: the prefetched entries must not wait for a load
 #pragma unroll
               for (int i = 0; i < 4; ++i) nn[i] = nb[i];
@@ -412,12 +414,14 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
               val4[i] = j < k;
               const int n = nn[i];
               const bool inr = val4[i] && static_cast<unsigned>(n) < static_cast<unsigned>(V);
-              if (val4[i] && !inr) atomicOr(&S.status, LANTERN_ST_BAD_TABLE);   // carries no mass
+              if (val4[i] && !inr && my_bad == kNone) my_bad = j;   // carries no mass
               run += inr ? static_cast<double>(numer(n)) : 0.0;
               pre4[i] = run;
             }
             incl = warp_incl_scan(run, lane);
             if (lane == 31) S.wt[warp] = incl;
+            const int wbad = __reduce_min_sync(kFull, my_bad);
+            if (lane == 0) S.badslot[warp] = wbad;
           }
           __syncthreads();
           if (jsd && base == 0) thr = S.thr;
@@ -452,6 +456,9 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
           if (warp == 0) {
             const int f = lane < GGW ? S.first[lane] : kNone;
             const int gfirst = __reduce_min_sync(kFull, f);
+            // a bad entry is reported where Algorithm 2's loop meets it, i.e. ahead of the slot that ends the set
+            const int gbad = __reduce_min_sync(kFull, lane < GGW ? S.badslot[lane] : kNone);
+            if (lane == 0 && gbad < gfirst) S.status |= LANTERN_ST_BAD_TABLE;
             const bool last = base + 4 * GGT >= k - 1;
             if (gfirst != kNone || last) {
               double sm = carry + tot;
@@ -510,7 +517,10 @@ __global__ void __launch_bounds__(GRT) lantern_greedy_bonus_kernel(VerifyParams 
     const bool finite = greedy_argmax<BF16, UNC>(P, static_cast<size_t>(b) * P.R + ctx, S, M, arg);
     if (threadIdx.x == 0) {
       P.out_tok[b] = finite ? arg : -1;
-      if (!finite && P.out_status) P.out_status[b] |= LANTERN_ST_NONFINITE;
+      if (!finite) {
+        if (P.out_status) P.out_status[b] |= LANTERN_ST_NONFINITE;
+        atomicOr(&P.counters->status_or, LANTERN_ST_NONFINITE);
+      }
     }
   }
 }

@@ -409,7 +409,7 @@ __global__ void __launch_bounds__(TKT, 2) lantern_topk_kernel(VerifyParams P, in
   auto job_item = [&](long long j) -> int {
     if (mode == 0) {
       const int w = static_cast<int>(j / per);
-      return P.work[w < n_heavy ? w : cap - 1 - (w - n_heavy)].item;
+      return P.work[P.ctx_slots[w < n_heavy ? w : cap - 1 - (w - n_heavy)]].item;
     }
     return P.bonus_seq[j] * R + P.bonus_ctx[j];
   };
@@ -430,7 +430,7 @@ __global__ void __launch_bounds__(TKT, 2) lantern_topk_kernel(VerifyParams P, in
     const long long jn = j + G < njobs ? j + G : j;
     const int item_next = job_item(jn);   // consumed after the keys are out: no select on it before
     const bool drafter = job_is_drafter(j);
-    const bool landed = __syncthreads_and(mbar_wait(bar, it & 1) ? 1 : 0) != 0;
+    const bool landed = __syncthreads_and(mbar_wait(bar, it & 1, P.wait_tries) ? 1 : 0) != 0;
     if (!landed) {   // the copy did not complete within the wait limit: no filter for this row, reported
       if (tid == 0) {
         (drafter ? P.thr_p : P.thr_q)[item] = __int_as_float(0xff800000);

@@ -9,7 +9,11 @@ across the window.  Probabilities must agree to REL: p(x~) relative to itself; s
 to the magnitude of the terms it was formed from -- for the first child of a context that is
 sum_A q itself, after sibling rejections the target is a difference (q' - p') / W evaluated in
 fp32, whose rounding error scales with q' + p', not with the difference (the oracle reports
-that magnitude as qa_mag).
+that magnitude as qa_mag; tests/test_oracle_verify.py pins it against a numpy replay).  The plain
+error relative to sum_A q itself is reported beside it (qa_rel_plain_max).
+
+The neighbour table the oracle reads is the ORACLE's: `oracle_table` builds, with the oracle, the
+rows that a call's drafted tokens name, and checks them against the library's table.
 """
 from __future__ import annotations
 
@@ -25,6 +29,37 @@ import paper_2410_03355_b200 as lt
 WINDOW = 1e-6
 REL = 1e-5
 
+_row_cache = {}
+
+
+def _content_key(codebook: np.ndarray):
+    import zlib
+    return (codebook.shape, zlib.crc32(np.ascontiguousarray(codebook).tobytes()))
+
+
+def oracle_table(codebook: np.ndarray, k: int, tokens, device_table=None, metric="l2") -> np.ndarray:
+    """[V, k] host table whose rows for `tokens` (any integer array) are built by the oracle; the other
+    rows hold -1 beyond the token itself, so that a read the walk should not make shows up as a table fault.
+    With `device_table`, asserts that the library's rows for those tokens are identical."""
+    V = codebook.shape[0]
+    key = (_content_key(codebook), k, metric)
+    cache = _row_cache.setdefault(key, {})
+    need = np.unique(np.asarray(tokens).ravel())
+    need = need[(need >= 0) & (need < V)]
+    miss = np.array([t for t in need if int(t) not in cache], dtype=np.int32)
+    if miss.size:
+        idx, _ = oracle.build_neighbors(codebook, k, rows=miss, metric=metric)
+        for r, t in enumerate(miss):
+            cache[int(t)] = idx[r]
+    tab = np.full((V, k), -1, np.int32)
+    tab[:, 0] = np.arange(V)
+    for t in need:
+        tab[t] = cache[int(t)]
+    if device_table is not None and need.size:
+        got = device_table[torch.from_numpy(need.astype(np.int64)).to(device_table.device)].cpu().numpy()
+        assert np.array_equal(got, tab[need]), "library and oracle neighbour rows differ"
+    return tab
+
 
 def to_device(inp: li.VerifyInputs, device="cuda"):
     def logits(a):
@@ -37,6 +72,29 @@ def to_device(inp: li.VerifyInputs, device="cuda"):
         draft_tokens=torch.from_numpy(inp.draft_tokens).to(device),
         tree_parents=None if inp.tree_parents is None else torch.from_numpy(inp.tree_parents).to(device),
         uniforms=torch.from_numpy(inp.uniforms).to(device))
+
+
+_dev_tables = {}
+
+
+def tables(codebook: np.ndarray, k: int, tokens):
+    """(host table for the oracle, device table for the library) of a codebook.  Up to 2048 codes both are
+    the oracle's full table.  Beyond that the device table is the library's own build, and the host table
+    holds the oracle's rows for `tokens` (a call's drafted tokens), checked against the library's rows."""
+    V = codebook.shape[0]
+    key = (_content_key(codebook), k)
+    if key not in _dev_tables:
+        if V <= 2048:
+            host = oracle.build_neighbors(codebook, k)[0]
+            _dev_tables[key] = (codebook, host, torch.from_numpy(host).cuda())
+        else:
+            dev = lt.build_neighbors(torch.from_numpy(codebook).cuda(), k, with_dist=False)[0]
+            torch.cuda.synchronize()
+            _dev_tables[key] = (codebook, None, dev)
+    _, host, dev = _dev_tables[key]
+    if host is None:
+        host = oracle_table(codebook, k, tokens, dev)
+    return host, dev
 
 
 DIV_NAME = {oracle.DIV_TVD: "tvd", oracle.DIV_JSD: "jsd"}
@@ -79,8 +137,11 @@ def _explained_by_window(inp, table, delta, b, ora, want, divergence=oracle.DIV_
             u = one.uniforms.copy()
             u[0, inp.N] = np.float32(min(max(u[0, inp.N] + s, 0.0), 1.0 - 2.0 ** -24))
             trials.append((u, delta))
-    for u, d in trials:
-        r = oracle.verify_inputs(dataclasses.replace(one, uniforms=u), table, max(d, 0.0), divergence, top_k)
+    trials = [(u, d, oracle.DEGENERATE_EPS) for u, d in trials]
+    if near_nodes:      # a residual's weight within the window of the threshold that makes it degenerate
+        trials += [(one.uniforms, delta, oracle.DEGENERATE_EPS - eps), (one.uniforms, delta, oracle.DEGENERATE_EPS + eps)]
+    for u, d, e in trials:
+        r = oracle.verify_inputs(dataclasses.replace(one, uniforms=u), table, max(d, 0.0), divergence, top_k, e)
         if (r.accept_len[0], r.next_token[0]) == want[:2] and np.array_equal(r.accept_path[0], want[2]):
             return True
     return False
@@ -96,7 +157,7 @@ def compare(inp: li.VerifyInputs, table: np.ndarray, delta: float, gpu: lt.Verif
     g_tok = gpu.next_token.cpu().numpy()
     g_path = gpu.accept_path.cpu().numpy()
     g_st = gpu.status.cpu().numpy()
-    near = outside = degenerate = 0
+    near = outside = 0
     bad = []
     st_mask = np.ones(inp.B, bool)
     for b in range(inp.B):
@@ -104,21 +165,14 @@ def compare(inp: li.VerifyInputs, table: np.ndarray, delta: float, gpu: lt.Verif
                 and np.array_equal(g_path[b], ora.accept_path[b]))
         if same:
             continue
-        # A residual whose total weight is exactly zero in double precision (possible only when the
-        # drafted token lies outside the drafter's own support, e.g. cut by the top-k filter, and target
-        # and drafter agree elsewhere) is rounding noise in fp32: the library may report it or draw
-        # from the noise; the walk up to that point must still agree.
-        if (ora.status[b] & oracle.ST_DEGENERATE) and g_len[b] == ora.accept_len[b] \
-                and np.array_equal(g_path[b], ora.accept_path[b]) and (g_st[b] & ~oracle.ST_DEGENERATE) == 0:
-            degenerate += 1
-            st_mask[b] = False
-            continue
+        st_mask[b] = False     # a different path may meet different faults; the path itself is judged here
         if _explained_by_window(inp, table, delta, b, ora, (g_len[b], g_tok[b], g_path[b]), divergence, top_k):
             near += 1
         else:
             outside += 1
             bad.append(b)
-    res = dict(n_seq=inp.B, near=near, mismatch_outside=outside, bad=bad, degenerate=degenerate,
+    res = dict(n_seq=inp.B, near=near, mismatch_outside=outside, bad=bad,
+               degenerate=int(((ora.status & oracle.ST_DEGENERATE) != 0).sum()),
                status_equal=bool(np.array_equal(g_st[st_mask], ora.status[st_mask])),
                accept_mean=float(ora.accept_len.mean()))
     if gpu.node_qa is not None:
@@ -130,8 +184,14 @@ def compare(inp: li.VerifyInputs, table: np.ndarray, delta: float, gpu: lt.Verif
         res["m_mismatch_outside"] = int((m[far] != ora.m[far]).sum())
         agree = t & (m == ora.m)
         rel_qa = np.abs(qa[agree] - ora.qa[agree]) / np.maximum(ora.qa_mag[agree], 1e-30)
+        rel_plain = np.abs(qa[agree] - ora.qa[agree]) / np.maximum(ora.qa[agree], 1e-30)
         rel_px = np.abs(px[t] - ora.px[t]) / np.maximum(ora.px[t], 1e-30)
         res["qa_rel_max"] = float(rel_qa.max()) if rel_qa.size else 0.0
+        res["qa_rel_plain_max"] = float(rel_plain.max()) if rel_plain.size else 0.0
+        # first children of their context: no residual round behind them, so the plain relative error binds
+        first = agree & (np.abs(ora.qa_mag - ora.qa) <= 1e-12 * np.maximum(ora.qa, 1e-300))
+        rel_first = np.abs(qa[first] - ora.qa[first]) / np.maximum(ora.qa[first], 1e-30)
+        res["qa_rel_first_max"] = float(rel_first.max()) if rel_first.size else 0.0
         res["px_rel_max"] = float(rel_px.max()) if rel_px.size else 0.0
         res["nodes_tested"] = int(t.sum())
     return res
@@ -142,4 +202,10 @@ def assert_parity(res):
     assert res["status_equal"], res
     if "qa_rel_max" in res:
         assert res["m_mismatch_outside"] == 0, res
-        assert res["qa_rel_max"] < REL and res["px_rel_max"] < REL, res
+        assert res["qa_rel_max"] < REL and res["px_rel_max"] < REL and res["qa_rel_first_max"] < REL, res
+
+
+def near_ceiling(n_seq: int) -> int:
+    """Most sequences of a call that may sit within the window of a threshold: the windows are 1e-6 wide and a
+    sequence takes a few dozen decisions, so more than a handful in a call means a tolerance problem."""
+    return max(2, n_seq // 50)

@@ -2,8 +2,9 @@
 
 The calls are made exactly as bench.py makes them (device-generated inputs, the library's own
 neighbour table, outputs without trace for the headline call).  The oracle then recomputes a
-seeded sample of sequences one by one from the device bytes copied back; every sequence is also
-checked for the properties that hold at any size.
+seeded sample of sequences one by one from the device bytes copied back, on neighbour rows that
+the oracle builds itself for the sampled sequences' drafted tokens (and that are compared with
+the library's rows first); every sequence is also checked for the properties that hold at any size.
 """
 import numpy as np
 import pytest
@@ -13,16 +14,25 @@ import lantern_inputs as li
 import lantern_inputs.device as lid
 import oracle
 import paper_2410_03355_b200 as lt
-from parity import assert_parity, compare
+from parity import assert_parity, compare, near_ceiling, oracle_table
 
 pytestmark = pytest.mark.gpu
 
 
+_codebooks = {}
+
+
 def _table(name):
     c = li.CONFIGS[name]
-    cb = torch.from_numpy(li.config_codebook(name)).cuda()
+    cbh = _codebooks.setdefault(name, li.config_codebook(name))
+    cb = torch.from_numpy(cbh).cuda()
     ws = torch.empty(max(lt.build_workspace_bytes(c["V"], c["D"], c["k"]), 16), dtype=torch.uint8, device="cuda")
     return lt.build_neighbors(cb, c["k"], with_dist=False, workspace=ws)[0]
+
+
+def _oracle_rows(name, host_inp, table):
+    """The oracle's own neighbour rows for every token the sampled sequences draft, checked against the library's."""
+    return oracle_table(_codebooks[name], li.CONFIGS[name]["k"], host_inp.draft_tokens, table)
 
 
 def _take(out: lt.VerifyOutputs, rows) -> lt.VerifyOutputs:
@@ -50,7 +60,7 @@ def _properties(d, out, N, V):
         assert np.all(path[b, al[b]:] == -1)
 
 
-@pytest.mark.parametrize("workload,sample", [("batch_chain", 96), ("stress", 128)])
+@pytest.mark.parametrize("workload,sample", [("batch_chain", 96), ("stress", 64)])
 def test_bench_sized_call_against_sampled_oracle(workload, sample):
     import bench
     w = bench.WORKLOADS[workload]
@@ -64,9 +74,10 @@ def test_bench_sized_call_against_sampled_oracle(workload, sample):
     _properties(d, out, N, V)
     rows = np.sort(np.random.default_rng(11).choice(B, size=min(sample, B), replace=False))
     host = lid.to_host(d, rows=rows)
-    res = compare(host, table.cpu().numpy(), delta, _take(out, rows))
+    res = compare(host, _oracle_rows(w["config"], host, table), delta, _take(out, rows))
     assert_parity(res)
     assert res["nodes_tested"] >= len(rows)
+    assert res["near"] <= near_ceiling(len(rows)), res
     # the headline call is made without trace outputs: same decisions
     out2 = lt.verify(d["target_logits"], d["draft_logits"], d["cfg_scale"], d["T"], d["draft_tokens"],
                      d["tree_parents"], table, delta, d["uniforms"])
@@ -96,6 +107,8 @@ def test_bench_sized_variants_against_sampled_oracle(workload, sample, divergenc
     _properties(d, out, N, V)
     rows = np.sort(np.random.default_rng(13).choice(B, size=min(sample, B), replace=False))
     host = lid.to_host(d, rows=rows)
-    res = compare(host, table.cpu().numpy(), delta, _take(out, rows), divergence=divergence, top_k=top_k)
+    res = compare(host, _oracle_rows(w["config"], host, table), delta, _take(out, rows), divergence=divergence,
+                  top_k=top_k)
     assert_parity(res)
     assert res["nodes_tested"] >= len(rows)
+    assert res["near"] <= near_ceiling(len(rows)), res

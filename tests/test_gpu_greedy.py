@@ -15,7 +15,7 @@ import torch
 import lantern_inputs as li
 import oracle
 import paper_2410_03355_b200 as lt
-from parity import DIV_NAME, REL, WINDOW, to_device
+from parity import DIV_NAME, REL, WINDOW, tables, to_device
 
 pytestmark = pytest.mark.gpu
 
@@ -102,14 +102,9 @@ def check_outputs(inp, host, delta, gpu, divergence=oracle.DIV_TVD, top_k=0):
 ])
 def test_chain_shapes(V, k, N, B, dtype, unc, delta):
     cb = li.codebook_gaussian(V, 8, seed=31)
-    if V <= 2048:
-        host = oracle.build_neighbors(cb, k)[0]
-        dev = torch.from_numpy(host).cuda()
-    else:
-        dev = lt.build_neighbors(torch.from_numpy(cb).cuda(), k, with_dist=False)[0]
-        host = dev.cpu().numpy()
     inp = li.verify_inputs(B, N, V, dtype=dtype, has_uncond=unc, cfg_scale=3.0 if unc else 1.0, sigma_target=1.0,
                            sigma_draft=0.4, rho=0.9, seed=101 + V + k)
+    host, dev = tables(cb, k, inp.draft_tokens)
     ora, _ = check(inp, host, dev, delta)
     if delta >= 2.0:
         assert (ora.accept_len == N).all()        # sum over everything = 1 >= any q
@@ -170,9 +165,8 @@ def test_bench_shape_sample():
     """The batch_chain shape (V = 16384, k = 1000, bf16 + guidance) at a batch the oracle finishes in seconds."""
     c = li.CONFIGS["batch_chain"]
     cb = li.config_codebook("batch_chain")
-    dev = lt.build_neighbors(torch.from_numpy(cb).cuda(), c["k"], with_dist=False)[0]
-    host = dev.cpu().numpy()
     inp = li.config_verify_inputs("batch_chain", step=0, B=48)
+    host, dev = tables(cb, c["k"], inp.draft_tokens)
     check(inp, host, dev, c["delta"])
 
 
@@ -181,7 +175,7 @@ def test_bench_sized_call_against_sampled_oracle(workload, sample):
     """The call `bench.py --greedy` times, checked on a seeded sample of its sequences."""
     import bench
     import lantern_inputs.device as lid
-    from test_gpu_fullsize import _properties, _table, _take
+    from test_gpu_fullsize import _oracle_rows, _properties, _table, _take
     w = bench.WORKLOADS[workload]
     cfg = li.CONFIGS[w["config"]]
     B, N, V, delta = w["B"], cfg["N"], cfg["V"], cfg["delta"]
@@ -192,7 +186,8 @@ def test_bench_sized_call_against_sampled_oracle(workload, sample):
     torch.cuda.synchronize()
     _properties(d, out, N, V)
     rows = np.sort(np.random.default_rng(12).choice(B, size=min(sample, B), replace=False))
-    check_outputs(lid.to_host(d, rows=rows), table.cpu().numpy(), delta, _take(out, rows))
+    host = lid.to_host(d, rows=rows)
+    check_outputs(host, _oracle_rows(w["config"], host, table), delta, _take(out, rows))
     out2 = lt.verify(d["target_logits"], None, d["cfg_scale"], 0.0, d["draft_tokens"], d["tree_parents"], table,
                      delta, None)
     torch.cuda.synchronize()

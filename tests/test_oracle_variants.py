@@ -1,5 +1,5 @@
-"""Pins of the oracle's variants: the JSD bound (Section 6.2.2), the cosine neighbour metric
-(Section 6.2.1) and the top-k logit filter (Appendix B.2).
+"""Pins of the oracle's variants: the JSD bound (Section 5.3.2), the cosine neighbour metric
+(Section 5.3.1) and the top-k logit filter (Appendix B.2).
 
   * JSD: the closed form on the collapsed tokens against the definition written out with numpy on
     whole distributions; the prefix rule by brute force; q(x~) = 0 reduces it to a TVD bound of

@@ -415,3 +415,95 @@ def test_status_bits():
     bad[:, 1] = V + 3
     res = oracle.verify_inputs(small_case(2, 2, V, seed=10), bad, 0.2)
     assert np.all(res.status & oracle.ST_BAD_TABLE)
+
+
+# ---------------------------------------------------------------------------------------
+# a residual without weight (reading R10): reported, next token from the context's own target
+# ---------------------------------------------------------------------------------------
+def test_residual_without_weight_draws_from_the_target():
+    V, k = 16, 3
+    table = oracle.build_neighbors(li.codebook_gaussian(V, 3, seed=4), k)[0]
+    inp = small_case(6, 2, V, seed=301)
+    inp.draft_logits[:] = inp.target_logits[0]          # drafter = target
+    for b in (0, 1, 2):
+        x = int(inp.draft_tokens[b, 0])
+        inp.target_logits[0, b, 0, table[x]] = -np.inf  # the drafted token and its neighbours carry no mass
+        inp.draft_logits[b, 0, table[x]] = -np.inf
+    res = oracle.verify_inputs(inp, table, 0.4)
+    for b in (0, 1, 2):
+        q = np_softmax(inp.target_logits[0, b, 0])
+        cdf = np.cumsum(q)
+        want = int(np.searchsorted(cdf, np.float64(inp.uniforms[b, 2]) * cdf[-1], side="right"))
+        assert res.status[b] == oracle.ST_DEGENERATE and res.accept_len[b] == 0 and res.w[b] == 0.0
+        assert res.next_token[b] == want and q[want] > 0
+    # drafter = target elsewhere: the ratio is 1 and every draft is accepted
+    assert (res.status[3:] == 0).all() and (res.accept_len[3:] == 2).all()
+
+
+def test_degenerate_threshold_is_a_threshold():
+    """W just above / below the threshold: p differs from q on two tokens by +-e, so the residual weighs e."""
+    V = 8
+    table = identity_table(V)
+    for e, degenerate in [(3e-5, False), (3e-6, True)]:
+        q = np.full(V, 1.0 / V)
+        p = q.copy()
+        p[0] += e          # the drafted token: p > q, so it can be rejected
+        p[1] -= e
+        inp = small_case(1, 1, V, seed=1)
+        inp.target_logits[0, 0, 0] = np.log(q).astype(np.float32)
+        inp.draft_logits[0, 0] = np.log(p).astype(np.float32)
+        inp.draft_tokens[0, 0] = 0
+        inp.uniforms[0] = [0.9999999, 0.5]
+        res = oracle.verify_inputs(inp, table, 0.0)
+        assert res.accept_len[0] == 0
+        assert bool(res.status[0] & oracle.ST_DEGENERATE) == degenerate, (e, res.w[0])
+        assert abs(res.w[0] - e) < 0.2 * e
+        if not degenerate:
+            assert res.next_token[0] == 1              # the only token with residual weight
+    # the threshold is an argument: at 0 only an exactly empty residual counts
+    assert not oracle.verify_inputs(inp, table, 0.0, degenerate_eps=0.0).status[0]
+
+
+# ---------------------------------------------------------------------------------------
+# qa_mag (the magnitude the GPU comparison divides the error of sum_A q by) against a numpy replay
+# ---------------------------------------------------------------------------------------
+def test_qa_magnitude_matches_a_numpy_replay_of_the_sibling_rounds():
+    """For the first child of a context the magnitude is sum_A q itself.  After a rejection the next target is
+    (q' - p') / W on the surviving tokens, evaluated from terms of size q' and p': the magnitude carried
+    forward is (mag + p') / W there and 0 elsewhere.  Replayed here with numpy on a 3-children root."""
+    V, k, delta = 12, 4, 0.15
+    table = oracle.build_neighbors(li.codebook_gaussian(V, 3, seed=9), k)[0]
+    parents = np.array([[-1, -1, -1]], dtype=np.int32)
+    checked = 0
+    for seed in range(40):
+        inp = small_case(1, 3, V, seed=400 + seed, parents=parents, sigma_draft=1.5)
+        inp.uniforms[0, :3] = 0.999          # reject whenever the rule allows it: sibling rounds happen
+        res = oracle.verify_inputs(inp, table, delta)
+        q = np_softmax(inp.target_logits[0, 0, 0])
+        p = np_softmax(inp.draft_logits[0, 0])
+        mag = q.copy()
+        for c in range(3):
+            if not res.tested[0, c]:
+                break
+            x = int(inp.draft_tokens[0, c])
+            m = int(res.m[0, c])
+            A = [x] + [int(t) for t in table[x, 1:m + 1]]
+            assert np.isclose(res.qa[0, c], q[A].sum(), rtol=1e-12)
+            assert np.isclose(res.qa_mag[0, c], mag[A].sum(), rtol=1e-12), (seed, c)
+            assert res.qa_mag[0, c] >= res.qa[0, c] * (1 - 1e-12)
+            if c == 0:
+                assert np.isclose(res.qa_mag[0, c], res.qa[0, c], rtol=1e-12)
+            if res.accept_len[0] > 0 and res.accept_path[0, 0] == c:
+                break
+            w = q.copy()
+            w[x] = q[A].sum()
+            w[A[1:]] = 0.0
+            w = np.maximum(w - p, 0.0)
+            W = w.sum()
+            mag = np.where(w > 0, (mag + p) / W, 0.0)
+            q = w / W
+            p = p.copy()
+            p[x] = 0.0
+            p = p / p.sum()
+            checked += c >= 0
+    assert checked > 20          # later siblings were reached

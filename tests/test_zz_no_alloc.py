@@ -3,11 +3,13 @@
 Some users of this library verify drafts at a point where a cudaMalloc is off the table: the
 serving process gave all of its HBM to the KV cache and activation arenas at start-up, or the
 step is latency-critical and cannot take the device-wide synchronisation an allocation brings.
-For them the library keeps a fixed 4 MiB scratch array inside its own device image.  This test
+For them the library keeps a fixed 6 MiB scratch array inside its own device image.  This test
 calls that entry point through the C ABI and checks that it returns exactly what the ordinary
 entry point (caller-supplied workspace) returns, on two calls in a row with different inputs --
 the second call finds the first call's leftovers in the shared array and must not be disturbed
-by them.  It also checks that a call too large for the fixed array is refused with a clear error.
+by them.  It also checks that a call too large for the fixed array is refused with a clear error,
+that greedy decoding (T = 0) goes through the same entry point, and that a warmed-up call leaves the
+device's free memory exactly where it was.
 
 The file is named so that pytest collects it last.
 """
@@ -33,12 +35,17 @@ def _outputs(B, N):
 
 
 def _same(a: lt.VerifyOutputs, b: lt.VerifyOutputs):
-    for f in ("accept_len", "next_token", "accept_path", "status", "node_m"):
+    for f in ("accept_len", "next_token", "accept_path", "status"):
         assert torch.equal(getattr(a, f), getattr(b, f)), f
-    for f in ("node_qa", "node_px"):   # same kernels, same inputs: bit-identical (NaN marks untested nodes)
-        x, y = getattr(a, f), getattr(b, f)
-        assert torch.equal(torch.isnan(x), torch.isnan(y)), f
-        assert torch.equal(torch.nan_to_num(x), torch.nan_to_num(y)), f
+    # Per-node values: same kernels, same inputs, so a node evaluated in both calls carries bit-identical
+    # values (NaN marks a node a call did not evaluate; which nodes off the accepted path get evaluated
+    # ahead of time may differ from call to call).  Every node on the accepted path is evaluated in both.
+    both = ~torch.isnan(a.node_qa) & ~torch.isnan(b.node_qa)
+    for f in ("node_qa", "node_px", "node_m"):
+        assert torch.equal(getattr(a, f)[both], getattr(b, f)[both]), f
+    on_path = a.accept_path >= 0
+    rows = torch.arange(a.accept_path.shape[0], device=a.accept_path.device)[:, None].expand_as(a.accept_path)
+    assert bool(both[rows[on_path], a.accept_path[on_path].long()].all())
 
 
 def test_static_workspace_matches_workspace_call_twice_in_a_row():
@@ -71,8 +78,8 @@ def test_static_workspace_matches_workspace_call_twice_in_a_row():
 def test_static_workspace_refuses_calls_beyond_its_size():
     V, k = 64, 4
     table = torch.from_numpy(oracle.build_neighbors(li.codebook_gaussian(V, 4, seed=42), k)[0]).cuda()
-    B, N = 4096, 60                       # needs several times the fixed 4 MiB of scratch
-    assert lt.verify_workspace_bytes(B, N) > lt.STATIC_WORKSPACE_BYTES
+    B, N = 4096, 60                       # needs several times the fixed 6 MiB of scratch
+    assert lt.verify_workspace_bytes(B, N, V, k) > lt.STATIC_WORKSPACE_BYTES
     tl = torch.zeros((1, B, N + 1, V), dtype=torch.bfloat16, device="cuda")
     dl = torch.zeros((B, N + 1, V), dtype=torch.bfloat16, device="cuda")
     tok = torch.zeros((B, N), dtype=torch.int32, device="cuda")
@@ -86,3 +93,27 @@ def test_static_workspace_refuses_calls_beyond_its_size():
     # the largest documented shapes do fit
     assert lt.verify_workspace_bytes(8192, 7) <= lt.STATIC_WORKSPACE_BYTES
     assert lt.verify_workspace_bytes(1024, 60) <= lt.STATIC_WORKSPACE_BYTES
+
+
+def test_static_workspace_greedy_and_no_allocation():
+    """T = 0 through the fixed array gives what the workspace call gives, and the call allocates nothing:
+    the device's free memory is the same before and after a call that has run once before."""
+    V, k, delta = 2048, 100, 0.3
+    table = torch.from_numpy(oracle.build_neighbors(li.codebook_gaussian(V, 8, seed=41), k)[0]).cuda()
+    inp = li.verify_inputs(40, 6, V, dtype=li.BF16, has_uncond=True, cfg_scale=3.0, rho=0.9, sigma_draft=0.5, seed=53)
+    d = to_device(inp)
+    want = lt.verify(d["target_logits"], None, inp.cfg_scale, 0.0, d["draft_tokens"], None, table, delta, None,
+                     trace=True)
+    out = _outputs(inp.B, inp.N)
+    lt.verify_static(d["target_logits"], None, inp.cfg_scale, 0.0, d["draft_tokens"], None, table, delta, None,
+                     out=out)
+    torch.cuda.synchronize()
+    _same(out, want)
+    assert int(want.accept_len.sum()) > 0
+    for T, dl, un in ((0.0, None, None), (1.0, d["draft_logits"], d["uniforms"])):
+        lt.verify_static(d["target_logits"], dl, inp.cfg_scale, T, d["draft_tokens"], None, table, delta, un, out=out)
+        torch.cuda.synchronize()
+        free0 = torch.cuda.mem_get_info()[0]
+        lt.verify_static(d["target_logits"], dl, inp.cfg_scale, T, d["draft_tokens"], None, table, delta, un, out=out)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free0

@@ -57,31 +57,57 @@ def load_peaks():
     return 6650.0, "fallback"
 
 
-def algorithmic_bytes(cfg: dict, B: int, parents, greedy: bool = False) -> int:
-    """Bytes the method must move per call: for each context with at least one child, two target
-    rows and one drafter row (one target row without guidance; no drafter row in greedy
-    decoding), plus one neighbour row of 4k bytes per drafted node.  Bonus rows, tokens, uniforms
-    and outputs (< 0.1 %) are left out."""
+def context_bytes(cfg: dict, greedy: bool = False) -> int:
+    """Logit bytes of one evaluated context: two target rows and one drafter row (one target row without
+    guidance; no drafter row in greedy decoding)."""
     import lantern_inputs as li
     esize = 2 if cfg["dtype"] == li.BF16 else 4
     rows = (2 if cfg["has_uncond"] else 1) + (0 if greedy else 1)
-    N, V, k = cfg["N"], cfg["V"], cfg["k"]
+    return rows * cfg["V"] * esize
+
+
+def work_bytes(cfg: dict, contexts: int, nodes: int, greedy: bool = False) -> int:
+    """Bytes that `contexts` evaluated contexts and `nodes` tested drafts must move: the contexts' logit rows
+    plus one neighbour row of 4k bytes per tested node.  Bonus rows, tokens, uniforms and outputs (< 0.1 %)
+    are left out."""
+    return contexts * context_bytes(cfg, greedy) + nodes * 4 * cfg["k"]
+
+
+def method_work(parents, accept_len, accept_path, N: int):
+    """(contexts, nodes) that Algorithm 1's loop itself evaluates and tests on the accepted paths: it goes on
+    from an accepted node only and stops at the first context whose children are all rejected.  For a tree
+    the children of a context are tried in node order up to and including the accepted one."""
+    al = accept_len.cpu().numpy().astype(np.int64)
     if parents is None:
-        n_ctx = B * N
-    else:
-        par = parents.cpu().numpy()
-        n_ctx = sum(len(set(par[b].tolist())) for b in range(B))
-    return n_ctx * rows * V * esize + B * N * 4 * k
+        n = np.minimum(al + 1, N)            # the context after the last accepted draft is tested unless the chain ended
+        return int(n.sum()), int(n.sum())
+    par = parents.cpu().numpy()
+    path = accept_path.cpu().numpy()
+    contexts = nodes = 0
+    for b in range(par.shape[0]):
+        kids = {}
+        for i, p_ in enumerate(par[b].tolist()):
+            kids.setdefault(p_ + 1, []).append(i)
+        cur = 0
+        for j in range(int(al[b])):
+            node = int(path[b, j])
+            contexts += 1
+            nodes += kids[cur].index(node) + 1
+            cur = node + 1
+        if cur in kids:                      # every child of the last context was rejected
+            contexts += 1
+            nodes += len(kids[cur])
+    return contexts, nodes
 
 
-# DRAM traffic of the fused kernel from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum)
-# of a 512-sequence call of the chain workload, as a ratio to that call's algorithmic bytes; traffic
-# grows in proportion to the contexts processed, so a full launch is scaled by its algorithmic bytes.
+# DRAM traffic of the fused kernel from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum) of a
+# small call of the chain workload, as a ratio to the bytes of the contexts and nodes that call evaluated;
+# traffic grows in proportion to the contexts evaluated, so a full launch is scaled by its evaluated bytes.
 # Tied to the kernel revision the capture was taken on: any other revision reports null.
-NCU_TRAFFIC = {"kernel_revision": 15, "workload": "batch_chain", "traffic_over_algorithmic": 377546752 / 366657536}
+NCU_TRAFFIC = {"kernel_revision": None, "workload": "batch_chain", "traffic_over_algorithmic": None}
 
 
-def ncu_traffic(workload, cfg, alg_bytes):
+def ncu_traffic(workload, alg_bytes):
     import paper_2410_03355_b200 as lt
     if NCU_TRAFFIC["traffic_over_algorithmic"] is None or workload != NCU_TRAFFIC["workload"]:
         return None
@@ -302,6 +328,211 @@ def run_aggregate(args):
     }), flush=True)
 
 
+def oracle_table_rows(cb, k, tokens, metric="l2"):
+    """[V, k] host table whose rows for the given drafted tokens are built by the oracle (the other rows are
+    never read by a verification of those sequences and hold -1 beyond the token itself)."""
+    import oracle
+    V = cb.shape[0]
+    need = np.unique(np.asarray(tokens).ravel())
+    need = need[(need >= 0) & (need < V)].astype(np.int32)
+    tab = np.full((V, k), -1, np.int32)
+    tab[:, 0] = np.arange(V)
+    if need.size:
+        tab[need] = oracle.build_neighbors(cb, k, rows=need, metric=metric)[0]
+    return tab, need
+
+
+def _oracle_worker(config, step, nseq, barrier, queue):
+    """One process of the all-cores oracle run: its own seeded sample of the workload, its own neighbour rows,
+    then -- together with the others -- the timed verification."""
+    import lantern_inputs as li
+    import oracle
+    cfg = li.CONFIGS[config]
+    inp = li.config_verify_inputs(config, step=step, B=nseq)
+    tab, _ = oracle_table_rows(li.config_codebook(config), cfg["k"], inp.draft_tokens)
+    barrier.wait()
+    t0 = time.perf_counter()
+    oracle.verify_inputs(inp, tab, cfg["delta"])
+    queue.put((nseq * cfg["N"], time.perf_counter() - t0))
+
+
+def oracle_all_cores(config: str, nseq: int = 48, max_procs: int = 32):
+    """The oracle as it stands (single-threaded code) run by one process per host core on disjoint seeded
+    samples of the workload at the same time: positions per second over the slowest process.  Processes are
+    started with `spawn`: a process forked after the first GPU call would hang."""
+    import multiprocessing as mp
+    ctx = mp.get_context("spawn")
+    n = max(1, min(os.cpu_count() or 1, max_procs))
+    barrier, queue = ctx.Barrier(n), ctx.Queue()
+    procs = [ctx.Process(target=_oracle_worker, args=(config, 1000 + i, nseq, barrier, queue)) for i in range(n)]
+    for p_ in procs:
+        p_.start()
+    got = [queue.get(timeout=600) for _ in procs]
+    for p_ in procs:
+        p_.join()
+    return sum(g[0] for g in got) / max(g[1] for g in got), n
+
+
+class Run:
+    """One workload resident in HBM: inputs, table, outputs, workspace, and the timed call."""
+
+    def __init__(self, args, workload, B=None, rank=0, seed=None):
+        import torch
+
+        import lantern_inputs as li
+        import lantern_inputs.device as lid
+        import paper_2410_03355_b200 as lt
+        self.lt, self.torch, self.args = lt, torch, args
+        self.workload = workload
+        w = WORKLOADS[workload]
+        self.cfg = cfg = li.CONFIGS[w["config"]]
+        self.B = B or w["B"]
+        self.N, self.V, self.k, self.delta = cfg["N"], cfg["V"], cfg["k"], cfg["delta"]
+        self.greedy = args.greedy
+        # ---- one-time neighbour table (timed separately) ----
+        self.cb_host = li.config_codebook(w["config"])
+        cb = torch.from_numpy(self.cb_host).cuda()
+        bws = torch.empty(max(lt.load_library().lantern_build_workspace_bytes_metric(
+            self.V, cfg["D"], self.k, lt.METRICS[args.metric]), 256), dtype=torch.uint8, device="cuda")
+        lt.build_neighbors(cb, self.k, with_dist=False, workspace=bws, metric=args.metric)      # warm-up
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        self.table, _ = lt.build_neighbors(cb, self.k, with_dist=False, workspace=bws, metric=args.metric)
+        e1.record()
+        torch.cuda.synchronize()
+        self.build_ms = e0.elapsed_time(e1)
+        del bws
+        # ---- inputs resident in HBM ----
+        self.d = d = lid.config_verify_inputs_device(
+            w["config"], B=self.B, seed=rank_seed(li.BASE_SEED, rank) if seed is None else seed, rho=args.rho)
+        torch.cuda.synchronize()
+        self.T = 0.0 if self.greedy else d["T"]
+        self.ws = torch.empty(lt.verify_workspace_bytes(self.B, self.N, self.V, self.k, cfg["dtype"], args.top_k),
+                              dtype=torch.uint8, device="cuda")
+        i32 = dict(dtype=torch.int32, device="cuda")
+        self.out = lt.VerifyOutputs(accept_len=torch.empty(self.B, **i32), next_token=torch.empty(self.B, **i32),
+                                    accept_path=torch.empty((self.B, self.N), **i32), status=torch.empty(self.B, **i32),
+                                    node_qa=None, node_px=None, node_m=None)
+        self.stream = torch.cuda.current_stream()
+        self.logit_gb = (d["target_logits"].numel() + (0 if self.greedy else d["draft_logits"].numel())) * \
+            d["target_logits"].element_size() / 1e9
+
+    def step(self, out=None, trace=False):
+        d, a = self.d, self.args
+        return self.lt.verify(d["target_logits"], None if self.greedy else d["draft_logits"], d["cfg_scale"], self.T,
+                              d["draft_tokens"], d["tree_parents"], self.table, self.delta,
+                              None if self.greedy else d["uniforms"], out=None if trace else (out or self.out),
+                              trace=trace, workspace=self.ws, stream=self.stream, divergence=a.divergence, top_k=a.top_k)
+
+    def timed(self, steps, warmup, dist=None, flush=None):
+        """`steps` calls between two events, with an event pair around every call's fused kernel.  `flush` (a
+        buffer larger than L2) is rewritten between calls when the call's own inputs are smaller than L2."""
+        torch, lt = self.torch, self.lt
+        for _ in range(warmup):
+            self.step()
+        torch.cuda.synchronize()
+        kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for a, b_ in kev:       # torch creates the CUDA event on first record
+            a.record()
+            b_.record()
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        cev = []
+        if flush is None:
+            t0.record()
+            for a, b_ in kev:
+                lt.profile_events(a, b_)
+                self.step()
+            t1.record()
+        else:                   # per-call events: the flush sits between calls, outside every timed interval
+            for a, b_ in kev:
+                flush.add_(1)
+                c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                lt.profile_events(a, b_)
+                c0.record()
+                self.step()
+                c1.record()
+                cev.append((c0, c1))
+        torch.cuda.synchronize()
+        lt.profile_events(None, None)
+        ms_total = t0.elapsed_time(t1) if flush is None else sum(c0.elapsed_time(c1) for c0, c1 in cev)
+        fused_ms = float(np.mean([a.elapsed_time(b_) for a, b_ in kev]))
+        return ms_total, fused_ms
+
+    def accounting(self, fused_ms, peak):
+        """Work and roofline figures of the last call."""
+        counts = self.lt.verify_counts(self.ws)
+        greedy = self.greedy
+        n_ctx = counts["contexts"]
+        ev_ctx = n_ctx if greedy else counts["evaluated"]
+        ev_nodes = self.B * self.N if greedy else counts["nodes_tested"]
+        m_ctx, m_nodes = method_work(self.d["tree_parents"], self.out.accept_len, self.out.accept_path, self.N)
+        ev_bytes = work_bytes(self.cfg, ev_ctx, ev_nodes, greedy)
+        m_bytes = work_bytes(self.cfg, m_ctx, m_nodes, greedy)
+        all_bytes = work_bytes(self.cfg, n_ctx, self.B * self.N, greedy)
+        sec = fused_ms * 1e-3
+        return dict(contexts_with_children=n_ctx, contexts_evaluated=ev_ctx, contexts_skipped=counts["skipped"],
+                    nodes_tested=ev_nodes, method_contexts=m_ctx, method_nodes=m_nodes,
+                    evaluated_bytes=int(ev_bytes), method_bytes=int(m_bytes), all_context_bytes=int(all_bytes),
+                    achieved=ev_bytes / sec / 1e9, frac=ev_bytes / sec / 1e9 / peak,
+                    method_achieved=m_bytes / sec / 1e9, method_frac=m_bytes / sec / 1e9 / peak)
+
+    def parity_sample(self, n_sample):
+        """A traced call compared with the oracle on a seeded sample of its sequences (the oracle reads its own
+        neighbour rows, which are first compared with the library's): counts of sequences with a decision
+        inside the 1e-6 window and of mismatches outside it."""
+        import lantern_inputs.device as lid
+        sys.path.insert(0, os.path.join(ROOT, "tests"))
+        import parity
+        torch = self.torch
+        out = self.step(trace=True)
+        torch.cuda.synchronize()
+        rows = np.sort(np.random.default_rng(5).choice(self.B, size=min(n_sample, self.B), replace=False))
+        host = lid.to_host(self.d, rows=rows)
+        tab, need = oracle_table_rows(self.cb_host, self.k, host.draft_tokens, self.args.metric)
+        lib_rows = self.table[torch.from_numpy(need.astype(np.int64)).cuda()].cpu().numpy()
+        idx = torch.as_tensor(rows, device="cuda")
+        pick = lambda t: None if t is None else t[idx]
+        sub = self.lt.VerifyOutputs(*(pick(getattr(out, f.name)) for f in __import__("dataclasses").fields(out)))
+        div = 1 if self.args.divergence == "jsd" else 0
+        res = parity.compare(host, tab, self.delta, sub, divergence=div, top_k=self.args.top_k)
+        return dict(sequences=int(len(rows)), near=res["near"], mismatch_outside=res["mismatch_outside"],
+                    status_equal=res["status_equal"], nodes_tested=res.get("nodes_tested"),
+                    qa_rel_max=res.get("qa_rel_max"), px_rel_max=res.get("px_rel_max"),
+                    table_rows_equal=bool(np.array_equal(lib_rows, tab[need])), table_rows_compared=int(need.size))
+
+
+def config_line(args, name, peak, run=None, steps=20, sample=16, flush=None):
+    """One entry of the `configs` block: the named configuration at its flattened call size."""
+    own = run is None
+    if own:
+        run = Run(args, name)
+    B, N = run.B, run.N
+    small = run.logit_gb < 0.2            # inputs smaller than L2: flush between calls
+    ms_total, fused_ms = run.timed(steps, 3, flush=flush if small else None)
+    ms = ms_total / steps
+    acc = run.accounting(fused_ms, peak)
+    line = {"workload": name, "sequences_per_call": B, "drafts_per_sequence": N, "V": run.V, "k": run.k,
+            "delta": run.delta, "positions_drafted_per_s": B * N / (ms * 1e-3),
+            "positions_tested_per_s": acc["method_nodes"] / (ms * 1e-3), "ms_per_call": ms, "kernel_ms": fused_ms,
+            "algorithmic_bytes": acc["evaluated_bytes"], "GB_per_s": acc["achieved"], "frac_of_hbm_peak": acc["frac"],
+            "method_bytes": acc["method_bytes"], "method_frac_of_hbm_peak": acc["method_frac"],
+            "contexts": {"with_children": acc["contexts_with_children"], "evaluated": acc["contexts_evaluated"],
+                         "on_accepted_paths": acc["method_contexts"]},
+            "mean_accept_len": float(run.out.accept_len.float().mean().item()),
+            "l2_policy": "L2 flushed between calls" if small else "inputs larger than L2",
+            "neighbor_build_ms": run.build_ms, "D": run.cfg["D"]}
+    if not args.greedy and sample:
+        line["parity"] = run.parity_sample(sample)
+    if own:
+        del run
+    return line
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -314,6 +545,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="leave out the per-configuration block (five named configurations, sampled oracle comparison)")
     ap.add_argument("--divergence", default="tvd", choices=["tvd", "jsd"],
                     help="what delta bounds (Section 5.3.2); the JSD run uses the workload's delta as it is")
     ap.add_argument("--metric", default="l2", choices=["l2", "cosine"], help="latent proximity of the table")
@@ -338,10 +571,21 @@ def main():
             run_aggregate(args)
         return
 
+    # the all-cores oracle run starts its processes before the first GPU call (rank 0 of a single-GPU run only)
+    cpu_all = None
+    plain = args.divergence == "tvd" and args.top_k == 0 and not args.greedy and args.metric == "l2"
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and plain:
+        try:
+            rate, procs = oracle_all_cores(WORKLOADS[args.workload]["config"],
+                                           nseq=48 if args.workload in ("batch_chain", "tiny") else 4)
+            cpu_all = {"value": rate, "unit": UNIT, "cores": procs, "kind": "oracle",
+                       "sample": "one process per core, each its own seeded sample of the workload, timed together"}
+        except Exception as e:      # the single-core figure below still stands
+            cpu_all = {"value": None, "error": repr(e)}
+
     import torch
 
     import lantern_inputs as li
-    import lantern_inputs.device as lid
     import paper_2410_03355_b200 as lt
 
     if not torch.cuda.is_available():
@@ -352,77 +596,25 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     lt.load_library()
+    peak, peak_kind = load_peaks()
 
-    w = WORKLOADS[args.workload]
-    cfg = li.CONFIGS[w["config"]]
-    B = args.batch or w["B"]
-    N, V, k, delta = cfg["N"], cfg["V"], cfg["k"], cfg["delta"]
-
-    # ---- one-time neighbour table (timed separately) ----
-    cb = torch.from_numpy(li.config_codebook(w["config"])).cuda()
-    bws = torch.empty(max(lt.load_library().lantern_build_workspace_bytes_metric(V, cfg["D"], k, lt.METRICS[args.metric]), 256),
-                      dtype=torch.uint8, device="cuda")
-    lt.build_neighbors(cb, k, with_dist=False, workspace=bws, metric=args.metric)      # warm-up
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    table, _ = lt.build_neighbors(cb, k, with_dist=False, workspace=bws, metric=args.metric)
-    e1.record()
-    torch.cuda.synchronize()
-    build_ms = e0.elapsed_time(e1)
-    del bws
-
-    # ---- inputs resident in HBM ----
-    d = lid.config_verify_inputs_device(w["config"], B=B, seed=rank_seed(li.BASE_SEED, rank), rho=args.rho)
-    torch.cuda.synchronize()
-    alg_bytes = algorithmic_bytes(cfg, B, d["tree_parents"], args.greedy)
-    T = 0.0 if args.greedy else d["T"]
-    ws = torch.empty(lt.verify_workspace_bytes(B, N, V, k, cfg["dtype"], args.top_k), dtype=torch.uint8, device="cuda")
-    i32 = dict(dtype=torch.int32, device="cuda")
-    out = lt.VerifyOutputs(accept_len=torch.empty(B, **i32), next_token=torch.empty(B, **i32),
-                           accept_path=torch.empty((B, N), **i32), status=torch.empty(B, **i32),
-                           node_qa=None, node_px=None, node_m=None)
-    stream = torch.cuda.current_stream()
-
-    def step():
-        lt.verify(d["target_logits"], None if args.greedy else d["draft_logits"], d["cfg_scale"], T, d["draft_tokens"],
-                  d["tree_parents"], table, delta, None if args.greedy else d["uniforms"], out=out, workspace=ws,
-                  stream=stream, divergence=args.divergence, top_k=args.top_k)
-
-    for _ in range(args.warmup):
-        step()
-    torch.cuda.synchronize()
-
-    # per-step events around the fused kernel (dominant kernel of the roofline)
-    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    for a, b_ in kev:       # torch creates the CUDA event on first record
-        a.record()
-        b_.record()
-    torch.cuda.synchronize()
+    run = Run(args, args.workload, B=args.batch or None, rank=rank)
+    cfg, B, N, V, k, delta = run.cfg, run.B, run.N, run.V, run.k, run.delta
+    d, out = run.d, run.out
+    T_used, logit_gb, build_ms = run.T, run.logit_gb, run.build_ms
 
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    if dist is not None:
-        dist.barrier()
-    torch.cuda.synchronize()
-    t_start, t_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t_start.record()
-    for a, b_ in kev:
-        lt.profile_events(a, b_)
-        step()
-    t_stop.record()
-    torch.cuda.synchronize()
-    lt.profile_events(None, None)
+    ms_total, fused_ms = run.timed(args.steps, args.warmup, dist)
     if dist is not None:
         dist.barrier()
     clocks = sampler.stop() if rank == 0 else None
-    ms_total = t_start.elapsed_time(t_stop)
-    fused_ms = float(np.mean([a.elapsed_time(b_) for a, b_ in kev]))
     ms_total, fused_ms = max_over_ranks([ms_total, fused_ms], dist, "cuda")
     ms_per_step = ms_total / args.steps
     value = aggregate_rate(world, B, N, ms_per_step)
+    acc = run.accounting(fused_ms, peak)
 
     status_bad = int((out.status != 0).sum().item())
     accept_mean = float(out.accept_len.float().mean().item())
@@ -445,7 +637,7 @@ def main():
             for name, t in host.items():
                 if t is not None:
                     d[name].copy_(t, non_blocking=True)
-            step()
+            run.step()
             h_len.copy_(out.accept_len, non_blocking=True)
             h_tok.copy_(out.next_token, non_blocking=True)
 
@@ -468,39 +660,74 @@ def main():
     # ---- CPU baseline: the oracle on a bounded sample of the same inputs (rank 0, N = 1) ----
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        n_s = min(B, 8192 if cfg["N"] <= 8 else 256)
+        import lantern_inputs.device as lid
+        # the oracle reads its own neighbour rows, built for the sampled sequences outside the timed part
+        n_s = min(B, 2048 if cfg["N"] <= 8 else 32)
         host_inp = lid.to_host(d, rows=np.arange(n_s))
-        rate, n_done, secs = oracle_sample_rate(host_inp, table.cpu().numpy(), delta, greedy=args.greedy,
+        tab, _ = oracle_table_rows(run.cb_host, k, host_inp.draft_tokens, args.metric)
+        rate, n_done, secs = oracle_sample_rate(host_inp, tab, delta, greedy=args.greedy,
                                                 divergence=1 if args.divergence == "jsd" else 0, top_k=args.top_k)
         cpu = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
-               "sample": f"first {n_done} sequences ({n_done * N} drafted positions) of this call, {secs:.1f} s"}
+               "sample": f"first {n_done} sequences ({n_done * N} drafted positions) of this call, {secs:.1f} s; "
+                         f"neighbour rows built by the oracle beforehand",
+               "all_cores": cpu_all}
+
+    # ---- the five named configurations, each with a sampled oracle comparison (rank 0, N = 1) ----
+    configs = None
+    if rank == 0 and world == 1 and not args.no_configs and plain and args.workload == "batch_chain" and not args.batch:
+        flush = torch.zeros(192 << 20, dtype=torch.uint8, device="cuda")       # larger than the 126 MB L2
+        configs = {}
+        chain = config_line(args, "batch_chain", peak, run=run, steps=20, sample=64)
+        # the configuration's literal call (32 sequences x 7 drafts), one call per step, plain stream launches
+        lit = Run(args, "batch_chain", B=cfg["B"], seed=li.BASE_SEED + 5)
+        lit_total, lit_fused = lit.timed(200, 5)
+        lit_cold, _ = lit.timed(50, 3, flush=flush)
+        chain["literal_call"] = {"sequences_per_call": lit.B, "us_per_call_back_to_back": 1e3 * lit_total / 200,
+                                 "us_per_call_l2_flushed": 1e3 * lit_cold / 50, "fused_kernel_us": 1e3 * lit_fused,
+                                 "stream_operations_per_call": lt.verify_launch_count(False, False),
+                                 "note": "back to back the 23 MB of rows stay in L2; flushed they come from HBM"}
+        del lit
+        configs["batch_chain"] = chain
+        del run, d, out
+        torch.cuda.empty_cache()
+        for name in ("tiny", "single_image", "px512_tree", "stress"):
+            configs[name] = config_line(args, name, peak, steps=20, sample=16 if name != "tiny" else 64, flush=flush)
+            torch.cuda.empty_cache()
+        del flush
 
     if rank == 0:
-        peak, peak_kind = load_peaks()
-        achieved = alg_bytes / (fused_ms * 1e-3) / 1e9
+        top_active = 0 < args.top_k < V
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": args.workload, "note": w["note"], "sequences_per_call": B, "drafts_per_sequence": N,
-                       "V": V, "k": k, "delta": delta, "cfg_scale": cfg["cfg_scale"], "T": T, "divergence": args.divergence, "metric": args.metric,
-                       "top_k": args.top_k,
+            "config": {"workload": args.workload, "note": WORKLOADS[args.workload]["note"], "sequences_per_call": B,
+                       "drafts_per_sequence": N,
+                       "V": V, "k": k, "delta": delta, "cfg_scale": cfg["cfg_scale"], "T": T_used,
+                       "divergence": args.divergence, "metric": args.metric, "top_k": args.top_k,
                        "logits": "bf16" if cfg["dtype"] == li.BF16 else "f32", "rho": args.rho,
-                       "l2_policy": "inputs larger than L2 (%.2f GB of logits per call)" %
-                                    ((d["target_logits"].numel() + (0 if args.greedy else d["draft_logits"].numel())) *
-                                     d["target_logits"].element_size() / 1e9),
+                       "l2_policy": "inputs larger than L2 (%.2f GB of logits per call)" % logit_gb,
                        "parallelism": "replicas" if world > 1 else "single"},
+            "positions": {"drafted_per_s": value, "tested_per_s": world * acc["method_nodes"] / (ms_per_step * 1e-3),
+                          "note": "drafted = every drafted position of the call; tested = the positions Algorithm 1's "
+                                  "loop tests before its first rejection"},
             "roofline": {"bound": "hbm", "kernel": "lantern_greedy_context_kernel" if args.greedy else "lantern_context_kernel",
-                         "achieved": achieved, "peak": peak,
-                         "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None if (args.greedy or args.divergence != "tvd" or 0 < args.top_k < V) else
-                                    ncu_traffic(args.workload, cfg, alg_bytes),
-                         "algorithmic_bytes_per_launch": int(alg_bytes), "kernel_ms": fused_ms},
+                         "achieved": acc["achieved"], "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                         "frac": acc["frac"],
+                         "traffic": None if (args.greedy or args.divergence != "tvd" or top_active) else
+                                    ncu_traffic(args.workload, acc["evaluated_bytes"]),
+                         "algorithmic_bytes_per_launch": acc["evaluated_bytes"], "kernel_ms": fused_ms,
+                         "contexts_with_children": acc["contexts_with_children"],
+                         "contexts_evaluated": acc["contexts_evaluated"], "nodes_tested": acc["nodes_tested"],
+                         "method_contexts": acc["method_contexts"], "method_bytes_per_launch": acc["method_bytes"],
+                         "method_achieved": acc["method_achieved"], "method_frac": acc["method_frac"],
+                         "note": "algorithmic bytes = rows of the contexts the kernel evaluated + neighbour rows of the "
+                                 "nodes it tested; method_* counts only what Algorithm 1's loop reaches"},
             "cpu_baseline": cpu, "e2e": e2e,
-            "gpu_launches": (4 + (0 if not 0 < args.top_k < V else (1 if args.greedy else 2))) * args.steps, "clocks": clocks,
-            "neighbor_build": {"ms": build_ms, "V": V, "D": cfg["D"], "k": k,
-                               "pairs_per_s": V * V / (build_ms * 1e-3)},
+            "gpu_launches": (lt.verify_launch_count(args.greedy, top_active) - 1) * args.steps, "clocks": clocks,
+            "neighbor_build": {"ms": build_ms, "V": V, "D": cfg["D"], "k": k, "pairs_per_s": V * V / (build_ms * 1e-3)},
             "outputs": {"mean_accept_len": accept_mean, "sequences_with_status_bits": status_bad},
+            "configs": configs,
         }
         print(json.dumps(line), flush=True)
     if dist is not None:

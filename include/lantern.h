@@ -302,7 +302,8 @@ lantern_status lantern_last_status(const void* workspace, void* cuda_stream, int
  *   out_counts[2]  the ones it left out because the walk could not reach them (Algorithm 1 stops
  *                  at the first rejection)
  *   out_counts[3]  next tokens drawn from a context's own q (bonus draws and degenerate residuals)
- * Greedy decoding evaluates every context: [1] and [2] stay 0 there. */
+ *   out_counts[4]  drafted nodes the fused pass tested
+ * out_counts holds five entries.  Greedy decoding evaluates every context: [1], [2] and [4] stay 0 there. */
 lantern_status lantern_verify_counts(const void* workspace, void* cuda_stream, int64_t* out_counts);
 
 /* Self-test of the kernels' bounded waits (not part of the method).  Every wait for an on-chip copy

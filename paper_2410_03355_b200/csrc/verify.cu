@@ -39,6 +39,7 @@ namespace lantern {
 // the fused pass overwrites; contexts without children are marked as leaves.
 // ---------------------------------------------------------------------------------------
 constexpr int PLAN_WARPS = 4;
+constexpr int kPlanArrays = 7;   // per-warp arrays of N + 2 ints in shared memory
 
 __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyParams P) {
   extern __shared__ int plan_smem[];
@@ -46,11 +47,14 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
   const int b = blockIdx.x * PLAN_WARPS + warp;
   if (b >= P.B) return;
   const int N = P.N, R = P.R, B = P.B;
-  int* cnt = plan_smem + warp * 4 * (R + 1);   // cnt[c]: number of children of context c
+  int* cnt = plan_smem + warp * kPlanArrays * (R + 1);   // cnt[c]: number of children of context c
   int* cur = cnt + (R + 1);                    // fill cursor, ends as the end offset of context c
-  int* dep = cur + (R + 1);                    // depth of context c (root = 0)
+  int* dep = cur + (R + 1);                    // depth of context c (root = 0), later its breadth-first rank
   int* dst = dep + (R + 1);                    // per depth: next breadth-first rank
-  for (int i = lane; i <= R; i += 32) cnt[i] = 0, dst[i] = 0;
+  int* siz = dst + (R + 1);                    // number of contexts in the subtree of context c, itself included
+  int* din = siz + (R + 1);                    // depth-first (pre-order) position of context c
+  int* nxt = din + (R + 1);                    // depth-first position the next child of context c gets
+  for (int i = lane; i <= R; i += 32) cnt[i] = 0, dst[i] = 0, siz[i] = 1;
   __syncwarp();
   int status = 0;
   const float qnan = __int_as_float(0x7fc00000);
@@ -89,11 +93,24 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
       cur[c] = run;
       run += cnt[c];
     }
+    // Subtree sizes (children have larger indices than their parents) and pre-order positions: the
+    // contexts behind a node then occupy one contiguous range of positions, which is what lets the
+    // fused pass strike a whole rejected subtree with a few byte stores.
+    for (int i = N - 1; i >= 0; --i) {
+      const int par = P.parents ? P.parents[static_cast<size_t>(b) * N + i] : i - 1;
+      siz[par + 1] += siz[i + 1];
+    }
     dep[0] = 0;
+    din[0] = 0;
+    nxt[0] = 1;
     for (int i = 0; i < N; ++i) {
       const size_t o = static_cast<size_t>(b) * N + i;
       const int par = P.parents ? P.parents[o] : i - 1;
-      ChildInfo ci = {i, P.tokens[o], P.uniforms ? P.uniforms[static_cast<size_t>(b) * R + i] : 0.0f, 0};
+      din[i + 1] = nxt[par + 1];
+      nxt[par + 1] += siz[i + 1];
+      nxt[i + 1] = din[i + 1] + 1;
+      ChildInfo ci = {i, P.tokens[o], P.uniforms ? P.uniforms[static_cast<size_t>(b) * R + i] : 0.0f,
+                      (din[i + 1] << 16) | siz[i + 1]};
       kids[cur[par + 1]++] = ci;
       dep[i + 1] = dep[par + 1] + 1;
     }
@@ -135,7 +152,7 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
         P.records[static_cast<size_t>(b) * R + c] = pending;
         const int start = cur[c] - n;
         const ChildInfo f = kids[start];
-        WorkItem w = {b * R + c, b * N + start, n, f.node, f.token, f.r, u_final, 0};
+        WorkItem w = {b * R + c, b * N + start, (n << 16) | f.node, f.span, f.token, f.r, u_final, b * R + din[c]};
         const int slot = dep[c] * B + b;
         P.work[slot] = w;
         P.ctx_slots[n >= 2 ? hb + __popc(heavy & below) : cap - 1 - (lb + __popc(light & below))] = slot;
@@ -391,6 +408,7 @@ extern "C" lantern_status lantern_verify_counts(const void* workspace, void* cud
   out_counts[1] = c.n_evaluated;
   out_counts[2] = c.n_skipped;
   out_counts[3] = c.n_bonus;
+  out_counts[4] = c.n_tested;
   return LANTERN_OK;
 }
 
@@ -531,7 +549,7 @@ static lantern_status verify_impl(const void* target_logits, const void* draft_l
   if (sms < 1) return LANTERN_E_CUDA;
 
   if (cudaMemsetAsync(P.counters, 0, 256, st) != cudaSuccess) return LANTERN_E_CUDA;
-  const size_t plan_smem = static_cast<size_t>(PLAN_WARPS) * 4 * (N + 2) * sizeof(int);
+  const size_t plan_smem = static_cast<size_t>(PLAN_WARPS) * kPlanArrays * (N + 2) * sizeof(int);
   if (plan_smem > 48 * 1024 &&
       cudaFuncSetAttribute(lantern_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            static_cast<int>(plan_smem)) != cudaSuccess)

@@ -39,18 +39,23 @@ struct ChildInfo {              // one drafted node, stored in the order its par
   int node;                     // node index within the sequence
   int token;                    // x~
   float r;                      // its acceptance uniform
-  int pad;
+  int span;                     // the contexts behind the node, in pre-order: (first position << 16) | count
 };
 
 struct WorkItem {               // one context with children: everything its CTA needs, in one 32-byte load
   int item;                     // b * R + c  (row index of the context); -1 = none
   int cbase;                    // index of its first child in the ChildInfo array
-  int nchild;
-  int node0;                    // first child, inlined
-  int tok0;
+  int nchild_node0;             // (number of children << 16) | first child's node index
+  int span0;                    // first child's ChildInfo::span
+  int tok0;                     // first child's token and uniform, inlined
   float r0;
   float u_final;                // the sequence's uniform for the final draw
-  int pad;
+  int mark;                     // index of the context's own entry in the array of dead marks
+};
+
+struct GroupItem {              // the same, as a producer hands it to its consumer group through shared memory
+  int item, cbase, nchild, node0, tok0, span0;
+  float r0, u_final;
 };
 
 struct VerifyParams {
@@ -72,7 +77,7 @@ struct VerifyParams {
   WorkItem* work;               // [N, B]: slot r * B + b holds the r-th context with children of sequence b in
                                 //         breadth-first order (by depth, then by index); item = -1 where there is none
   int32_t* ctx_slots;           // [B*N]: the occupied slots, heavy ones from the front, light ones from the back
-  unsigned char* dead;          // [B, R]: 1 once the walk is known not to reach the context
+  unsigned char* dead;          // [B, R], a sequence's contexts in pre-order: 1 once the walk is known not to reach one
   ChildInfo* children;          // [B, N]
   Record* records;              // [B, R]
   int32_t* seq_status;          // [B]

@@ -28,8 +28,8 @@
 // Which contexts are evaluated.  Algorithm 1 stops at the first rejection, so a context behind a
 // rejected node is never tested by the method.  Work items come in breadth-first order per sequence
 // (see the plan kernel); when a context has been decided, its group marks the contexts behind every
-// child it did not accept as dead, and a producer that meets a dead context leaves it out (and marks
-// that context's children in turn).  A context whose parent is still undecided when its turn comes is
+// child it did not accept as dead (a sequence's contexts are numbered in pre-order for this, so that a
+// subtree is one contiguous range of marks), and a producer that meets a dead context leaves it out.  A context whose parent is still undecided when its turn comes is
 // evaluated anyway: with few sequences per call that keeps every SM busy (all contexts of a tree run
 // side by side), with many sequences it is rare, and the walk kernel reads only records on the
 // accepted path either way, so the result never depends on what was speculated.
@@ -81,7 +81,7 @@ struct GroupShared {
   int tok;
   int fail;                     // a bounded wait for the target rows ran out (sticky)
   float thr[2][2];              // top-k thresholds (target, drafter) of the context in work[i]
-  WorkItem work[2];             // descriptor of context i in work[i & 1]: the next one is published while the current one runs
+  GroupItem work[2];            // descriptor of context i in work[i & 1]: the next one is published while the current one runs
 };
 
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -254,25 +254,31 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
     const int G = gridDim.x * NGRP;              // producers in the grid
     const int me = blockIdx.x * NGRP + grp;
     const uint32_t tries = P.wait_tries;
+    // Slots per batch: a share of what is left that shrinks towards the end of the list (so that the
+    // groups finish together), but at least as many slots as it has taken so far to find one live
+    // context (tree workloads leave most slots empty or dead, and every batch costs a round trip).
+    int slots_seen = 0, live_seen = 0;
     auto batch_size = [&](int at) {
-      const int s = (total - at) / (4 * G);
+      const int share = (total - at) / (4 * G);
+      const int sparse = (slots_seen + 1) / (live_seen + 1);
+      const int s = share > sparse ? share : sparse;
       return s < 1 ? 1 : (s > 32 ? 32 : s);
     };
     struct Cand {
-      int item, cbase, nchild, node0, tok0;
+      int item, cbase, nchild_node0, span0, tok0, mark;
       float r0, u_final, tq, tp;
     };
     auto load_cand = [&](int start, int size) -> Cand {
       Cand c;
       c.item = -1;
-      c.cbase = c.nchild = c.node0 = c.tok0 = 0;
+      c.cbase = c.nchild_node0 = c.span0 = c.tok0 = c.mark = 0;
       c.r0 = c.u_final = c.tq = c.tp = 0.0f;
       const int w = start + lane;
       if (lane < size && w < total) {
         const int4 lo = __ldg(reinterpret_cast<const int4*>(P.work + w));
         const int4 hi = __ldg(reinterpret_cast<const int4*>(P.work + w) + 1);
-        c.item = lo.x, c.cbase = lo.y, c.nchild = lo.z, c.node0 = lo.w;
-        c.tok0 = hi.x, c.r0 = __int_as_float(hi.y), c.u_final = __int_as_float(hi.z);
+        c.item = lo.x, c.cbase = lo.y, c.nchild_node0 = lo.z, c.span0 = lo.w;
+        c.tok0 = hi.x, c.r0 = __int_as_float(hi.y), c.u_final = __int_as_float(hi.z), c.mark = hi.w;
         if (TOPK && c.item >= 0) {   // the context's thresholds travel with its descriptor: (target, drafter)
           c.tq = __ldg(P.thr_q + c.item);
           c.tp = __ldg(P.thr_p + c.item);
@@ -280,25 +286,18 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       }
       return c;
     };
-    auto is_dead = [&](int item) -> bool {
-      return *reinterpret_cast<const volatile unsigned char*>(P.dead + item) != 0;
-    };
-    // the walk cannot reach a dead context, hence none of the contexts behind its children either
-    auto bury = [&](const Cand& c) {
-      const size_t row0 = static_cast<size_t>(c.item / R) * R;
-      for (int j = 0; j < c.nchild; ++j) {
-        const int node = j == 0 ? c.node0 : __ldg(&P.children[c.cbase + j].node);
-        P.dead[row0 + node + 1] = 1;
-      }
+    auto is_dead = [&](int mark) -> bool {
+      return *reinterpret_cast<const volatile unsigned char*>(P.dead + mark) != 0;
     };
     int n_eval = 0, n_skip = 0;
     // live candidates of a batch, as a lane mask
     auto filter = [&](const Cand& c) -> unsigned {
       const bool has = c.item >= 0;
-      const bool dead = has && is_dead(c.item);
-      if (dead) bury(c);
+      const bool dead = has && is_dead(c.mark);
       n_skip += __popc(__ballot_sync(kFull, dead));
-      return __ballot_sync(kFull, has && !dead);
+      const unsigned live = __ballot_sync(kFull, has && !dead);
+      live_seen += __popc(live);
+      return live;
     };
     const int b0 = batch_size(0);
     Cand cur = load_cand(me * b0, b0);
@@ -311,6 +310,7 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       if (lane == 0) st = G * b0 + atomicAdd(&P.counters->work_next, size);
       st = __shfl_sync(kFull, st, 0);
       seen = st;
+      slots_seen += size;
       return st;
     };
     int nsize = 0;
@@ -342,23 +342,23 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
         break;
       }
       // as late as possible: has the context died meanwhile, has the call been given up?
-      const int gone = (lane == l && is_dead(cur.item)) ? 1 : 0;
+      const int gone = (lane == l && is_dead(cur.mark)) ? 1 : 0;
       const int stop = *reinterpret_cast<const volatile int*>(&P.counters->abort);
       if (__any_sync(kFull, stop != 0)) break;
       if (__any_sync(kFull, gone)) {
-        if (lane == l) bury(cur);
         ++n_skip;
         continue;
       }
-      WorkItem it;
+      GroupItem it;
       it.item = __shfl_sync(kFull, cur.item, l);
       it.cbase = __shfl_sync(kFull, cur.cbase, l);
-      it.nchild = __shfl_sync(kFull, cur.nchild, l);
-      it.node0 = __shfl_sync(kFull, cur.node0, l);
+      const int nn0 = __shfl_sync(kFull, cur.nchild_node0, l);
+      it.nchild = nn0 >> 16;
+      it.node0 = nn0 & 0xffff;
+      it.span0 = __shfl_sync(kFull, cur.span0, l);
       it.tok0 = __shfl_sync(kFull, cur.tok0, l);
       it.r0 = __shfl_sync(kFull, cur.r0, l);
       it.u_final = __shfl_sync(kFull, cur.u_final, l);
-      it.pad = 0;
       const float tq_cur = TOPK ? __shfl_sync(kFull, cur.tq, l) : 0.0f;
       const float tp_cur = TOPK ? __shfl_sync(kFull, cur.tp, l) : 0.0f;
       // the rows of the context after this one, for the L2 prefetch below
@@ -475,7 +475,7 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       give_up(iter, true);
       break;
     }
-    const WorkItem cur = S.work[iter & 1];
+    const GroupItem cur = S.work[iter & 1];
     const int item = cur.item;
     if (item < 0) break;
     float tq = 0.0f, tp = 0.0f;   // top-k thresholds of this context's target and drafter rows
@@ -734,6 +734,7 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       }
 
       for (int ci = 0; ci < nchild; ++ci) {
+        if (gt == 0) atomicAdd(&P.counters->n_tested, 1);   // work accounting (a fire-and-forget reduction)
         const int32_t* nrow = P.nbr + static_cast<size_t>(xt) * k;
         // the next sibling's description, wanted only after a rejection: in flight meanwhile
         ChildInfo sib = {0, 0, 0.0f, 0};
@@ -1094,10 +1095,18 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       Record rec = {accepted, -1, status, 0};
       P.records[item] = rec;
     }
-    // Algorithm 1 goes on from the accepted child only: the contexts behind the other children are dead
-    for (int j = gt; j < nchild; j += GT) {
-      const int nd = j == 0 ? cur.node0 : __ldg(&kids[j].node);
-      if (nd != accepted) P.dead[static_cast<size_t>(b) * R + nd + 1] = 1;
+    // Algorithm 1 goes on from the accepted child only: every context behind another child is dead.  In
+    // pre-order those are one contiguous range per child.
+    for (int j = 0; j < nchild; ++j) {
+      int node_j = cur.node0, span_j = cur.span0;
+      if (j > 0) {
+        const int4 kid = __ldg(reinterpret_cast<const int4*>(kids + j));
+        node_j = kid.x, span_j = kid.w;
+      }
+      if (node_j != accepted) {
+        unsigned char* first = P.dead + static_cast<size_t>(b) * R + (span_j >> 16);
+        for (int o = gt; o < (span_j & 0xffff); o += GT) first[o] = 1;
+      }
     }
     // this context's staging area (rows and E) is no longer needed by this warp
     __syncwarp();

@@ -379,8 +379,8 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
       };
       const double thr_tvd = static_cast<double>(P.delta) * Z;   // the bound in units of the unnormalised sums
       const ChildInfo* kids = P.children + cur.cbase;
-      for (int ci = 0; ci < cur.nchild && accepted < 0; ++ci) {
-        int node = cur.node0, xt = cur.tok0;
+      for (int ci = 0; ci < (cur.nchild_node0 >> 16) && accepted < 0; ++ci) {
+        int node = cur.nchild_node0 & 0xffff, xt = cur.tok0;
         if (ci > 0) {
           const int4 info = __ldg(reinterpret_cast<const int4*>(kids + ci));
           node = info.x, xt = info.y;

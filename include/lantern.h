@@ -283,7 +283,8 @@ int lantern_kernel_revision(void);
 
 /* Number of kernels (and memsets) one verification call enqueues: memset, plan, fused pass or greedy
  * pass, walk, bonus; a call whose top-k filter is active (0 < top_k < V) enqueues one threshold kernel
- * more in greedy decoding (greedy != 0) and two more in sampling.  For launch accounting. */
+ * more (ahead of the greedy pass; in sampling ahead of the bonus draw -- the fused pass finds the
+ * thresholds of its own contexts).  For launch accounting. */
 int lantern_verify_launch_count(int greedy, int top_k_active);
 
 /* ------------------------------------------------------------------------------------------
@@ -303,7 +304,8 @@ lantern_status lantern_last_status(const void* workspace, void* cuda_stream, int
  *                  at the first rejection)
  *   out_counts[3]  next tokens drawn from a context's own q (bonus draws and degenerate residuals)
  *   out_counts[4]  drafted nodes the fused pass tested
- * out_counts holds five entries.  Greedy decoding evaluates every context: [1], [2] and [4] stay 0 there. */
+ *   out_counts[5]  rows whose top-k threshold needed the slow exact search (with a top-k filter only)
+ * out_counts holds six entries.  Greedy decoding evaluates every context: [1], [2] and [4] stay 0 there. */
 lantern_status lantern_verify_counts(const void* workspace, void* cuda_stream, int64_t* out_counts);
 
 /* Self-test of the kernels' bounded waits (not part of the method).  Every wait for an on-chip copy

@@ -155,13 +155,13 @@ def last_status(workspace: torch.Tensor, stream: Optional[torch.cuda.Stream] = N
 
 def verify_counts(workspace: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> dict:
     """lantern_verify_counts: work accounting of the last verify() call that used `workspace`."""
-    out = (ctypes.c_int64 * 5)()
+    out = (ctypes.c_int64 * 6)()
     with torch.cuda.device(workspace.device):
         rc = load_library().lantern_verify_counts(_ptr(workspace), _stream_ptr(stream), out)
     if rc != 0:
         raise LanternError(rc, "lantern_verify_counts")
     return dict(contexts=int(out[0]), evaluated=int(out[1]), skipped=int(out[2]), from_q=int(out[3]),
-                nodes_tested=int(out[4]))
+                nodes_tested=int(out[4]), slow_topk_rows=int(out[5]))
 
 
 def debug_wait_test(max_tries: int = 0, withhold_context: int = -1) -> None:

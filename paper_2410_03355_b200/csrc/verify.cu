@@ -314,11 +314,7 @@ static cudaError_t launch_bonus(const VerifyParams& P, int sms, cudaStream_t st)
 template <bool BF16, bool UNC, bool TOPK>
 static cudaError_t launch_verify(const VerifyParams& P, int CH, bool tone, bool jsd, long long items, int sms,
                                  int grid_ctx, size_t smem_bytes, cudaStream_t st) {
-  cudaError_t e;
-  if (TOPK) {
-    e = launch_topk<BF16, UNC>(P, 0, 2 * items, sms, st);
-    if (e != cudaSuccess) return e;
-  }
+  cudaError_t e;   // (with the top-k filter the fused pass finds the thresholds of its contexts itself)
   if (g_ev_before && g_ev_after) cudaEventRecord(g_ev_before, st);
   e = launch_context_kernel(P, CH, BF16, UNC, tone, jsd, TOPK, grid_ctx, smem_bytes, st);
   if (e != cudaSuccess) return e;
@@ -382,9 +378,10 @@ extern "C" size_t lantern_verify_workspace_bytes(int B, int N, int V, int k, int
 }
 
 extern "C" int lantern_verify_launch_count(int greedy, int top_k_active) {
-  // memset, plan, fused pass (or greedy pass), walk, bonus; with the filter one threshold kernel ahead of
-  // the pass and, in sampling, one more ahead of the bonus draw
-  return 5 + (top_k_active ? (greedy ? 1 : 2) : 0);
+  // memset, plan, fused pass (or greedy pass), walk, bonus; with the filter one threshold kernel more: ahead
+  // of the greedy pass, or ahead of the bonus draw in sampling (the fused pass finds its own thresholds)
+  (void)greedy;
+  return 5 + (top_k_active ? 1 : 0);
 }
 
 extern "C" lantern_status lantern_last_status(const void* workspace, void* cuda_stream, int32_t* out_bits) {
@@ -409,6 +406,7 @@ extern "C" lantern_status lantern_verify_counts(const void* workspace, void* cud
   out_counts[2] = c.n_skipped;
   out_counts[3] = c.n_bonus;
   out_counts[4] = c.n_tested;
+  out_counts[5] = c.n_slow_topk;
   return LANTERN_OK;
 }
 
@@ -491,7 +489,7 @@ static lantern_status verify_impl(const void* target_logits, const void* draft_l
   // one staging area of three row slots per consumer group; the numerators are kept over the rows they came from
   const size_t smem_bytes = NGRP * ((static_cast<size_t>(3) * V * esize + 127) & ~static_cast<size_t>(127));
   (void)nrows;
-  if (!greedy && (smem_bytes > 220 * 1024 || (dtype == LANTERN_F32 && V > 8192))) return LANTERN_E_SHAPE;
+  if (!greedy && (smem_bytes > 192 * 1024 || (dtype == LANTERN_F32 && V > 8192))) return LANTERN_E_SHAPE;   // plus the kernel's static part: within the 227 KB of a CTA
   if (B == 0) return LANTERN_OK;
   if (!target_logits || !neighbor_idx || !out_accept_len || !out_next_token) return LANTERN_E_NULL;
   if (!greedy && !uniforms) return LANTERN_E_NULL;

@@ -25,6 +25,7 @@ struct Counters {               // first 256 bytes of the workspace, zeroed per 
   int n_tested;                 // drafted nodes it tested
   int status_or;                // OR of every sequence's status bits (written by the walk and later kernels)
   int abort;                    // a bounded wait ran out somewhere: no further work is handed out
+  int n_slow_topk;              // rows whose top-k threshold needed the slow exact search
 };
 
 struct Record {                 // result of one context

@@ -66,6 +66,12 @@ __device__ __forceinline__ int owner_slice(int x) {
   return ((g >> (LOG_GT + LOG_CP)) << LOG_GT) | (g & (GT - 1));
 }
 
+__device__ __forceinline__ void gbar(int grp);   // barrier among the threads of one consumer group (below)
+
+}  // namespace lantern
+#include "verify_context_topk.cuh"
+namespace lantern {
+
 struct GroupShared {
   double wzq[GW], wzp[GW];      // per-warp sums of numerators, common units
   double wt[8 * GW];            // per-(chunk, warp) totals for scans and block sums
@@ -80,7 +86,7 @@ struct GroupShared {
   int acc_valid;                // acc_e / acc_p are usable for the current child
   int tok;
   int fail;                     // a bounded wait for the target rows ran out (sticky)
-  float thr[2][2];              // top-k thresholds (target, drafter) of the context in work[i]
+  GroupTopk tk;                 // scratch of the top-k threshold search (TOPK variants)
   GroupItem work[2];            // descriptor of context i in work[i & 1]: the next one is published while the current one runs
 };
 
@@ -266,23 +272,19 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
     };
     struct Cand {
       int item, cbase, nchild_node0, span0, tok0, mark;
-      float r0, u_final, tq, tp;
+      float r0, u_final;
     };
     auto load_cand = [&](int start, int size) -> Cand {
       Cand c;
       c.item = -1;
       c.cbase = c.nchild_node0 = c.span0 = c.tok0 = c.mark = 0;
-      c.r0 = c.u_final = c.tq = c.tp = 0.0f;
+      c.r0 = c.u_final = 0.0f;
       const int w = start + lane;
       if (lane < size && w < total) {
         const int4 lo = __ldg(reinterpret_cast<const int4*>(P.work + w));
         const int4 hi = __ldg(reinterpret_cast<const int4*>(P.work + w) + 1);
         c.item = lo.x, c.cbase = lo.y, c.nchild_node0 = lo.z, c.span0 = lo.w;
         c.tok0 = hi.x, c.r0 = __int_as_float(hi.y), c.u_final = __int_as_float(hi.z), c.mark = hi.w;
-        if (TOPK && c.item >= 0) {   // the context's thresholds travel with its descriptor: (target, drafter)
-          c.tq = __ldg(P.thr_q + c.item);
-          c.tp = __ldg(P.thr_p + c.item);
-        }
       }
       return c;
     };
@@ -359,8 +361,6 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       it.tok0 = __shfl_sync(kFull, cur.tok0, l);
       it.r0 = __shfl_sync(kFull, cur.r0, l);
       it.u_final = __shfl_sync(kFull, cur.u_final, l);
-      const float tq_cur = TOPK ? __shfl_sync(kFull, cur.tq, l) : 0.0f;
-      const float tp_cur = TOPK ? __shfl_sync(kFull, cur.tp, l) : 0.0f;
       // the rows of the context after this one, for the L2 prefetch below
       const unsigned nraw = __ballot_sync(kFull, nxt.item >= 0);
       const int item_ahead = mask ? __shfl_sync(kFull, cur.item, __ffs(mask) - 1)
@@ -368,10 +368,6 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       bool ok = true;
       if (lane == 0) {
         S.work[i & 1] = it;                   // published by the mbarrier operation of the copy below
-        if (TOPK) {
-          S.thr[i & 1][0] = tq_cur;
-          S.thr[i & 1][1] = tp_cur;
-        }
         const bool withheld = it.item == P.withhold_item;   // self-test of the bounded waits: nothing is copied
         fence_proxy_async();
         if (!withheld) ctx_issue_drafter(P, it.item, smem + grp * stage_bytes, rowbytes, &bar_full_d[grp]);
@@ -478,11 +474,7 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
     const GroupItem cur = S.work[iter & 1];
     const int item = cur.item;
     if (item < 0) break;
-    float tq = 0.0f, tp = 0.0f;   // top-k thresholds of this context's target and drafter rows
-    if (TOPK) {
-      tq = S.thr[iter & 1][0];
-      tp = S.thr[iter & 1][1];
-    }
+    float tq = 0.0f, tp = 0.0f;   // top-k thresholds of this context's target and drafter rows (found below)
     const int b = item / R;
     const ChildInfo* kids = P.children + cur.cbase;
     const int nchild = cur.nchild;
@@ -534,6 +526,19 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       unpack2(v, lo, hi);
       return pack2(__fdiv_rn(lo, P.T), __fdiv_rn(hi, P.T));
     };
+    if (TOPK) {   // the drafter row's top-k threshold, from the staged row (the row came early)
+      auto zd = [&](int g, float (&z)[8]) {
+        uint64_t d2[4];
+        pairs_of(rd, g, d2);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          uint64_t l2 = d2[i];
+          if (!T_is_one) l2 = divide_T(l2);
+          unpack2(l2, z[2 * i], z[2 * i + 1]);
+        }
+      };
+      tp = tkg_kth_largest(zd, P.top_k, V, CH, S.tk, 0, grp, gt, &P.counters->n_slow_topk);
+    }
     // --- drafter first (its row came early): slice maximum and partial sum of numerators ---
 #pragma unroll
     for (int p = 0; p < NP; ++p) {
@@ -591,6 +596,22 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
     // row is streamed.  Every thread waits for itself (bounded); a wait that runs out is reported after
     // the next group barrier, where every thread sees it alike.
     if (!mbar_wait(&bar_full_t[grp], iter & 1, tries)) S.fail = 1;
+    if (TOPK) {   // the target row's threshold, on the guided (and tempered) logits the streaming loop forms
+      const uint64_t s2 = pack2(P.cfg_scale, P.cfg_scale);
+      auto zt = [&](int g, float (&z)[8]) {
+        uint64_t c2[4], u2[4];
+        pairs_of(rc, g, c2);
+        if (UNC) pairs_of(ru, g, u2);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          uint64_t l2 = c2[i];
+          if (UNC) l2 = fma2(s2, sub2(c2[i], u2[i]), u2[i]);
+          if (!T_is_one) l2 = divide_T(l2);
+          unpack2(l2, z[2 * i], z[2 * i + 1]);
+        }
+      };
+      tq = tkg_kth_largest(zt, P.top_k, V, CH, S.tk, 1, grp, gt, &P.counters->n_slow_topk);
+    }
     // --- target: guidance combine, slice maximum, numerators, partial sum; E replaces the raw rows ---
 #pragma unroll
     for (int p = 0; p < NP; ++p) {

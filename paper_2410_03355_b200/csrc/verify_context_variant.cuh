@@ -8,7 +8,7 @@ namespace lantern {
 template <int CHC, bool BF16, bool UNC>
 static cudaError_t launch_one(const VerifyParams& P, int grid, size_t smem_bytes, cudaStream_t st) {
   auto kc = lantern_context_kernel<CHC, BF16, UNC, LANTERN_VARIANT_TONE, LANTERN_VARIANT_JSD, LANTERN_VARIANT_TOPK>;
-  cudaError_t e = cudaFuncSetAttribute(kc, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+  cudaError_t e = cudaFuncSetAttribute(kc, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_bytes));
   if (e != cudaSuccess) return e;
   kc<<<grid, CTX_THREADS, smem_bytes, st>>>(P);
   return cudaGetLastError();

@@ -57,6 +57,7 @@ struct WorkItem {               // one context with children: everything its CTA
 struct GroupItem {              // the same, as a producer hands it to its consumer group through shared memory
   int item, cbase, nchild, node0, tok0, span0;
   float r0, u_final;
+  float bracket[2][4];          // top-k filter only: where the thresholds of the drafter row [0] and the target row [1] lie
 };
 
 struct VerifyParams {

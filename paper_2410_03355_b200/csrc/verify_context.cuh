@@ -239,10 +239,12 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       mbar_init(&bar_empty_d[g], GW);
       mbar_init(&bar_empty_t[g], GW);
       SG[g].fail = 0;
+      SG[g].tk.n_list[0] = SG[g].tk.n_list[1] = 0;
     }
     fence_mbar_init();
     fence_proxy_async();
   }
+  if (TOPK && tid < NGRP * GT) SG[tid >> LOG_GT].tk.hist[0][tid & (GT - 1)] = SG[tid >> LOG_GT].tk.hist[1][tid & (GT - 1)] = 0;
   __syncthreads();
 
   // ======================= producer warps =======================
@@ -336,6 +338,51 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       if (mask == 0) break;
       const int l = __ffs(mask) - 1;
       mask &= mask - 1;
+      // Top-k filter: where the two thresholds of this context lie, from a sample of its rows in global memory
+      // (they have been asked into L2 already) -- found now, while the group is busy with the context before.
+      float br_d[4] = {0.0f, 0.0f, 0.0f, 0.0f}, br_t[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+      if (TOPK) {
+        const int item_l = __shfl_sync(kFull, cur.item, l);
+        const size_t row = static_cast<size_t>(item_l) * V;
+        const size_t branch = static_cast<size_t>(P.B) * R * V;
+        auto raw8 = [&](const void* base, size_t elem, float (&z)[8]) {
+          if (BF16) {
+            const uint4 x = __ldg(reinterpret_cast<const uint4*>(static_cast<const unsigned short*>(base) + elem));
+            const uint32_t xw[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              z[2 * q] = __uint_as_float(xw[q] << 16);
+              z[2 * q + 1] = __uint_as_float(xw[q] & 0xffff0000u);
+            }
+          } else {
+            const float4 x0 = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(base) + elem));
+            const float4 x1 = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(base) + elem) + 1);
+            z[0] = x0.x, z[1] = x0.y, z[2] = x0.z, z[3] = x0.w, z[4] = x1.x, z[5] = x1.y, z[6] = x1.z, z[7] = x1.w;
+          }
+        };
+        auto zd_g = [&](int g, float (&z)[8]) {      // the same operations as the streaming loop, lane by lane
+          raw8(P.draft, row + static_cast<size_t>(g) * 8, z);
+          if (!TONE) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) z[e] = __fdiv_rn(z[e], P.T);
+          }
+        };
+        auto zt_g = [&](int g, float (&z)[8]) {
+          raw8(P.target, row + static_cast<size_t>(g) * 8, z);
+          if (UNC) {
+            float u[8];
+            raw8(P.target, branch + row + static_cast<size_t>(g) * 8, u);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) z[e] = __fmaf_rn(P.cfg_scale, __fsub_rn(z[e], u[e]), u[e]);
+          }
+          if (!TONE) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) z[e] = __fdiv_rn(z[e], P.T);
+          }
+        };
+        tkg_warp_bracket(zd_g, P.top_k, V, lane, br_d);
+        tkg_warp_bracket(zt_g, P.top_k, V, lane, br_t);
+      }
       // The drafter slot is free once every warp of the group has streamed the previous context's
       // drafter row (nothing reads it afterwards), i.e. while that context is still being decided:
       // the next drafter row travels early, and the group streams it while its target rows are copied.
@@ -361,6 +408,8 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       it.tok0 = __shfl_sync(kFull, cur.tok0, l);
       it.r0 = __shfl_sync(kFull, cur.r0, l);
       it.u_final = __shfl_sync(kFull, cur.u_final, l);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) it.bracket[0][q] = br_d[q], it.bracket[1][q] = br_t[q];
       // the rows of the context after this one, for the L2 prefetch below
       const unsigned nraw = __ballot_sync(kFull, nxt.item >= 0);
       const int item_ahead = mask ? __shfl_sync(kFull, cur.item, __ffs(mask) - 1)
@@ -537,7 +586,7 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
           unpack2(l2, z[2 * i], z[2 * i + 1]);
         }
       };
-      tp = tkg_kth_largest(zd, P.top_k, V, CH, S.tk, 0, grp, gt, &P.counters->n_slow_topk);
+      tp = tkg_kth_largest(zd, cur.bracket[0], P.top_k, V, CH, S.tk, 0, grp, gt, &P.counters->n_slow_topk);
     }
     // --- drafter first (its row came early): slice maximum and partial sum of numerators ---
 #pragma unroll
@@ -610,7 +659,7 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
           unpack2(l2, z[2 * i], z[2 * i + 1]);
         }
       };
-      tq = tkg_kth_largest(zt, P.top_k, V, CH, S.tk, 1, grp, gt, &P.counters->n_slow_topk);
+      tq = tkg_kth_largest(zt, cur.bracket[1], P.top_k, V, CH, S.tk, 1, grp, gt, &P.counters->n_slow_topk);
     }
     // --- target: guidance combine, slice maximum, numerators, partial sum; E replaces the raw rows ---
 #pragma unroll

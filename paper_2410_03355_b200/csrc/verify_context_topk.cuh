@@ -3,11 +3,12 @@
 // Included by verify_context.cuh; used by the TOPK variants of the fused kernel only.
 //
 // The row sits in shared memory as raw logits; `zchunk(g, z)` turns 16-byte group g into its eight
-// processed logits (guidance combine, temperature) with exactly the operations the streaming loop uses.
+// processed logits (guidance combine, temperature) with exactly the roundings of the streaming loop.
 // Steps, all exact in the end (the sample only decides where to look):
-//   1. one warp takes a 512-value sample spread over the row and finds, by bisection with warp-wide
+//   1. the group's producer warp, while the group is still busy with the context before, takes a
+//      512-value sample spread over the row (from global memory) and finds, by bisection with warp-wide
 //      counts, two values (lo, hi) whose sample ranks lie three standard deviations to either side of
-//      the rank the K-th largest is expected to have in the sample;
+//      the rank the K-th largest is expected to have in the sample; they travel with the work item;
 //   2. every thread goes over its 64 values once, without a branch: it counts those >= hi and notes
 //      down, one byte each, which of its values lie in [lo, hi); the notes of all threads are then
 //      gathered into one list (one counter update per warp), so that what follows is evenly spread;
@@ -37,7 +38,6 @@ struct GroupTopk {
   float tiny[2][TKG_TINY];          //     clears what a slow warp may still be reading from the call before
   int n_tiny[2], n_list[2];
   int wsum[GW][2];
-  float lo, hi, base, scale;        // the bracket, and the map value -> bin
 };
 
 // order-preserving bit pattern of a processed logit: NaN lowest, -0 as +0
@@ -151,67 +151,62 @@ __device__ __forceinline__ float tkg_exact_by_passes(ZF& zchunk, int K, int V, i
   return tkg_value(L);
 }
 
-// The K-th largest processed logit of the row behind `zchunk` (0 < K < V); every thread of the group calls
-// it and gets the same value.  CH = 16-byte groups per thread.
-// `which` = 0 for a context's drafter row, 1 for its target row (see GroupTopk).
+// Step 1 of the header comment, run by one warp (all 32 lanes call it and get the same values): the
+// bracket of a row from a 512-value sample.  `zchunk(g, z)` gives the eight processed logits of 16-byte
+// group g, from wherever the caller keeps the row.  out = {lo, hi, base, scale}.
 template <class ZF>
-__device__ __forceinline__ float tkg_kth_largest(ZF& zchunk, int K, int V, int CH, GroupTopk& T, int which, int grp,
-                                                 int gt, int* slow_count) {
-  const int gw = gt >> 5, lane = gt & 31;
+__device__ __forceinline__ void tkg_warp_bracket(ZF& zchunk, int K, int V, int lane, float (&out)[4]) {
   const float qnan = __int_as_float(0x7fc00000);
   const float pinf = __int_as_float(0x7f800000), ninf = __int_as_float(0xff800000);
-  // ---- 1. bracket from a sample (warp 0 of the group) ----
-  if (gw == 0) {
-    const int groups = V >> 3;
-    const int take = groups < 64 ? groups : 64;          // sampled 16-byte groups, spread evenly
-    float s[16];
-    uint32_t kmin = 0xffffffffu, kmax = 0u;
+  const int groups = V >> 3;
+  const int take = groups < 64 ? groups : 64;            // sampled 16-byte groups, spread evenly
+  float s[16];
+  uint32_t kmin = 0xffffffffu, kmax = 0u;
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const int j = lane + 32 * h;
-      float z[8];
-      if (j < take) zchunk(static_cast<int>(static_cast<long long>(j) * groups / take), z);
+  for (int h = 0; h < 2; ++h) {
+    const int j = lane + 32 * h;
+    float z[8];
+    if (j < take) zchunk(j * groups / take, z);           // j < 64 and groups <= 2048: no overflow
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const float v = j < take ? z[e] : qnan;
-        s[8 * h + e] = v;
-        const uint32_t kk = tkg_key(v);
-        if (kk > 0x007fffffu) {                           // above -inf
-          kmin = kk < kmin ? kk : kmin;
-          kmax = kk > kmax ? kk : kmax;
-        }
+    for (int e = 0; e < 8; ++e) {
+      const float v = j < take ? z[e] : qnan;
+      s[8 * h + e] = v;
+      const uint32_t kk = tkg_key(v);
+      if (kk > 0x007fffffu) {                             // above -inf
+        kmin = kk < kmin ? kk : kmin;
+        kmax = kk > kmax ? kk : kmax;
       }
-    }
-    kmin = __reduce_min_sync(kFull, kmin);
-    kmax = __reduce_max_sync(kFull, kmax);
-    float lo = ninf, hi = pinf;
-    if (kmax >= kmin) {                                   // the sample holds a finite value
-      const float ns = static_cast<float>(take * 8);
-      const float mean = static_cast<float>(K) * ns / static_cast<float>(V);
-      const float sd = sqrtf(mean * (1.0f - static_cast<float>(K) / static_cast<float>(V)));
-      const int slack = static_cast<int>(0.25f * sd) + 1;
-      const int r_hi = static_cast<int>(mean - 3.0f * sd) - slack - 1;
-      const int r_lo = static_cast<int>(mean + 3.0f * sd) + slack + 2;
-      tkg_sample_bracket(s, kmin, kmax, r_hi, r_lo, slack, r_hi > slack, r_lo < static_cast<int>(ns) - slack, lo, hi);
-      if (lane == 0) {
-        // bins: over [lo, hi) where both are finite, else over the sample's own range (values beyond it are clamped)
-        const float b0 = lo > ninf ? lo : tkg_value(kmin), b1 = hi < pinf ? hi : tkg_value(kmax);
-        T.base = b0;
-        T.scale = b1 > b0 ? static_cast<float>(TKG_BINS) / (b1 - b0) : 0.0f;
-      }
-    } else if (lane == 0) {
-      T.base = 0.0f;
-      T.scale = 0.0f;
-    }
-    if (lane == 0) {
-      T.lo = lo;
-      T.hi = hi;
     }
   }
-  T.hist[which][gt] = 0;                                  // GT == TKG_BINS
-  if (gt == 0) T.n_tiny[which] = 0, T.n_list[which] = 0;
-  gbar(grp);
-  const float lo = T.lo, hi = T.hi, base = T.base, scale = T.scale;
+  kmin = __reduce_min_sync(kFull, kmin);
+  kmax = __reduce_max_sync(kFull, kmax);
+  float lo = ninf, hi = pinf, base = 0.0f, scale = 0.0f;
+  if (kmax >= kmin) {                                     // the sample holds a finite value
+    const float ns = static_cast<float>(take * 8);
+    const float mean = static_cast<float>(K) * ns / static_cast<float>(V);
+    const float sd = sqrtf(mean * (1.0f - static_cast<float>(K) / static_cast<float>(V)));
+    const int slack = static_cast<int>(0.25f * sd) + 1;
+    const int r_hi = static_cast<int>(mean - 3.0f * sd) - slack - 1;
+    const int r_lo = static_cast<int>(mean + 3.0f * sd) + slack + 2;
+    tkg_sample_bracket(s, kmin, kmax, r_hi, r_lo, slack, r_hi > slack, r_lo < static_cast<int>(ns) - slack, lo, hi);
+    // bins: over [lo, hi) where both are finite, else over the sample's own range (values beyond it are clamped)
+    const float b0 = lo > ninf ? lo : tkg_value(kmin), b1 = hi < pinf ? hi : tkg_value(kmax);
+    base = b0;
+    scale = b1 > b0 ? static_cast<float>(TKG_BINS) / (b1 - b0) : 0.0f;
+  }
+  out[0] = lo, out[1] = hi, out[2] = base, out[3] = scale;
+}
+
+// Steps 2-4: the K-th largest processed logit of the row behind `zchunk` (0 < K < V), given the bracket
+// br = {lo, hi, base, scale}; every thread of the group calls it and gets the same value.  CH = 16-byte
+// groups per thread.  `which` = 0 for a context's drafter row, 1 for its target row (see GroupTopk).  The
+// histogram and the list counter of `which` are zero on entry and left zero on exit.
+template <class ZF>
+__device__ __forceinline__ float tkg_kth_largest(ZF& zchunk, const float (&br)[4], int K, int V, int CH, GroupTopk& T,
+                                                 int which, int grp, int gt, int* slow_count) {
+  const int gw = gt >> 5, lane = gt & 31;
+  if (gt == 0) T.n_tiny[which] = 0;                       // next touched behind two group barriers
+  const float lo = br[0], hi = br[1], base = br[2], scale = br[3];
   auto bin_of = [&](float v) {
     const float x = (v - base) * scale;
     return x < 0.0f ? 0 : (x >= static_cast<float>(TKG_BINS) ? TKG_BINS - 1 : static_cast<int>(x));
@@ -259,8 +254,9 @@ __device__ __forceinline__ float tkg_kth_largest(ZF& zchunk, int K, int V, int C
   }
   int c_in = n_in + (n_in > TKG_OWN ? (1 << 20) : 0);     // bit 20 and up: threads whose notes overflowed
   tkg_group_sum2(T, grp, gw, lane, c_hi, c_in);           // its barriers also publish the list
-  const bool overflow = (c_in >> 20) != 0 || (c_in & 0xfffff) > TKG_LIST;
+  const bool overflow = (c_in >> 20) != 0 || (c_in & 0xfffff) > TKG_LIST;   // (no overflowing thread: c_in = listed values)
   c_in &= 0xfffff;
+  if (gt == 0) T.n_list[which] = 0;                       // everybody has read it (the sum above went through two barriers)
   if (overflow || !(c_hi < K && K <= c_hi + c_in)) {
     if (gt == 0) atomicAdd(slow_count, 1);
     return tkg_exact_by_passes(zchunk, K, V, CH, T, grp, gt);
@@ -306,6 +302,7 @@ __device__ __forceinline__ float tkg_kth_largest(ZF& zchunk, int K, int V, int C
     }
   }
   gbar(grp);
+  T.hist[which][gt] = 0;                                  // nobody reads the histogram past this barrier
   const int n_tiny = T.n_tiny[which];
   if (n_tiny > TKG_TINY) {                                // a crowded bin (many equal values)
     if (gt == 0) atomicAdd(slow_count, 1);

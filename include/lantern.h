@@ -298,7 +298,8 @@ int lantern_verify_launch_count(int greedy, int top_k_active);
 lantern_status lantern_last_status(const void* workspace, void* cuda_stream, int32_t* out_bits);
 
 /* Work accounting of the last verification call that used `workspace` (waits for `cuda_stream`):
- *   out_counts[0]  contexts with at least one drafted child
+ *   out_counts[0]  contexts with at least one drafted child (in sampling: [1] + [2], which falls short of it
+ *                  only if the call was abandoned after a wait ran out)
  *   out_counts[1]  of those, the ones the fused pass evaluated
  *   out_counts[2]  the ones it left out because the walk could not reach them (Algorithm 1 stops
  *                  at the first rejection)

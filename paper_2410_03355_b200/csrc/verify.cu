@@ -123,7 +123,8 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
     }
     for (int c = 0; c < R; ++c)
       if (cnt[c] > 0) dep[c] = dst[dep[c]]++; // dep[c] becomes the context's rank
-    if (n_ctx > 0) atomicMax(&P.counters->n_rank, n_ctx);
+    // (thousands of warps would otherwise queue up on one address: most find the maximum already there)
+    if (n_ctx > *reinterpret_cast<volatile int*>(&P.counters->n_rank)) atomicMax(&P.counters->n_rank, n_ctx);
   }
   n_ctx = __shfl_sync(kFull, n_ctx, 0);
   __syncwarp();         // lane 0's writes to cur[], dep[] and kids[] are visible to the warp
@@ -136,7 +137,7 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
     const unsigned heavy = __ballot_sync(kFull, n >= 2);
     const unsigned light = __ballot_sync(kFull, n == 1);
     int hb = 0, lb = 0;
-    if (lane == 0) {
+    if (P.ctx_slots && lane == 0) {
       if (heavy) hb = atomicAdd(&P.counters->n_heavy, __popc(heavy));
       if (light) lb = atomicAdd(&P.counters->n_light, __popc(light));
     }
@@ -155,7 +156,7 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
         WorkItem w = {b * R + c, b * N + start, (n << 16) | f.node, f.span, f.token, f.r, u_final, b * R + din[c]};
         const int slot = dep[c] * B + b;
         P.work[slot] = w;
-        P.ctx_slots[n >= 2 ? hb + __popc(heavy & below) : cap - 1 - (lb + __popc(light & below))] = slot;
+        if (P.ctx_slots) P.ctx_slots[n >= 2 ? hb + __popc(heavy & below) : cap - 1 - (lb + __popc(light & below))] = slot;
       }
     }
   }
@@ -401,7 +402,9 @@ extern "C" lantern_status lantern_verify_counts(const void* workspace, void* cud
   Counters c;
   if (cudaMemcpyAsync(&c, workspace, sizeof(c), cudaMemcpyDeviceToHost, st) != cudaSuccess) return LANTERN_E_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return LANTERN_E_CUDA;
-  out_counts[0] = static_cast<int64_t>(c.n_heavy) + c.n_light;
+  // sampling keeps no count of its own: every context with children is either evaluated or left out
+  const int64_t listed = static_cast<int64_t>(c.n_heavy) + c.n_light;
+  out_counts[0] = listed ? listed : static_cast<int64_t>(c.n_evaluated) + c.n_skipped;
   out_counts[1] = c.n_evaluated;
   out_counts[2] = c.n_skipped;
   out_counts[3] = c.n_bonus;
@@ -536,7 +539,7 @@ static lantern_status verify_impl(const void* target_logits, const void* draft_l
   P.top_k = topk ? top_k : 0;
   P.thr_q = topk ? reinterpret_cast<float*>(ws + L.thrq) : nullptr;
   P.thr_p = topk ? reinterpret_cast<float*>(ws + L.thrp) : nullptr;
-  P.ctx_slots = reinterpret_cast<int32_t*>(ws + L.slots);
+  P.ctx_slots = greedy ? reinterpret_cast<int32_t*>(ws + L.slots) : nullptr;   // only the greedy kernels walk the compact list
   P.dead = ws + L.dead;
   P.wait_tries = g_wait_tries;
   P.withhold_item = g_withhold_item;

@@ -468,8 +468,8 @@ class Run:
         counts = self.lt.verify_counts(self.ws)
         greedy = self.greedy
         n_ctx = counts["contexts"]
-        ev_ctx = n_ctx if greedy else counts["evaluated"]
-        ev_nodes = self.B * self.N if greedy else counts["nodes_tested"]
+        ev_ctx = counts["evaluated"]
+        ev_nodes = counts["nodes_tested"]
         m_ctx, m_nodes = method_work(self.d["tree_parents"], self.out.accept_len, self.out.accept_path, self.N)
         ev_bytes = work_bytes(self.cfg, ev_ctx, ev_nodes, greedy)
         m_bytes = work_bytes(self.cfg, m_ctx, m_nodes, greedy)

@@ -306,7 +306,7 @@ lantern_status lantern_last_status(const void* workspace, void* cuda_stream, int
  *   out_counts[3]  next tokens drawn from a context's own q (bonus draws and degenerate residuals)
  *   out_counts[4]  drafted nodes the fused pass tested
  *   out_counts[5]  rows whose top-k threshold needed the slow exact search (with a top-k filter only)
- * out_counts holds six entries.  Greedy decoding evaluates every context: [1], [2] and [4] stay 0 there. */
+ * out_counts holds six entries. */
 lantern_status lantern_verify_counts(const void* workspace, void* cuda_stream, int64_t* out_counts);
 
 /* Self-test of the kernels' bounded waits (not part of the method).  Every wait for an on-chip copy

@@ -150,6 +150,8 @@ struct GreedyCtxShared {
   int done, accept;
   double thr;                       // JSD bound only: the current child's mass bound
   unsigned long long bar_full[GRING_MAX];
+  WorkItem item[GRING_MAX];         // the context whose rows are on their way into (or sit in) each staging area
+  int cursor;                       // next work slot this CTA looks at
 };
 
 // a neighbour entry, by an instruction the compiler neither hoists nor merges into a select
@@ -230,42 +232,57 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
   const uint32_t area_bytes = (UNC ? 2 : 1) * rowbytes;   // a multiple of 16: V % 8 == 0
   const float L_hi = 1.44269502162933349609375f;
   const float NEG_INF = __int_as_float(0xff800000);
-  const int n_heavy = P.counters->n_heavy;
-  const int total = n_heavy + P.counters->n_light;
-  const int cap = P.B * N;
+  const int total = P.counters->n_rank * P.B;   // occupied part of the slot array (breadth-first order per sequence)
   const int quads = V >> 2;
   const int G = gridDim.x;
-  auto slot = [&](int w) { return __ldg(P.ctx_slots + (w < n_heavy ? w : cap - 1 - (w - n_heavy))); };   // compact list -> work slot
+  int n_eval = 0, n_skip = 0, n_test = 0;       // thread 0: work accounting
+  // Thread 0 keeps the staging areas filled.  The CTA walks the slots blockIdx.x, blockIdx.x + G, ... and, as in
+  // the sampling pass, leaves out the empty ones and the contexts known to be unreachable (Algorithm 1 stops at
+  // the first rejection); a context whose parent is still undecided is evaluated anyway.
+  auto refill = [&](int area) {
+    for (;;) {
+      const int w = S.cursor;
+      if (w >= total) {
+        S.item[area].item = -1;
+        return;
+      }
+      S.cursor = w + G;
+      const int4 lo = __ldg(reinterpret_cast<const int4*>(P.work + w));
+      if (lo.x < 0) continue;
+      const int4 hi = __ldg(reinterpret_cast<const int4*>(P.work + w) + 1);
+      if (*reinterpret_cast<const volatile unsigned char*>(P.dead + hi.w) != 0) {
+        ++n_skip;
+        continue;
+      }
+      WorkItem wi;
+      wi.item = lo.x, wi.cbase = lo.y, wi.nchild_node0 = lo.z, wi.span0 = lo.w;
+      wi.tok0 = hi.x, wi.r0 = __int_as_float(hi.y), wi.u_final = __int_as_float(hi.z), wi.mark = hi.w;
+      S.item[area] = wi;
+      greedy_issue_rows<BF16, UNC>(P, wi.item, gsm + static_cast<size_t>(area) * area_bytes, rowbytes, &S.bar_full[area]);
+      ++n_eval;
+      return;
+    }
+  };
 
   if (tid == 0) {
     for (int r = 0; r < ring; ++r) mbar_init(reinterpret_cast<uint64_t*>(&S.bar_full[r]), 1);
     fence_mbar_init();
     S.status = 0;
     S.flags[0] = S.flags[1] = 0;
-    for (int r = 0; r < ring; ++r) {
-      const long long w = blockIdx.x + static_cast<long long>(r) * G;
-      if (w < total)
-        greedy_issue_rows<BF16, UNC>(P, P.work[slot(static_cast<int>(w))].item, gsm + static_cast<size_t>(r) * area_bytes,
-                                     rowbytes, &S.bar_full[r]);
-    }
+    S.cursor = blockIdx.x;
+    for (int r = 0; r < ring; ++r) refill(r);
   }
   __syncthreads();
-  if (static_cast<int>(blockIdx.x) >= total) return;   // nothing was requested for this CTA
 
-  WorkItem cur = P.work[slot(blockIdx.x)];
-  float tq = 0.0f;
-  if (TOPK) tq = __ldg(P.thr_q + cur.item);
-  uint32_t it = 0, phase = 0;
+  uint32_t phase = 0;
   int buf = 0;
-  for (long long w = blockIdx.x; w < total; w += G, ++it) {
-    // Loads that are consumed much later are issued without any select on their result (clamped
-    // indices instead of predicates), so that no instruction waits for them before their use:
-    // the next context's descriptor, the context that will take over this staging area, and the
-    // first child's neighbour entries.
-    const long long w_next = w + G < total ? w + G : w;
-    const long long w_refill = w + static_cast<long long>(ring) * G;
-    const WorkItem nxt = P.work[slot(static_cast<int>(w_next))];
-    const int refill = P.work[slot(static_cast<int>(w_refill < total ? w_refill : w))].item;
+  for (uint32_t it = 0;; ++it) {
+    const WorkItem cur = S.item[buf];
+    if (cur.item < 0) break;                    // the areas are refilled in order: an empty one ends the list
+    float tq = 0.0f;
+    if (TOPK) tq = __ldg(P.thr_q + cur.item);
+    // The first child's neighbour entries are consumed much later: issued without any select on their result
+    // (clamped indices instead of predicates), so that no instruction waits for them before their use.
     int nb[4];
     if (tid < GGT) {
       const int32_t* nrow0 = P.nbr + static_cast<size_t>(cur.tok0) * k;
@@ -328,8 +345,6 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
         S.ws[warp] = static_cast<double>(f);
       }
     }
-    float tq_next = 0.0f;   // the next context's threshold: its descriptor has arrived during the sweep
-    if (TOPK) tq_next = __ldg(P.thr_q + nxt.item);
     if (bad || !ok) atomicOr(&S.flags[it & 1], (bad ? 1 : 0) | (ok ? 0 : 2));
     __syncthreads();   // A
     if (warp == 0) {   // lane v combines warp v
@@ -358,9 +373,9 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
         P.records[cur.item] = rec;
         // give the copies still on their way to the other staging areas the same bounded wait
         for (int d = 1; d < ring; ++d) {
-          const long long wj = w + static_cast<long long>(d) * G;
           const uint32_t j = it + d;
-          if (wj < total) mbar_wait(reinterpret_cast<uint64_t*>(&S.bar_full[j % ring]), (j / ring) & 1, P.wait_tries);
+          if (S.item[j % ring].item >= 0)
+            mbar_wait(reinterpret_cast<uint64_t*>(&S.bar_full[j % ring]), (j / ring) & 1, P.wait_tries);
         }
       }
       __syncthreads();
@@ -380,6 +395,7 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
       const double thr_tvd = static_cast<double>(P.delta) * Z;   // the bound in units of the unnormalised sums
       const ChildInfo* kids = P.children + cur.cbase;
       for (int ci = 0; ci < (cur.nchild_node0 >> 16) && accepted < 0; ++ci) {
+        ++n_test;
         int node = cur.nchild_node0 & 0xffff, xt = cur.tok0;
         if (ci > 0) {
           const int4 info = __ldg(reinterpret_cast<const int4*>(kids + ci));
@@ -489,19 +505,39 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
         if (S.accept) accepted = node;
       }
     }
+    // Algorithm 1 goes on from the accepted child only: every context behind another child is dead (one
+    // contiguous range of marks per child, see the plan kernel)
+    {
+      const ChildInfo* kids = P.children + cur.cbase;
+      const int nchild = cur.nchild_node0 >> 16;
+      unsigned char* marks = P.dead + static_cast<size_t>(cur.item / R) * R;
+      for (int j = 0; j < nchild; ++j) {
+        int node_j = cur.nchild_node0 & 0xffff, span_j = cur.span0;
+        if (j > 0) {
+          const int4 kid = __ldg(reinterpret_cast<const int4*>(kids + j));
+          node_j = kid.x, span_j = kid.w;
+        }
+        if (node_j != accepted)
+          for (int o = tid; o < (span_j & 0xffff); o += GCT) marks[(span_j >> 16) + o] = 1;
+      }
+    }
     // every thread's reads of this staging area came before the barrier it passed last
     if (tid == 0) {
-      if (w_refill < total) greedy_issue_rows<BF16, UNC>(P, refill, raw, rowbytes, &S.bar_full[buf]);
       Record rec = {accepted, finite ? arg : -1, status | S.status, 0};
       P.records[cur.item] = rec;
       S.status = 0;
+      refill(buf);
     }
-    cur = nxt;
-    tq = tq_next;
+    __syncthreads();   // the area's next context (or the end of the list) is visible to everybody
     if (++buf == ring) {
       buf = 0;
       phase ^= 1;
     }
+  }
+  if (tid == 0) {
+    if (n_eval) atomicAdd(&P.counters->n_evaluated, n_eval);
+    if (n_skip) atomicAdd(&P.counters->n_skipped, n_skip);
+    if (n_test) atomicAdd(&P.counters->n_tested, n_test);
   }
 }
 

@@ -418,6 +418,19 @@ class Run:
         self.logit_gb = (d["target_logits"].numel() + (0 if self.greedy else d["draft_logits"].numel())) * \
             d["target_logits"].element_size() / 1e9
 
+    def variant(self, args):
+        """The same inputs and table under other settings (greedy decoding, logit filter, bound): own outputs and workspace."""
+        import copy
+        v = copy.copy(self)
+        torch, lt = self.torch, self.lt
+        v.args, v.greedy = args, args.greedy
+        v.T = 0.0 if args.greedy else self.d["T"]
+        v.ws = torch.empty(lt.verify_workspace_bytes(self.B, self.N, self.V, self.k, self.cfg["dtype"], args.top_k),
+                           dtype=torch.uint8, device="cuda")
+        v.out = lt.VerifyOutputs(*(None if t is None else torch.empty_like(t)
+                                   for t in (getattr(self.out, f.name) for f in __import__("dataclasses").fields(self.out))))
+        return v
+
     def step(self, out=None, trace=False):
         d, a = self.d, self.args
         return self.lt.verify(d["target_logits"], None if self.greedy else d["draft_logits"], d["cfg_scale"], self.T,
@@ -687,12 +700,39 @@ def main():
                                  "stream_operations_per_call": lt.verify_launch_count(False, False),
                                  "note": "back to back the 23 MB of rows stay in L2; flushed they come from HBM"}
         del lit
+        # the same call under the paper's other settings (same inputs, same table): greedy decoding (tau = 0), the
+        # top-k 1000 logit filter of the generation settings, the JSD bound
+        variants = {}
+        for vname, kw in (("greedy", dict(greedy=True)), ("top_k_1000", dict(top_k=1000)), ("jsd", dict(divergence="jsd"))):
+            va = argparse.Namespace(**{**vars(args), **kw})
+            vr = run.variant(va)
+            v_total, v_fused = vr.timed(20, 3)
+            v_acc = vr.accounting(v_fused, peak)
+            variants[vname] = {"ms_per_call": v_total / 20, "kernel_ms": v_fused,
+                               "positions_drafted_per_s": B * N / (v_total / 20 * 1e-3),
+                               "contexts_evaluated": v_acc["contexts_evaluated"], "GB_per_s": v_acc["achieved"],
+                               "frac_of_hbm_peak": v_acc["frac"],
+                               "mean_accept_len": float(vr.out.accept_len.float().mean().item())}
+            del vr
+        chain["variants"] = variants
         configs["batch_chain"] = chain
         del run, d, out
         torch.cuda.empty_cache()
         for name in ("tiny", "single_image", "px512_tree", "stress"):
             configs[name] = config_line(args, name, peak, steps=20, sample=16 if name != "tiny" else 64, flush=flush)
             torch.cuda.empty_cache()
+        # throughput mode of the stress trees: 16 of its steps (128 sequences each) flattened into one call
+        flat = Run(args, "stress", B=16 * WORKLOADS["stress"]["B"], seed=li.BASE_SEED + 7)
+        f_total, f_fused = flat.timed(10, 3)
+        f_acc = flat.accounting(f_fused, peak)
+        configs["stress"]["flattened_16_steps"] = {
+            "sequences_per_call": flat.B, "ms_per_call": f_total / 10, "kernel_ms": f_fused,
+            "positions_drafted_per_s": flat.B * flat.N / (f_total / 10 * 1e-3), "contexts": {
+                "with_children": f_acc["contexts_with_children"], "evaluated": f_acc["contexts_evaluated"],
+                "on_accepted_paths": f_acc["method_contexts"]},
+            "GB_per_s": f_acc["achieved"], "frac_of_hbm_peak": f_acc["frac"], "method_frac_of_hbm_peak": f_acc["method_frac"]}
+        del flat
+        torch.cuda.empty_cache()
         del flush
 
     if rank == 0:

@@ -262,14 +262,16 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
     const int G = gridDim.x * NGRP;              // producers in the grid
     const int me = blockIdx.x * NGRP + grp;
     const uint32_t tries = P.wait_tries;
-    // Slots per batch: a share of what is left that shrinks towards the end of the list (so that the
-    // groups finish together), but at least as many slots as it has taken so far to find one live
-    // context (tree workloads leave most slots empty or dead, and every batch costs a round trip).
+    // Slots per batch.  Few live contexts per batch (two; one towards the end of the list, so that the groups
+    // finish together): a batch is worked through in order, and the longer that takes the more of its
+    // contexts meet an undecided parent and are evaluated for nothing.  But as many slots as it has taken so
+    // far to find that many live ones: tree workloads leave most slots empty or dead, and every batch costs a
+    // round trip to the work list.
     int slots_seen = 0, live_seen = 0;
     auto batch_size = [&](int at) {
       const int share = (total - at) / (4 * G);
-      const int sparse = (slots_seen + 1) / (live_seen + 1);
-      const int s = share > sparse ? share : sparse;
+      const int live = share < 1 ? 1 : (share > 2 ? 2 : share);
+      const int s = live * ((slots_seen + 1) / (live_seen + 1));
       return s < 1 ? 1 : (s > 32 ? 32 : s);
     };
     struct Cand {

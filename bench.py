@@ -101,10 +101,10 @@ def method_work(parents, accept_len, accept_path, N: int):
 
 
 # DRAM traffic of the fused kernel from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum) of a
-# small call of the chain workload, as a ratio to the bytes of the contexts and nodes that call evaluated;
+# 1024-sequence call of the chain workload, as a ratio to the bytes of the 5348 contexts and nodes that call evaluated;
 # traffic grows in proportion to the contexts evaluated, so a full launch is scaled by its evaluated bytes.
 # Tied to the kernel revision the capture was taken on: any other revision reports null.
-NCU_TRAFFIC = {"kernel_revision": None, "workload": "batch_chain", "traffic_over_algorithmic": None}
+NCU_TRAFFIC = {"kernel_revision": 17, "workload": "batch_chain", "traffic_over_algorithmic": 562767360 / 547121792}
 
 
 def ncu_traffic(workload, alg_bytes):

@@ -33,7 +33,7 @@
 // evaluated anyway: with few sequences per call that keeps every SM busy (all contexts of a tree run
 // side by side), with many sequences it is rare, and the walk kernel reads only records on the
 // accepted path either way, so the result never depends on what was speculated.
-#define LANTERN_CONTEXT_KERNEL_REVISION 16   // bump on every change to this file
+#define LANTERN_CONTEXT_KERNEL_REVISION 17   // bump on every change to this file
 
 namespace lantern {
 
@@ -326,7 +326,7 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
     unsigned mask = filter(cur);
     int i = 0;        // contexts handed to the group so far
     bool clean = true;
-    for (;;) {
+    auto next_batch = [&]() {   // make `mask` non-empty if any live context is left
       while (mask == 0 && !cur_end) {
         cur = nxt;
         cur_end = nxt_end;
@@ -337,6 +337,9 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
         }
         mask = filter(cur);
       }
+    };
+    for (;;) {
+      next_batch();
       if (mask == 0) break;
       const int l = __ffs(mask) - 1;
       mask &= mask - 1;
@@ -412,10 +415,6 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       it.u_final = __shfl_sync(kFull, cur.u_final, l);
 #pragma unroll
       for (int q = 0; q < 4; ++q) it.bracket[0][q] = br_d[q], it.bracket[1][q] = br_t[q];
-      // the rows of the context after this one, for the L2 prefetch below
-      const unsigned nraw = __ballot_sync(kFull, nxt.item >= 0);
-      const int item_ahead = mask ? __shfl_sync(kFull, cur.item, __ffs(mask) - 1)
-                                  : (nraw && !cur_end ? __shfl_sync(kFull, nxt.item, __ffs(nraw) - 1) : -1);
       bool ok = true;
       if (lane == 0) {
         S.work[i & 1] = it;                   // published by the mbarrier operation of the copy below
@@ -427,7 +426,6 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
         if (ok && !withheld) {
           fence_proxy_async();
           ctx_issue_target<UNC>(P, it.item, smem + grp * stage_bytes, rowbytes, &bar_full_t[grp]);
-          if (item_ahead >= 0) ctx_prefetch_rows<BF16, UNC>(P, item_ahead, rowbytes);
         }
       }
       ok = __shfl_sync(kFull, ok ? 1 : 0, 0) != 0;
@@ -436,6 +434,14 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
       if (!ok) {
         clean = false;
         break;
+      }
+      // Look ahead: the next live context (a batch swap, if the current batch is used up, happens here, where
+      // nothing waits for it) and an L2 prefetch of its rows -- of a context that has passed the dead check,
+      // so that hardly any prefetched row goes unused.
+      next_batch();
+      if (mask) {
+        const int item_ahead = __shfl_sync(kFull, cur.item, __ffs(mask) - 1);
+        if (lane == 0) ctx_prefetch_rows<BF16, UNC>(P, item_ahead, rowbytes);
       }
     }
     if (lane == 0) {

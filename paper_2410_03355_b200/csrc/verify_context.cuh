@@ -835,10 +835,13 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
 
         // ---- A_{k,delta}(x~): gather + prefix scan with the strict bound ----
         double thr = delta * Zq_c;   // the bound in the units of the unnormalised sums
-        // Section 5.3.2: the mass whose JSD is delta; one thread, published by [scan 1] through the last
-        // slot of wt[], which nothing else touches between the start of a child and its [scan 2]
-        if (JSD && gt == GT - 32)
-          S.wt[8 * GW - 1] = jsd_mass_bound(delta, static_cast<double>(e_xt_bulk) / Zq_c) * Zq_c;
+        // Section 5.3.2: the mass whose JSD is delta; the group's last warp finds it together, published by
+        // [scan 1] through the last slot of wt[], which nothing else touches between the start of a child and
+        // its [scan 2]
+        if (JSD && gw == GW - 1) {
+          const double sstar = jsd_mass_bound_warp(delta, static_cast<double>(e_xt_bulk) / Zq_c, lane) * Zq_c;
+          if (lane == 0) S.wt[8 * GW - 1] = sstar;
+        }
         double carry = 0.0, sm = 0.0;
         int m = k - 1;
         bool cut = false;

@@ -23,7 +23,7 @@
 
 namespace lantern {
 
-constexpr int TKG_OWN = 16;         // bracket values a thread can note down
+constexpr int TKG_OWN = 24;         // bracket values a thread can note down (about five are expected)
 constexpr int TKG_LIST = 2048;      // bracket values of the whole row
 constexpr int TKG_BINS = 256;
 constexpr int TKG_TINY = 32;        // values of the wanted bin that one warp can rank
@@ -232,7 +232,7 @@ __device__ __forceinline__ float tkg_kth_largest(ZF& zchunk, const float (&br)[4
         const float v = z[e];
         c_hi += v >= hi;
         const bool in = v >= lo && v < hi;
-        if (in) T.code[(n_in & (TKG_OWN - 1)) * GT + gt] = static_cast<unsigned char>(ch * 8 + e);
+        if (in) T.code[(n_in < TKG_OWN ? n_in : TKG_OWN - 1) * GT + gt] = static_cast<unsigned char>(ch * 8 + e);
         n_in += in;
       }
     }
@@ -312,11 +312,10 @@ __device__ __forceinline__ float tkg_kth_largest(ZF& zchunk, const float (&br)[4
   // `rank` values not below it (equal values give the same answer)
   const float mine_v = lane < n_tiny ? T.tiny[which][lane] : __int_as_float(0xff800000);
   int gtr = 0, geq = 0;
-#pragma unroll 8
-  for (int j = 0; j < TKG_TINY; ++j) {
+  for (int j = 0; j < n_tiny; ++j) {                      // (a handful; the bound is the same for every thread)
     const float o = __shfl_sync(kFull, mine_v, j);
-    gtr += (j < n_tiny && o > mine_v) ? 1 : 0;
-    geq += (j < n_tiny && o >= mine_v) ? 1 : 0;
+    gtr += o > mine_v ? 1 : 0;
+    geq += o >= mine_v ? 1 : 0;
   }
   const unsigned hit = __ballot_sync(kFull, lane < n_tiny && gtr < rank && rank <= geq);
   if (hit == 0u) {                                        // cannot happen with a consistent histogram

@@ -39,7 +39,7 @@ namespace lantern {
 // the fused pass overwrites; contexts without children are marked as leaves.
 // ---------------------------------------------------------------------------------------
 constexpr int PLAN_WARPS = 4;
-constexpr int kPlanArrays = 7;   // per-warp arrays of N + 2 ints in shared memory
+constexpr int kPlanArrays = 12;  // per-warp arrays of N + 2 ints in shared memory
 
 __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyParams P) {
   extern __shared__ int plan_smem[];
@@ -54,7 +54,12 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
   int* siz = dst + (R + 1);                    // number of contexts in the subtree of context c, itself included
   int* din = siz + (R + 1);                    // depth-first (pre-order) position of context c
   int* nxt = din + (R + 1);                    // depth-first position the next child of context c gets
-  for (int i = lane; i <= R; i += 32) cnt[i] = 0, dst[i] = 0, siz[i] = 1;
+  int* s_par = nxt + (R + 1);                  // the sequence's parents, tokens and uniforms, staged once by all
+  int* s_tok = s_par + (R + 1);                //   lanes: the serial parts below then run out of shared memory
+  int* s_uni = s_tok + (R + 1);
+  int* s_pos = s_uni + (R + 1);                // place of node i in the child lists
+  int* s_first = s_pos + (R + 1);              // first child (smallest node index) of context c
+  for (int i = lane; i <= R; i += 32) cnt[i] = 0, dst[i] = 0, siz[i] = 1, s_first[i] = -1;
   __syncwarp();
   int status = 0;
   const float qnan = __int_as_float(0x7fc00000);
@@ -65,6 +70,8 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
     const int par = P.parents ? P.parents[o] : i - 1;
     if (par < -1 || par >= i) status |= LANTERN_ST_BAD_PARENT;
     else atomicAdd(&cnt[par + 1], 1);
+    s_par[i] = par;
+    s_tok[i] = tok;
     if (P.out_path) P.out_path[o] = -1;
     if (P.out_qa) P.out_qa[o] = qnan;
     if (P.out_px) P.out_px[o] = qnan;
@@ -74,7 +81,10 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
     for (int i = lane; i <= N; i += 32) {
       const float r = P.uniforms[static_cast<size_t>(b) * R + i];
       if (!(r >= 0.0f && r < 1.0f)) status |= LANTERN_ST_BAD_UNIFORM;
+      s_uni[i] = __float_as_int(r);
     }
+  } else {
+    for (int i = lane; i <= N; i += 32) s_uni[i] = 0;
   }
   for (int c = lane; c < R; c += 32) P.dead[static_cast<size_t>(b) * R + c] = 0;
   status = __reduce_or_sync(kFull, status);
@@ -96,22 +106,17 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
     // Subtree sizes (children have larger indices than their parents) and pre-order positions: the
     // contexts behind a node then occupy one contiguous range of positions, which is what lets the
     // fused pass strike a whole rejected subtree with a few byte stores.
-    for (int i = N - 1; i >= 0; --i) {
-      const int par = P.parents ? P.parents[static_cast<size_t>(b) * N + i] : i - 1;
-      siz[par + 1] += siz[i + 1];
-    }
+    for (int i = N - 1; i >= 0; --i) siz[s_par[i] + 1] += siz[i + 1];
     dep[0] = 0;
     din[0] = 0;
     nxt[0] = 1;
     for (int i = 0; i < N; ++i) {
-      const size_t o = static_cast<size_t>(b) * N + i;
-      const int par = P.parents ? P.parents[o] : i - 1;
+      const int par = s_par[i];
       din[i + 1] = nxt[par + 1];
       nxt[par + 1] += siz[i + 1];
       nxt[i + 1] = din[i + 1] + 1;
-      ChildInfo ci = {i, P.tokens[o], P.uniforms ? P.uniforms[static_cast<size_t>(b) * R + i] : 0.0f,
-                      (din[i + 1] << 16) | siz[i + 1]};
-      kids[cur[par + 1]++] = ci;
+      s_pos[i] = cur[par + 1]++;
+      if (s_first[par + 1] < 0) s_first[par + 1] = i;
       dep[i + 1] = dep[par + 1] + 1;
     }
     for (int c = 0; c < R; ++c)
@@ -127,9 +132,13 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
     if (n_ctx > *reinterpret_cast<volatile int*>(&P.counters->n_rank)) atomicMax(&P.counters->n_rank, n_ctx);
   }
   n_ctx = __shfl_sync(kFull, n_ctx, 0);
-  __syncwarp();         // lane 0's writes to cur[], dep[] and kids[] are visible to the warp
+  __syncwarp();         // lane 0's writes to the shared arrays are visible to the warp
+  for (int i = lane; i < N; i += 32) {   // the child lists, written by all lanes
+    ChildInfo ci = {i, s_tok[i], __int_as_float(s_uni[i]), (din[i + 1] << 16) | siz[i + 1]};
+    kids[s_pos[i]] = ci;
+  }
   for (int r = n_ctx + lane; r < N; r += 32) P.work[static_cast<size_t>(r) * B + b].item = -1;
-  const float u_final = P.uniforms ? P.uniforms[static_cast<size_t>(b) * R + N] : 0.0f;
+  const float u_final = __int_as_float(s_uni[N]);
   const int cap = B * N;
   for (int base = 0; base < R; base += 32) {
     const int c = base + lane;
@@ -152,8 +161,9 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
         Record pending = {-1, -1, LANTERN_ST_INTERNAL, 0};   // stands until the fused pass has evaluated the context
         P.records[static_cast<size_t>(b) * R + c] = pending;
         const int start = cur[c] - n;
-        const ChildInfo f = kids[start];
-        WorkItem w = {b * R + c, b * N + start, (n << 16) | f.node, f.span, f.token, f.r, u_final, b * R + din[c]};
+        const int f = s_first[c];             // the context's first child (smallest node index)
+        WorkItem w = {b * R + c, b * N + start, (n << 16) | f, (din[f + 1] << 16) | siz[f + 1], s_tok[f],
+                      __int_as_float(s_uni[f]), u_final, b * R + din[c]};
         const int slot = dep[c] * B + b;
         P.work[slot] = w;
         if (P.ctx_slots) P.ctx_slots[n >= 2 ? hb + __popc(heavy & below) : cap - 1 - (lb + __popc(light & below))] = slot;

@@ -96,6 +96,24 @@ def test_trees(depth, N):
     assert n_sib > 24 * 4 * 3 * 1.5        # sibling rounds were exercised
 
 
+def test_long_chain_and_wide_tree():
+    """Draft lengths far beyond the paper's settings: the plan's per-sequence arrays, the breadth-first ranks
+    and the dead marks over hundreds of contexts (a rejection at depth d strikes the N - d contexts behind it)."""
+    V, k = 256, 16
+    cb = li.codebook_gaussian(V, 8, seed=39)
+    host = oracle.build_neighbors(cb, k)[0]
+    dev = torch.from_numpy(host).cuda()
+    inp = li.verify_inputs(5, 300, V, dtype=li.BF16, has_uncond=True, cfg_scale=1.5, sigma_target=1.0, sigma_draft=0.15,
+                           rho=0.95, seed=61)
+    res = check(inp, host, dev, 0.3, min_tested=5)
+    assert res["accept_mean"] > 3
+    wide = li.verify_inputs(6, 200, V, dtype=li.F32, has_uncond=False, cfg_scale=1.0, sigma_draft=0.6,
+                            parents=li.tree_parents(6, 200, depth=6, seed=4), seed=62)
+    check(wide, host, dev, 0.1, min_tested=6)
+    inp = li.verify_inputs(2, 1024, V, dtype=li.BF16, has_uncond=False, cfg_scale=1.0, sigma_draft=0.05, seed=63)
+    check(inp, host, dev, 0.5, min_tested=2)          # the longest supported chain
+
+
 def test_chain_equals_explicit_tree():
     V, k = 1024, 32
     cb = li.codebook_gaussian(V, 8, seed=33)

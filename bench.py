@@ -543,7 +543,23 @@ def config_line(args, name, peak, run=None, steps=20, sample=16, flush=None):
         line["parity"] = run.parity_sample(sample)
     if own:
         del run
+        lit_B = li_config(name)["B"]
+        if lit_B != B and name != "tiny":
+            # the configuration's literal call (one verification step of its batch), plain stream launches
+            import lantern_inputs as li
+            lit = Run(args, name, B=lit_B, seed=li.BASE_SEED + 5)
+            t_warm, f_warm = lit.timed(100, 5)
+            t_cold, _ = lit.timed(30, 3, flush=flush)
+            line["literal_call"] = {"sequences_per_call": lit_B, "us_per_call_back_to_back": 1e3 * t_warm / 100,
+                                    "us_per_call_l2_flushed": 1e3 * t_cold / 30, "fused_kernel_us": 1e3 * f_warm,
+                                    "mean_accept_len": float(lit.out.accept_len.float().mean().item())}
+            del lit
     return line
+
+
+def li_config(name):
+    import lantern_inputs as li
+    return li.CONFIGS[WORKLOADS[name]["config"]]
 
 
 def main():

@@ -169,6 +169,12 @@ lantern_status lantern_build_neighbors_metric(const float* codebook, int V, int 
  *                  values of a test made ahead of time that the walk did not need.  Each may be NULL.
  *   workspace       lantern_verify_workspace_bytes(B, N, V, k, dtype) bytes, 256-byte aligned
  *
+ * The call only enqueues work on cuda_stream (one memset and four or five kernels): it allocates
+ * nothing, reads nothing back and does not wait for the stream, and it re-initialises the part
+ * of the workspace it relies on.  It may therefore be recorded by a stream capture and replayed
+ * as a CUDA graph on inputs rewritten in place; make one call with the same shape, logit type
+ * and options outside the capture first (kernel attributes are set then).
+ *
  * lantern_verify_workspace_bytes returns 0 for sizes lantern_verify would refuse.
  * ---------------------------------------------------------------------------------------- */
 size_t lantern_verify_workspace_bytes(int B, int N, int V, int k, int dtype);

@@ -21,8 +21,11 @@ namespace lantern {
 constexpr int BT = 512;          // threads of the per-row kernel
 constexpr int BW = BT / 32;
 constexpr int SMALL_D = 32;
-constexpr int TILE = 64;         // distance tile edge
+constexpr int TM = 128;          // distance tile edge (rows and columns of one CTA)
 constexpr int DK = 16;           // dimensions staged per step
+constexpr int HB = 11;           // radix-select digit: 2048 bins, kept in the (still unused) list area
+constexpr int HBINS = 1 << HB;
+constexpr int FAST_POP = 256;    // largest bin the counting-sort path ranks by pairwise comparison
 
 struct BuildParams {
   const float* codebook;
@@ -32,54 +35,127 @@ struct BuildParams {
   int V, D, k, row0;
 };
 
+// Two fp32 lanes in one 64-bit register; each lane of the packed operations rounds exactly like the
+// scalar instruction, so the key sequence is unchanged.
+__device__ __forceinline__ unsigned long long dup2(float a) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %1};" : "=l"(r) : "f"(a));
+  return r;
+}
+__device__ __forceinline__ unsigned long long sub2(unsigned long long a, unsigned long long b) {
+  unsigned long long r;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+
 // ---------------------------------------------------------------------------------------
-// keys of a block of rows, large D
+// keys of a block of rows, large D: a 128 x 128 tile per CTA, 8 x 8 accumulators per thread
+// (rows ty*4.. and 64+ty*4.., columns tx*4.. and 64+tx*4.., so that every shared-memory read is
+// one conflict-free 16-byte load), the next 16 dimensions fetched into registers while the
+// current ones are used.  Every (i, j) accumulator still runs over d in order.
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) lantern_distance_tile_kernel(const float* __restrict__ cb, uint32_t* out, int V,
-                                                                    int D, int row0, int rows) {
-  __shared__ float As[TILE][DK + 1];
-  __shared__ float Bs[TILE][DK + 1];
+__device__ __forceinline__ float4 fetch_quad(const float* __restrict__ cb, int row, int row_end, int D, int d, bool vec) {
+  float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);   // zero padding adds fma(0, 0, acc) = acc exactly
+  if (row < row_end) {
+    const float* p = cb + static_cast<size_t>(row) * D + d;
+    if (vec && d + 3 < D) {
+      v = __ldg(reinterpret_cast<const float4*>(p));
+    } else {
+      if (d < D) v.x = __ldg(p);
+      if (d + 1 < D) v.y = __ldg(p + 1);
+      if (d + 2 < D) v.z = __ldg(p + 2);
+      if (d + 3 < D) v.w = __ldg(p + 3);
+    }
+  }
+  return v;
+}
+
+__global__ void __launch_bounds__(256, 2) lantern_distance_tile_kernel(const float* __restrict__ cb, uint32_t* out, int V,
+                                                                       int D, int row0, int rows) {
+  __shared__ __align__(16) float As[DK][TM];
+  __shared__ __align__(16) float Bs[DK][TM];
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-  const int rbase = row0 + blockIdx.y * TILE, cbase = blockIdx.x * TILE;
-  float acc[4][4];
+  const int rbase = row0 + blockIdx.y * TM, cbase = blockIdx.x * TM;
+  const int row_end = (row0 + rows < V) ? row0 + rows : V;
+  const bool vec = (D & 3) == 0;
+  unsigned long long acc[8][4];
 #pragma unroll
-  for (int r = 0; r < 4; ++r)
+  for (int r = 0; r < 8; ++r)
 #pragma unroll
-    for (int c = 0; c < 4; ++c) acc[r][c] = 0.0f;
+    for (int c = 0; c < 4; ++c) acc[r][c] = 0ull;
+  // staging: element e = l * 256 + tid of a 128 x 16 tile is (row e & 127, dimensions 4 * (e >> 7) ..+3)
+  const int srow = tid & 127, squad = tid >> 7;
+  float4 ra[2], rb[2];
+#pragma unroll
+  for (int l = 0; l < 2; ++l) {
+    ra[l] = fetch_quad(cb, rbase + srow, row_end, D, 4 * (squad + 2 * l), vec);
+    rb[l] = fetch_quad(cb, cbase + srow, V, D, 4 * (squad + 2 * l), vec);
+  }
   for (int d0 = 0; d0 < D; d0 += DK) {
 #pragma unroll
-    for (int l = 0; l < (TILE * DK) / 256; ++l) {
-      const int e = l * 256 + tid, rr = e / DK, dd = e % DK;
-      const int gr = rbase + rr, gc = cbase + rr, gd = d0 + dd;
-      As[rr][dd] = (gr < row0 + rows && gr < V && gd < D) ? cb[static_cast<size_t>(gr) * D + gd] : 0.0f;
-      Bs[rr][dd] = (gc < V && gd < D) ? cb[static_cast<size_t>(gc) * D + gd] : 0.0f;
+    for (int l = 0; l < 2; ++l) {
+      const int q = 4 * (squad + 2 * l);
+      As[q][srow] = ra[l].x;
+      As[q + 1][srow] = ra[l].y;
+      As[q + 2][srow] = ra[l].z;
+      As[q + 3][srow] = ra[l].w;
+      Bs[q][srow] = rb[l].x;
+      Bs[q + 1][srow] = rb[l].y;
+      Bs[q + 2][srow] = rb[l].z;
+      Bs[q + 3][srow] = rb[l].w;
     }
     __syncthreads();
+    if (d0 + DK < D) {
 #pragma unroll
-    for (int dd = 0; dd < DK; ++dd) {   // zero padding beyond D adds fma(0,0,acc) = acc exactly
-      float a[4], b[4];
+      for (int l = 0; l < 2; ++l) {
+        ra[l] = fetch_quad(cb, rbase + srow, row_end, D, d0 + DK + 4 * (squad + 2 * l), vec);
+        rb[l] = fetch_quad(cb, cbase + srow, V, D, d0 + DK + 4 * (squad + 2 * l), vec);
+      }
+    }
 #pragma unroll
-      for (int r = 0; r < 4; ++r) a[r] = As[ty + 16 * r][dd];
+    for (int dd = 0; dd < DK; ++dd) {
+      const float4 a0 = *reinterpret_cast<const float4*>(&As[dd][ty * 4]);
+      const float4 a1 = *reinterpret_cast<const float4*>(&As[dd][64 + ty * 4]);
+      const ulonglong2 b0 = *reinterpret_cast<const ulonglong2*>(&Bs[dd][tx * 4]);
+      const ulonglong2 b1 = *reinterpret_cast<const ulonglong2*>(&Bs[dd][64 + tx * 4]);
+      const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+      const unsigned long long b[4] = {b0.x, b0.y, b1.x, b1.y};
 #pragma unroll
-      for (int c = 0; c < 4; ++c) b[c] = Bs[tx + 16 * c][dd];
-#pragma unroll
-      for (int r = 0; r < 4; ++r)
+      for (int r = 0; r < 8; ++r) {
+        const unsigned long long aa = dup2(a[r]);
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-          const float t = __fsub_rn(a[r], b[c]);
-          acc[r][c] = __fmaf_rn(t, t, acc[r][c]);
+          const unsigned long long t = sub2(aa, b[c]);
+          acc[r][c] = fma2(t, t, acc[r][c]);
         }
+      }
     }
     __syncthreads();
   }
+  const bool vec_out = (V & 3) == 0;
 #pragma unroll
-  for (int r = 0; r < 4; ++r) {
-    const int gr = rbase + ty + 16 * r;
-    if (gr >= row0 + rows || gr >= V) continue;
+  for (int r = 0; r < 8; ++r) {
+    const int gr = rbase + (r < 4 ? ty * 4 + r : 64 + ty * 4 + (r - 4));
+    if (gr >= row_end) continue;
+    uint32_t* orow = out + static_cast<size_t>(gr - row0) * V;
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      const int gc = cbase + tx + 16 * c;
-      if (gc < V) out[static_cast<size_t>(gr - row0) * V + gc] = __float_as_uint(acc[r][c]);
+    for (int h = 0; h < 2; ++h) {
+      const int gc = cbase + 64 * h + tx * 4;
+      const unsigned long long p0 = acc[r][2 * h], p1 = acc[r][2 * h + 1];
+      const uint32_t w[4] = {static_cast<uint32_t>(p0), static_cast<uint32_t>(p0 >> 32), static_cast<uint32_t>(p1),
+                             static_cast<uint32_t>(p1 >> 32)};
+      if (vec_out && gc + 3 < V) {
+        *reinterpret_cast<uint4*>(orow + gc) = make_uint4(w[0], w[1], w[2], w[3]);
+      } else {
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          if (gc + c < V) orow[gc + c] = w[c];
+      }
     }
   }
 }
@@ -87,24 +163,68 @@ __global__ void __launch_bounds__(256) lantern_distance_tile_kernel(const float*
 // ---------------------------------------------------------------------------------------
 // one row: keys -> select -> sort -> store
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(BT) lantern_knn_row_kernel(BuildParams P, int P2 /* pow2 >= k-1 */) {
+__device__ __forceinline__ unsigned long long shfl_xor_u64(unsigned long long x, int m) {
+  const unsigned lo = __shfl_xor_sync(kFull, static_cast<unsigned>(x), m);
+  const unsigned hi = __shfl_xor_sync(kFull, static_cast<unsigned>(x >> 32), m);
+  return (static_cast<unsigned long long>(hi) << 32) | lo;
+}
+
+// Bitonic merge steps of strides 32..1 on one 64-element block held by a warp (elements lane and
+// lane + 32), for every merge size from size_lo to size_hi whose strides all lie inside the block.
+__device__ __forceinline__ void bitonic_block64(unsigned long long* list, int block, int lane, int size_lo, int size_hi) {
+  const int e0 = block * 64 + lane, e1 = e0 + 32;
+  unsigned long long x0 = list[e0], x1 = list[e1];
+  for (int size = size_lo; size <= size_hi; size <<= 1) {
+    if (size >= 64) {
+      const bool up = (e0 & size) == 0;
+      if ((x0 > x1) == up) {
+        const unsigned long long t = x0;
+        x0 = x1;
+        x1 = t;
+      }
+    }
+    for (int stride = size >= 64 ? 16 : (size >> 1); stride > 0; stride >>= 1) {
+      const bool am_lo = (lane & stride) == 0;
+      const unsigned long long o0 = shfl_xor_u64(x0, stride), o1 = shfl_xor_u64(x1, stride);
+      const bool up0 = (e0 & size) == 0, up1 = (e1 & size) == 0;
+      x0 = (am_lo == up0) ? (x0 < o0 ? x0 : o0) : (x0 > o0 ? x0 : o0);
+      x1 = (am_lo == up1) ? (x1 < o1 ? x1 : o1) : (x1 > o1 ? x1 : o1);
+    }
+  }
+  list[e0] = x0;
+  list[e1] = x1;
+}
+
+__global__ void __launch_bounds__(BT) lantern_knn_row_kernel(BuildParams P, int P2 /* pow2 >= max(k-1, 64) */) {
   extern __shared__ __align__(16) unsigned char dsm[];
   uint32_t* keys = reinterpret_cast<uint32_t*>(dsm);                                  // [V]
   unsigned long long* list =
       reinterpret_cast<unsigned long long*>(dsm + ((static_cast<size_t>(P.V) * 4 + 15) & ~size_t(15)));  // [P2]
-  __shared__ int hist[256];
+  // [HBINS] 16-bit counters, two to a word (a row has fewer than 65536 keys); used before the list is filled
+  unsigned* hist = reinterpret_cast<unsigned*>(list);
+  unsigned short* list16 = reinterpret_cast<unsigned short*>(hist + HBINS / 2);   // [k - 1 + FAST_POP] indices, fast path
+  auto bin_count = [hist](int b) { return static_cast<int>((hist[b >> 1] >> ((b & 1) << 4)) & 0xffffu); };
   __shared__ int wcnt[BW];
+  __shared__ uint32_t wmin[BW], wmax[BW];
   __shared__ float ai[SMALL_D];
-  __shared__ int s_digit, s_below, s_cnt;
+  __shared__ int s_digit, s_below, s_ties, s_cnt;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int V = P.V, D = P.D, K = P.k - 1;
   const int i = P.row0 + blockIdx.x;
 
-  // ---- keys ----
+  // ---- keys (and their range over j != i) ----
+  uint32_t kmin = 0xffffffffu, kmax = 0u;
   if (P.scratch) {
     const uint32_t* src = P.scratch + static_cast<size_t>(blockIdx.x) * V;
-    for (int j = tid; j < V; j += BT) keys[j] = src[j];
+    for (int j = tid; j < V; j += BT) {
+      const uint32_t key = src[j];
+      keys[j] = key;
+      if (j != i) {
+        kmin = key < kmin ? key : kmin;
+        kmax = key > kmax ? key : kmax;
+      }
+    }
   } else {
     if (tid < D) ai[tid] = P.codebook[static_cast<size_t>(i) * D + tid];
     __syncthreads();
@@ -123,7 +243,12 @@ __global__ void __launch_bounds__(BT) lantern_knn_row_kernel(BuildParams P, int 
           t = __fsub_rn(ai[d + 3], v.w);
           acc = __fmaf_rn(t, t, acc);
         }
-        keys[j] = __float_as_uint(acc);
+        const uint32_t key = __float_as_uint(acc);
+        keys[j] = key;
+        if (j != i) {
+          kmin = key < kmin ? key : kmin;
+          kmax = key > kmax ? key : kmax;
+        }
       }
     } else {
       for (int j = tid; j < V; j += BT) {
@@ -133,83 +258,165 @@ __global__ void __launch_bounds__(BT) lantern_knn_row_kernel(BuildParams P, int 
           const float t = __fsub_rn(ai[d], __ldg(b + d));
           acc = __fmaf_rn(t, t, acc);
         }
-        keys[j] = __float_as_uint(acc);
+        const uint32_t key = __float_as_uint(acc);
+        keys[j] = key;
+        if (j != i) {
+          kmin = key < kmin ? key : kmin;
+          kmax = key > kmax ? key : kmax;
+        }
       }
     }
   }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const uint32_t a = __shfl_xor_sync(kFull, kmin, o), b = __shfl_xor_sync(kFull, kmax, o);
+    kmin = a < kmin ? a : kmin;
+    kmax = b > kmax ? b : kmax;
+  }
+  if (lane == 0) {
+    wmin[warp] = kmin;
+    wmax[warp] = kmax;
+  }
+  if (tid == 0) s_cnt = 0;
   __syncthreads();
   const uint32_t self_key = keys[i];
-  __syncthreads();
-  if (tid == 0) {
-    keys[i] = 0xffffffffu;   // the code itself is placed in slot 0, not ranked
-    s_cnt = 0;
+#pragma unroll
+  for (int w = 0; w < BW; ++w) {
+    kmin = wmin[w] < kmin ? wmin[w] : kmin;
+    kmax = wmax[w] > kmax ? wmax[w] : kmax;
   }
-  __syncthreads();
 
   if (K > 0) {
-    // ---- radix select: tau = K-th smallest key; `need` ties at tau are taken, smallest index first ----
-    uint32_t prefix = 0, mask = 0;
-    int need = K, ties_total = 0;
-    for (int pass = 0; pass < 4; ++pass) {
-      const int shift = 24 - 8 * pass;
-      if (tid < 256) hist[tid] = 0;
+    // ---- radix select on rel = key - kmin, 11 bits at a time from the top of the occupied range:
+    //      tau = K-th smallest key over j != i; `need` ties at tau are taken, smallest index first ----
+    const uint32_t range = kmax - kmin;
+    int hi = range ? 32 - __clz(range) : 0;
+    uint32_t prefix = 0;
+    int need = K, ties_total = V - 1;
+    bool first_pass = true;
+    while (hi > 0) {
+      const int lo = hi > HB ? hi - HB : 0;
+      const uint32_t dmask = (1u << (hi - lo)) - 1u;
+      for (int t = tid; t < HBINS / 2; t += BT) hist[t] = 0u;
       __syncthreads();
       for (int j = tid; j < V; j += BT) {
-        const uint32_t key = keys[j];
-        if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 0xff], 1);
+        const uint32_t rel = keys[j] - kmin;
+        if (j != i && (hi >= 32 || (rel >> hi) == (prefix >> hi))) {
+          const uint32_t b = (rel >> lo) & dmask;
+          atomicAdd(&hist[b >> 1], 1u << ((b & 1u) << 4));
+        }
       }
       __syncthreads();
-      if (warp == 0) {
-        int loc[8], s = 0;
+      int loc[HBINS / BT], s = 0;
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          loc[q] = hist[lane * 8 + q];
-          s += loc[q];
-        }
-        int incl = s;
+      for (int q = 0; q < HBINS / BT; ++q) {
+        loc[q] = bin_count(tid * (HBINS / BT) + q);
+        s += loc[q];
+      }
+      int incl = s;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const int t = __shfl_up_sync(kFull, incl, o);
-          if (lane >= o) incl += t;
-        }
-        const int excl = incl - s;
-        if (excl < need && need <= incl) {   // exactly one lane
-          int run = excl;
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(kFull, incl, o);
+        if (lane >= o) incl += t;
+      }
+      if (lane == 31) wcnt[warp] = incl;
+      __syncthreads();
+      int excl = incl - s;
 #pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            if (run < need && need <= run + loc[q]) {
-              s_digit = lane * 8 + q;
-              s_below = run;
-            }
-            run += loc[q];
+      for (int w = 0; w < BW; ++w)
+        if (w < warp) excl += wcnt[w];
+      if (excl < need && need <= excl + s) {   // exactly one thread
+        int run = excl;
+#pragma unroll
+        for (int q = 0; q < HBINS / BT; ++q) {
+          if (run < need && need <= run + loc[q]) {
+            s_digit = tid * (HBINS / BT) + q;
+            s_below = run;
+            s_ties = loc[q];
           }
+          run += loc[q];
         }
       }
       __syncthreads();
-      const int digit = s_digit;
+      if (first_pass) {
+        // Common case: no bin up to the one that holds the K-th key is crowded.  The prefix sums of the
+        // histogram are then the places of a counting sort by bin: scatter the indices of those keys,
+        // rank every key inside its bin by (key, index), and store it at its final place.
+        first_pass = false;
+        const int digit = s_digit, n_cand = s_below + s_ties;
+        bool crowded = false;
+#pragma unroll
+        for (int q = 0; q < HBINS / BT; ++q) crowded |= (tid * (HBINS / BT) + q <= digit) && loc[q] > FAST_POP;
+        if (!__syncthreads_or(crowded)) {
+          // own words only: each counter becomes its bin's cursor (offsets stay below 65536; bins past `digit`
+          // are never advanced)
+          static_assert(HBINS / BT == 4, "a thread owns two words of counters");
+          hist[2 * tid] = static_cast<unsigned>(excl) | (static_cast<unsigned>(excl + loc[0]) << 16);
+          hist[2 * tid + 1] = static_cast<unsigned>(excl + loc[0] + loc[1]) |
+                              (static_cast<unsigned>(excl + loc[0] + loc[1] + loc[2]) << 16);
+          __syncthreads();
+          for (int j = tid; j < V; j += BT) {
+            const int b = static_cast<int>((keys[j] - kmin) >> lo);
+            if (j != i && b <= digit) {
+              const int sh = (b & 1) << 4;
+              const unsigned old = atomicAdd(&hist[b >> 1], 1u << sh);
+              list16[(old >> sh) & 0xffffu] = static_cast<unsigned short>(j);
+            }
+          }
+          __syncthreads();   // every cursor now holds the end of its bin = the start of the next
+          int32_t* irow = P.idx + static_cast<size_t>(i) * P.k;
+          float* drow = P.dist ? P.dist + static_cast<size_t>(i) * P.k : nullptr;
+          if (tid == 0) {
+            irow[0] = i;
+            if (drow) drow[0] = __uint_as_float(self_key);
+          }
+          for (int t = tid; t < n_cand; t += BT) {
+            const unsigned j = list16[t];
+            const uint32_t key = keys[j];
+            const int b = static_cast<int>((key - kmin) >> lo);
+            const int start = b ? bin_count(b - 1) : 0, end = bin_count(b);
+            const unsigned long long comp = (static_cast<unsigned long long>(key) << 32) | j;
+            int rank = start;
+            for (int u = start; u < end; ++u) {
+              const unsigned ju = list16[u];
+              rank += ((static_cast<unsigned long long>(keys[ju]) << 32) | ju) < comp;
+            }
+            if (rank < K) {   // in the last bin: the `need` smallest, ties by smaller index
+              irow[1 + rank] = static_cast<int32_t>(j);
+              if (drow) drow[1 + rank] = __uint_as_float(key);
+            }
+          }
+          return;
+        }
+      }
       need -= s_below;
-      ties_total = hist[digit];
-      prefix |= static_cast<uint32_t>(digit) << shift;
-      mask |= 0xffu << shift;
-      __syncthreads();
+      ties_total = s_ties;
+      prefix |= static_cast<uint32_t>(s_digit) << lo;
+      hi = lo;
     }
-    const uint32_t tau = prefix;
+    __syncthreads();   // the histogram's storage becomes the list
+    const uint32_t tau = kmin + prefix;
     const int n_less = K - need;
 
-    // ---- compaction ----
+    // ---- compaction (one counter update per warp) ----
     const bool all_ties = (ties_total == need);
-    for (int j = tid; j < V; j += BT) {
-      const uint32_t key = keys[j];
-      if (key < tau || (all_ties && key == tau)) {
-        const int pos = atomicAdd(&s_cnt, 1);
-        list[pos] = (static_cast<unsigned long long>(key) << 32) | static_cast<unsigned>(j);
+    for (int base = 0; base < V; base += BT) {
+      const int j = base + tid;
+      const uint32_t key = j < V ? keys[j] : 0u;
+      const bool sel = j < V && j != i && (key < tau || (all_ties && key == tau));
+      const unsigned bal = __ballot_sync(kFull, sel);
+      if (bal) {
+        int pos = 0;
+        if (lane == 0) pos = atomicAdd(&s_cnt, __popc(bal));
+        pos = __shfl_sync(kFull, pos, 0) + __popc(bal & ((1u << lane) - 1u));
+        if (sel) list[pos] = (static_cast<unsigned long long>(key) << 32) | static_cast<unsigned>(j);
       }
     }
     if (!all_ties) {   // more ties than places: take them in index order
       int run = 0;
       for (int base = 0; base < V && run < need; base += BT) {
         const int j = base + tid;
-        const bool flag = j < V && keys[j] == tau;
+        const bool flag = j < V && j != i && keys[j] == tau;
         const unsigned bal = __ballot_sync(kFull, flag);
         if (lane == 0) wcnt[warp] = __popc(bal);
         __syncthreads();
@@ -230,21 +437,26 @@ __global__ void __launch_bounds__(BT) lantern_knn_row_kernel(BuildParams P, int 
     for (int t = K + tid; t < P2; t += BT) list[t] = ~0ull;
     __syncthreads();
 
-    // ---- bitonic sort of (key, index) composites ----
-    for (int size = 2; size <= P2; size <<= 1) {
-      for (int stride = size >> 1; stride > 0; stride >>= 1) {
+    // ---- bitonic sort of (key, index) composites: strides below 64 in registers by shuffles ----
+    const int nblk = P2 >> 6;
+    for (int blk = warp; blk < nblk; blk += BW) bitonic_block64(list, blk, lane, 2, 64);
+    __syncthreads();
+    for (int size = 128; size <= P2; size <<= 1) {
+      for (int stride = size >> 1; stride >= 64; stride >>= 1) {
         for (int t = tid; t < (P2 >> 1); t += BT) {
           const int lo = ((t & ~(stride - 1)) << 1) | (t & (stride - 1));
-          const int hi = lo | stride;
+          const int hi2 = lo | stride;
           const bool up = (lo & size) == 0;
-          const unsigned long long x = list[lo], y = list[hi];
+          const unsigned long long x = list[lo], y = list[hi2];
           if ((x > y) == up) {
             list[lo] = y;
-            list[hi] = x;
+            list[hi2] = x;
           }
         }
         __syncthreads();
       }
+      for (int blk = warp; blk < nblk; blk += BW) bitonic_block64(list, blk, lane, size, size);
+      __syncthreads();
     }
   }
 
@@ -270,7 +482,7 @@ static int next_pow2(int x) {
 
 static int rows_per_block(int V) {
   int r = V < 1024 ? V : 1024;
-  return (r + TILE - 1) / TILE * TILE;
+  return (r + TM - 1) / TM * TM;
 }
 
 }  // namespace lantern
@@ -294,8 +506,10 @@ extern "C" lantern_status lantern_build_neighbors(const float* codebook, int V, 
   if (need_ws && (!workspace || workspace_bytes < need_ws || (reinterpret_cast<uintptr_t>(workspace) & 15)))
     return LANTERN_E_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  const int P2 = k > 1 ? next_pow2(k - 1 < 2 ? 2 : k - 1) : 2;
-  const size_t smem = ((static_cast<size_t>(V) * 4 + 15) & ~size_t(15)) + static_cast<size_t>(P2) * 8;
+  const int P2 = next_pow2(k - 1 < 64 ? 64 : k - 1);   // the sort works on whole 64-element blocks
+  const size_t fast_bytes = HBINS * 2 + ((static_cast<size_t>(k - 1 + FAST_POP) * 2 + 15) & ~size_t(15));
+  const size_t list_bytes = static_cast<size_t>(P2) * 8 > fast_bytes ? static_cast<size_t>(P2) * 8 : fast_bytes;
+  const size_t smem = ((static_cast<size_t>(V) * 4 + 15) & ~size_t(15)) + list_bytes;
   if (smem > 220 * 1024) return LANTERN_E_SHAPE;
   if (cudaFuncSetAttribute(lantern_knn_row_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) !=
       cudaSuccess)
@@ -317,7 +531,7 @@ extern "C" lantern_status lantern_build_neighbors(const float* codebook, int V, 
   uint32_t* scratch = static_cast<uint32_t*>(workspace);
   for (int row0 = 0; row0 < V; row0 += rb) {
     const int rows = V - row0 < rb ? V - row0 : rb;
-    dim3 grid((V + TILE - 1) / TILE, (rows + TILE - 1) / TILE);
+    dim3 grid((V + TM - 1) / TM, (rows + TM - 1) / TM);
     lantern_distance_tile_kernel<<<grid, 256, 0, st>>>(codebook, scratch, V, D, row0, rows);
     if (cudaGetLastError() != cudaSuccess) return LANTERN_E_CUDA;
     P.scratch = scratch;

@@ -41,7 +41,27 @@ def test_ties_and_duplicates_exact():
     assert np.array_equal(gi, oi)
 
 
-@pytest.mark.parametrize("V,D,k", [(1100, 256, 64), (640, 40, 640), (2000, 100, 1000)])
+def test_outliers_and_overflowing_distances_exact():
+    # One code far away stretches the key range so that every other key falls into the select's first bin
+    # (the crowded-bin path with all of its passes); codes of magnitude 1e30 make distances overflow to inf
+    # (equal keys, ordered by index).
+    cb = li.codebook_gaussian(3000, 8, seed=77)
+    cb[1234] *= 1e15
+    for k in (5, 300, 3000):
+        gi, gd = _gpu(cb, k)
+        oi, od = oracle.build_neighbors(cb, k)
+        assert np.array_equal(gi, oi), k
+        assert np.array_equal(gd.view(np.uint32), od.view(np.uint32)), k
+    cb = li.codebook_gaussian(900, 4, seed=78)
+    cb[::7] *= 1e30
+    with np.errstate(over="ignore"):
+        gi, gd = _gpu(cb, 200)
+        oi, od = oracle.build_neighbors(cb, 200)
+    assert np.array_equal(gi, oi)
+    assert np.array_equal(gd.view(np.uint32), od.view(np.uint32))
+
+
+@pytest.mark.parametrize("V,D,k", [(1100, 256, 64), (640, 40, 640), (2000, 100, 1000), (1001, 37, 100), (130, 33, 130)])
 def test_large_d_exact(V, D, k):
     cb = li.codebook_clustered(V, D, centres=37, seed=8)
     gi, gd = _gpu(cb, k)

@@ -4,28 +4,27 @@
 // staging helpers it shares.
 //
 // Persistent CTAs of BNT threads, three to an SM; the context's raw target rows are staged in
-// shared memory by bulk copy and read twice:
-//   sweep 1  guidance combine (+ temperature, + top-k mask), maximum M;
-//   sweep 2  numerators exp(z - M); every thread keeps one partial sum per block-wide iteration j
-//            (iteration j covers the 4 * BNT consecutive tokens starting at 4 * BNT * j), so that
-//            token order is: iteration, then thread, then position in the thread's quad.
-// The iteration totals give Z and the iteration in which the cumulative weight first exceeds
-// u * Z; a block scan of that iteration's per-thread sums gives the thread, which re-reads its
-// four tokens.  All sums beyond four terms are in double precision.
+// shared memory by bulk copy.  A thread owns Q consecutive quads of four tokens (Q odd: the stride
+// between threads then spreads over all banks), so token order is thread order:
+//   sweep 1  guidance combine (+ temperature, + top-k mask), maximum M; the processed logits are
+//            written back over the raw logits they came from (16 bytes either way) where there
+//            are two rows or fp32 logits, so that sweep 2 does not form them again;
+//   sweep 2  numerators exp(z - M), one partial sum per quad, the thread's total.
+// One block scan of the totals gives Z and the thread in which the cumulative weight first
+// exceeds u * Z; that thread finds the quad among its partial sums and re-forms its four
+// numerators.  All sums beyond four terms are in double precision.
 #pragma once
 
 namespace lantern {
 
 constexpr int BNT = 320;
 constexpr int BNW = BNT / 32;
-constexpr int BN_ITERS = (16384 / 4 + BNT - 1) / BNT;   // 13: iterations of a 16384-token row
+constexpr int BN_ITERS = (16384 / 4 + BNT - 1) / BNT;   // 13: quads per thread of a 16384-token row
+static_assert(BN_ITERS % 2 == 1, "the largest quad count per thread is odd");
 
 struct BonusShared {
-  double wj[BNW][BN_ITERS];         // per-warp totals of every iteration
-  double wscan[BNW];
+  double wscan[BNW];                // per-warp running totals of the block scan
   float wm[BNW];
-  double Z, base;
-  int jstar;
   int tok;
   unsigned long long bar_full;
 };
@@ -61,6 +60,21 @@ __global__ void __launch_bounds__(BNT, 3) lantern_bonus_stream_kernel(VerifyPara
     return z;
   };
 
+  // quads per thread: the smallest odd number that covers the row
+  int Q = (quads + BNT - 1) / BNT;
+  Q |= 1;
+  constexpr bool IN_PLACE = UNC || !BF16;   // 16 bytes of raw logits per quad: room for its four processed logits
+  // the four processed logits of quad qd as sweep 1 left them
+  auto stored = [&](int qd, float tq) {
+    if (!IN_PLACE) return quad(qd, tq);
+    if (BF16) {
+      const float2 a = *reinterpret_cast<const float2*>(bsm + static_cast<size_t>(qd) * 8);
+      const float2 b = *reinterpret_cast<const float2*>(bsm + rowbytes + static_cast<size_t>(qd) * 8);
+      return make_float4(a.x, a.y, b.x, b.y);
+    }
+    return *reinterpret_cast<const float4*>(bsm + static_cast<size_t>(qd) * 16);
+  };
+
   if (tid == 0) {
     mbar_init(bar, 1);
     fence_mbar_init();
@@ -79,14 +93,29 @@ __global__ void __launch_bounds__(BNT, 3) lantern_bonus_stream_kernel(VerifyPara
     if (TOPK) tq = __ldg(P.thr_q + item);
     const double u = static_cast<double>(P.uniforms[static_cast<size_t>(b) * R + N]);
     const bool ok = mbar_wait(bar, it & 1, P.wait_tries);
+    const int q0 = tid * Q;                  // this thread's quads: q0 .. q0 + Q - 1, as far as the row goes
 
-    // ---- sweep 1: maximum ----
+    // ---- sweep 1: processed logits (kept in place), maximum ----
     float m = NEG_INF;
     int bad = 0;
-    for (int qd = tid; qd < quads; qd += BNT) {
-      const float4 z = quad(qd, tq);
-      bad |= (z.x != z.x) | (z.y != z.y) | (z.z != z.z) | (z.w != z.w);
-      m = fmaxf(fmaxf(m, fmaxf(z.x, z.y)), fmaxf(z.z, z.w));
+    if (ok) {
+#pragma unroll
+      for (int j = 0; j < BN_ITERS; ++j) {
+        const int qd = q0 + j;
+        if (j < Q && qd < quads) {
+          const float4 z = quad(qd, tq);
+          bad |= (z.x != z.x) | (z.y != z.y) | (z.z != z.z) | (z.w != z.w);
+          m = fmaxf(fmaxf(m, fmaxf(z.x, z.y)), fmaxf(z.z, z.w));
+          if (IN_PLACE) {
+            if (BF16) {
+              *reinterpret_cast<float2*>(bsm + static_cast<size_t>(qd) * 8) = make_float2(z.x, z.y);
+              *reinterpret_cast<float2*>(bsm + rowbytes + static_cast<size_t>(qd) * 8) = make_float2(z.z, z.w);
+            } else {
+              *reinterpret_cast<float4*>(bsm + static_cast<size_t>(qd) * 16) = z;
+            }
+          }
+        }
+      }
     }
     m = warp_max(m);
     if (lane == 0) S.wm[warp] = m;
@@ -117,7 +146,7 @@ __global__ void __launch_bounds__(BNT, 3) lantern_bonus_stream_kernel(VerifyPara
       __syncthreads();   // every thread has read S.wm and is done with the rows
     } else {
       // ---- sweep 2: numerators 2^((z - M) log2 e) through the ex2 unit (as in the fused pass), one partial
-      // sum per iteration ----
+      // sum per quad, the thread's total ----
       const float L_hi = 1.44269502162933349609375f;
       const uint64_t L2 = pack2(L_hi, L_hi), nM2 = pack2(-(M * L_hi), -(M * L_hi));
       auto numer4 = [&](const float4& z) {
@@ -127,78 +156,57 @@ __global__ void __launch_bounds__(BNT, 3) lantern_bonus_stream_kernel(VerifyPara
         return make_float4(greedy_ex2(a0), greedy_ex2(a1), greedy_ex2(a2_), greedy_ex2(a3));
       };
       float s[BN_ITERS];
+      double mine = 0.0;
 #pragma unroll
       for (int j = 0; j < BN_ITERS; ++j) {
-        const int qd = tid + j * BNT;
+        const int qd = q0 + j;
         s[j] = 0.0f;
-        if (qd < quads) {
-          const float4 z = quad(qd, tq);
-          const float4 e = numer4(z);
+        if (j < Q && qd < quads) {
+          const float4 e = numer4(stored(qd, tq));
           s[j] = (e.x + e.y) + (e.z + e.w);
         }
+        mine += static_cast<double>(s[j]);
       }
-#pragma unroll
-      for (int j = 0; j < BN_ITERS; ++j) {
-        const double v = warp_sum(static_cast<double>(s[j]));
-        if (lane == 0) S.wj[warp][j] = v;
-      }
-      __syncthreads();
-      if (warp == 0) {   // lane j owns iteration j: its total, the running total, the crossing
-        double t = 0.0;
-        if (lane < BN_ITERS) {
-#pragma unroll
-          for (int w = 0; w < BNW; ++w) t += S.wj[w][lane];
-        }
-        const double incl = warp_incl_scan(t, lane);
-        const double Z = __shfl_sync(kFull, incl, 31);
-        const double target = u * Z;
-        const unsigned over = __ballot_sync(kFull, lane < BN_ITERS && incl > target);
-        if (lane == 0) S.Z = Z;
-        if (over) {
-          const int js = __ffs(over) - 1;
-          const double before = __shfl_sync(kFull, incl - t, js);
-          if (lane == 0) {
-            S.jstar = js;
-            S.base = before;
-          }
-        } else if (lane == 0) {
-          S.jstar = -1;
-        }
-      }
+      const double incl = warp_incl_scan(mine, lane);
+      if (lane == 31) S.wscan[warp] = incl;
       if (tid == 0) S.tok = -1;
       __syncthreads();
-      const double Z = S.Z;
-      const int jstar = S.jstar;
+      double excl = incl - mine, Z = 0.0;
+#pragma unroll
+      for (int w = 0; w < BNW; ++w) {
+        const double t = S.wscan[w];
+        if (w < warp) excl += t;
+        Z += t;
+      }
       if (!(Z > 0.0 && Z < 1e300)) {
         st = LANTERN_ST_NONFINITE;
-      } else if (jstar >= 0) {
+      } else {
         const double target = u * Z;
-        float mine = 0.0f;
-#pragma unroll
-        for (int j = 0; j < BN_ITERS; ++j) mine = j == jstar ? s[j] : mine;
-        const double md = static_cast<double>(mine);
-        const double incl = warp_incl_scan(md, lane);
-        if (lane == 31) S.wscan[warp] = incl;
-        __syncthreads();
-        double excl = S.base + incl - md;
-#pragma unroll
-        for (int w = 0; w < BNW; ++w)
-          if (w < warp) excl += S.wscan[w];
-        if (excl + md > target && !(excl > target)) {   // the first thread whose inclusive sum exceeds the target
-          const int qd = tid + jstar * BNT;
-          const float4 z = quad(qd, tq);
-          const float4 e4 = numer4(z);
-          const float e[4] = {e4.x, e4.y, e4.z, e4.w};
+        if (excl + mine > target && !(excl > target)) {   // the first thread whose inclusive sum exceeds the target
           double cum = excl;
-          int pick = -1, lastpos = -1;
+          int jq = -1, jlast = -1;
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            cum += static_cast<double>(e[c]);
-            if (e[c] > 0.0f) lastpos = c;
-            if (pick < 0 && cum > target) pick = c;
+          for (int j = 0; j < BN_ITERS; ++j) {
+            if (s[j] > 0.0f) jlast = j;
+            if (jq < 0 && cum + static_cast<double>(s[j]) > target) jq = j;
+            if (jq < 0) cum += static_cast<double>(s[j]);
           }
-          if (pick < 0) pick = lastpos;   // the quad's own rounding: its largest token of positive weight
-          S.tok = 4 * qd + pick;
+          const bool rounded = jq < 0;   // the thread's own rounding: its largest token of positive weight
+          if (rounded) jq = jlast;
+          if (jq >= 0) {
+            const int qd = q0 + jq;
+            const float4 e4 = numer4(stored(qd, tq));
+            const float e[4] = {e4.x, e4.y, e4.z, e4.w};
+            int pick = -1, lastpos = -1;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              cum += static_cast<double>(e[c]);
+              if (e[c] > 0.0f) lastpos = c;
+              if (pick < 0 && cum > target) pick = c;
+            }
+            if (rounded || pick < 0) pick = lastpos;   // (the quad's own rounding likewise)
+            if (pick >= 0) S.tok = 4 * qd + pick;
+          }
         }
         __syncthreads();
         tok = S.tok;
@@ -206,12 +214,16 @@ __global__ void __launch_bounds__(BNT, 3) lantern_bonus_stream_kernel(VerifyPara
       if (st == 0 && tok < 0) {
         // rounding left no token above the target: the largest token of positive weight
         int last = -1;
-        for (int qd = tid; qd < quads; qd += BNT) {
-          const float4 z = quad(qd, tq);
-          if (z.x > NEG_INF) last = 4 * qd;
-          if (z.y > NEG_INF) last = 4 * qd + 1;
-          if (z.z > NEG_INF) last = 4 * qd + 2;
-          if (z.w > NEG_INF) last = 4 * qd + 3;
+#pragma unroll
+        for (int j = 0; j < BN_ITERS; ++j) {
+          const int qd = q0 + j;
+          if (j < Q && qd < quads) {
+            const float4 z = stored(qd, tq);
+            if (z.x > NEG_INF) last = 4 * qd;
+            if (z.y > NEG_INF) last = 4 * qd + 1;
+            if (z.z > NEG_INF) last = 4 * qd + 2;
+            if (z.w > NEG_INF) last = 4 * qd + 3;
+          }
         }
         if (last >= 0) atomicMax(&S.tok, last);
         __syncthreads();

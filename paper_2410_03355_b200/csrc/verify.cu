@@ -39,7 +39,7 @@ namespace lantern {
 // the fused pass overwrites; contexts without children are marked as leaves.
 // ---------------------------------------------------------------------------------------
 constexpr int PLAN_WARPS = 4;
-constexpr int kPlanArrays = 12;  // per-warp arrays of N + 2 ints in shared memory
+constexpr int kPlanArrays = 13;  // per-warp arrays of N + 2 ints in shared memory
 
 __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyParams P) {
   extern __shared__ int plan_smem[];
@@ -50,16 +50,17 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
   int* cnt = plan_smem + warp * kPlanArrays * (R + 1);   // cnt[c]: number of children of context c
   int* cur = cnt + (R + 1);                    // fill cursor, ends as the end offset of context c
   int* dep = cur + (R + 1);                    // depth of context c (root = 0), later its breadth-first rank
-  int* dst = dep + (R + 1);                    // per depth: next breadth-first rank
-  int* siz = dst + (R + 1);                    // number of contexts in the subtree of context c, itself included
+  int* lvl = dep + (R + 1);                    // per depth: where its nodes lie in the (depth, index) order
+  int* siz = lvl + (R + 1);                    // number of contexts in the subtree of context c, itself included
   int* din = siz + (R + 1);                    // depth-first (pre-order) position of context c
-  int* nxt = din + (R + 1);                    // depth-first position the next child of context c gets
-  int* s_par = nxt + (R + 1);                  // the sequence's parents, tokens and uniforms, staged once by all
+  int* tmp = din + (R + 1);                    // per context: children placed so far; later running sums of sizes
+  int* anc = tmp + (R + 1);                    // pointer jumping: an ancestor of node i; later the (depth, index) order
+  int* s_par = anc + (R + 1);                  // the sequence's parents, tokens and uniforms, staged once by all
   int* s_tok = s_par + (R + 1);                //   lanes: the serial parts below then run out of shared memory
   int* s_uni = s_tok + (R + 1);
   int* s_pos = s_uni + (R + 1);                // place of node i in the child lists
   int* s_first = s_pos + (R + 1);              // first child (smallest node index) of context c
-  for (int i = lane; i <= R; i += 32) cnt[i] = 0, dst[i] = 0, siz[i] = 1, s_first[i] = -1;
+  for (int i = lane; i <= R; i += 32) cnt[i] = 0, siz[i] = 1, s_first[i] = -1;
   __syncwarp();
   int status = 0;
   const float qnan = __int_as_float(0x7fc00000);
@@ -96,43 +97,159 @@ __global__ void __launch_bounds__(PLAN_WARPS * 32) lantern_plan_kernel(VerifyPar
   }
 
   ChildInfo* kids = P.children + static_cast<size_t>(b) * N;
+  // Children of each context in node order (cur, s_pos, s_first), subtree sizes and pre-order positions
+  // (siz, din: the contexts behind a node then occupy one contiguous range of positions, which is what lets
+  // the fused pass strike a whole rejected subtree with a few byte stores), and the breadth-first rank of every
+  // context with children (dep).  All of it by the whole warp, 32 nodes at a time.
   int n_ctx = 0;
-  if (lane == 0) {      // children of each context in node order; depths; breadth-first ranks
-    int run = 0;
-    for (int c = 0; c < R; ++c) {
-      cur[c] = run;
-      run += cnt[c];
+  const unsigned below = (1u << lane) - 1u;
+  if (!P.parents) {
+    // a chain: context c has the one child c, lies c deep, and has the R - c contexts from itself on behind it
+    for (int c = lane; c < R; c += 32) {
+      cur[c] = c < N ? c + 1 : N;
+      siz[c] = R - c;
+      din[c] = c;
+      dep[c] = c;
+      if (c < N) s_pos[c] = c, s_first[c] = c;
     }
-    // Subtree sizes (children have larger indices than their parents) and pre-order positions: the
-    // contexts behind a node then occupy one contiguous range of positions, which is what lets the
-    // fused pass strike a whole rejected subtree with a few byte stores.
-    for (int i = N - 1; i >= 0; --i) siz[s_par[i] + 1] += siz[i + 1];
-    dep[0] = 0;
-    din[0] = 0;
-    nxt[0] = 1;
-    for (int i = 0; i < N; ++i) {
-      const int par = s_par[i];
-      din[i + 1] = nxt[par + 1];
-      nxt[par + 1] += siz[i + 1];
-      nxt[i + 1] = din[i + 1] + 1;
-      s_pos[i] = cur[par + 1]++;
-      if (s_first[par + 1] < 0) s_first[par + 1] = i;
-      dep[i + 1] = dep[par + 1] + 1;
+    n_ctx = N;
+  } else {
+    // -- child-list offsets: cur[c] = end of the children of context c
+    int carry = 0;
+    for (int base = 0; base < R; base += 32) {
+      const int c = base + lane;
+      int incl = c < R ? cnt[c] : 0;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(kFull, incl, o);
+        if (lane >= o) incl += t;
+      }
+      if (c < R) cur[c] = carry + incl, tmp[c] = 0;
+      carry += __shfl_sync(kFull, incl, 31);
     }
-    for (int c = 0; c < R; ++c)
-      if (cnt[c] > 0) ++dst[dep[c]];          // contexts with children per depth
-    for (int d = 0; d < R; ++d) {             // exclusive prefix: first rank of each depth
-      const int n = dst[d];
-      dst[d] = n_ctx;
-      n_ctx += n;
+    __syncwarp();
+    // -- place of every node among its siblings (tmp[c]: children of c placed so far), first child
+    for (int base = 0; base < N; base += 32) {
+      const int i = base + lane;
+      const unsigned act = __ballot_sync(kFull, i < N);
+      if (i < N) {
+        const int pc = s_par[i] + 1;
+        const unsigned peers = __match_any_sync(act, pc);
+        const int before = tmp[pc];
+        const int rk = before + __popc(peers & below);
+        s_pos[i] = cur[pc] - cnt[pc] + rk;
+        if (rk == 0) s_first[pc] = i;
+        __syncwarp(act);
+        if ((peers & below) == 0) tmp[pc] = before + __popc(peers);
+      }
+      __syncwarp();
     }
-    for (int c = 0; c < R; ++c)
-      if (cnt[c] > 0) dep[c] = dst[dep[c]]++; // dep[c] becomes the context's rank
-    // (thousands of warps would otherwise queue up on one address: most find the maximum already there)
-    if (n_ctx > *reinterpret_cast<volatile int*>(&P.counters->n_rank)) atomicMax(&P.counters->n_rank, n_ctx);
+    // -- depth of every context by pointer jumping: dep[i + 1] = distance from node i to anc[i] (or to the root)
+    for (int i = lane; i < N; i += 32) anc[i] = s_par[i], dep[i + 1] = 1;
+    if (lane == 0) dep[0] = 0;
+    __syncwarp();
+    for (int round = 0; round < 12; ++round) {   // every round at least doubles the distance covered: 2^11 > 1024
+      bool more = false;
+      for (int base = 0; base < N; base += 32) {
+        const int i = base + lane;
+        const int a = i < N ? anc[i] : -1;
+        int da = 0, aa = -1;
+        if (a >= 0) da = dep[a + 1], aa = anc[a];   // a < i: a pair that is consistent whether or not a has moved this round
+        __syncwarp();
+        if (a >= 0) {
+          dep[i + 1] += da;
+          anc[i] = aa;
+          more |= aa >= 0;
+        }
+        __syncwarp();
+      }
+      if (!__any_sync(kFull, more)) break;
+    }
+    int maxd = 0;
+    for (int i = lane; i < N; i += 32) maxd = max(maxd, dep[i + 1]);
+    maxd = __reduce_max_sync(kFull, maxd);
+    // -- nodes ordered by (depth, index): lvl[d] counts, then is the cursor, and ends as the end of level d
+    for (int d = lane; d <= maxd; d += 32) lvl[d] = 0;
+    __syncwarp();
+    for (int i = lane; i < N; i += 32) atomicAdd(&lvl[dep[i + 1]], 1);
+    __syncwarp();
+    carry = 0;
+    for (int base = 0; base <= maxd; base += 32) {
+      const int d = base + lane;
+      const int n = d <= maxd ? lvl[d] : 0;
+      int incl = n;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(kFull, incl, o);
+        if (lane >= o) incl += t;
+      }
+      if (d <= maxd) lvl[d] = carry + incl - n;
+      carry += __shfl_sync(kFull, incl, 31);
+    }
+    __syncwarp();
+    int* order = anc;   // (the ancestors are no longer needed)
+    for (int base = 0; base < N; base += 32) {
+      const int i = base + lane;
+      const unsigned act = __ballot_sync(kFull, i < N);
+      if (i < N) {
+        const int d = dep[i + 1];
+        const unsigned peers = __match_any_sync(act, d);
+        const int before = lvl[d];
+        order[before + __popc(peers & below)] = i;
+        __syncwarp(act);
+        if ((peers & below) == 0) lvl[d] = before + __popc(peers);
+      }
+      __syncwarp();
+    }
+    // -- subtree sizes, deepest level first (level d occupies order[lvl[d - 1] .. lvl[d]))
+    for (int d = maxd; d >= 1; --d) {
+      for (int pos = lvl[d - 1] + lane; pos < lvl[d]; pos += 32) {
+        const int i = order[pos];
+        atomicAdd(&siz[s_par[i] + 1], siz[i + 1]);
+      }
+      __syncwarp();
+    }
+    // -- sizes in child-list order and their running sum: tmp[pos] = sizes of everything placed before pos
+    for (int i = lane; i < N; i += 32) tmp[s_pos[i]] = siz[i + 1];
+    __syncwarp();
+    carry = 0;
+    for (int base = 0; base < N; base += 32) {
+      const int pos = base + lane;
+      const int n = pos < N ? tmp[pos] : 0;
+      int incl = n;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(kFull, incl, o);
+        if (lane >= o) incl += t;
+      }
+      if (pos < N) tmp[pos] = carry + incl - n;
+      carry += __shfl_sync(kFull, incl, 31);
+    }
+    if (lane == 0) din[0] = 0;
+    __syncwarp();
+    // -- pre-order positions, top level first: after the parent come the subtrees of the earlier siblings
+    for (int d = 1; d <= maxd; ++d) {
+      for (int pos = lvl[d - 1] + lane; pos < lvl[d]; pos += 32) {
+        const int i = order[pos];
+        const int pc = s_par[i] + 1;
+        din[i + 1] = din[pc] + 1 + tmp[s_pos[i]] - tmp[cur[pc] - cnt[pc]];
+      }
+      __syncwarp();
+    }
+    // -- breadth-first rank of the contexts with children: the root, then the nodes by (depth, index)
+    n_ctx = cnt[0] > 0 ? 1 : 0;
+    for (int base = 0; base < N; base += 32) {
+      const int pos = base + lane;
+      const int i = pos < N ? order[pos] : 0;
+      const bool has = pos < N && cnt[i + 1] > 0;
+      const unsigned bal = __ballot_sync(kFull, has);
+      if (has) dep[i + 1] = n_ctx + __popc(bal & below);   // the depth is no longer needed: dep[c] becomes the rank
+      n_ctx += __popc(bal);
+    }
   }
-  n_ctx = __shfl_sync(kFull, n_ctx, 0);
-  __syncwarp();         // lane 0's writes to the shared arrays are visible to the warp
+  // (thousands of warps would otherwise queue up on one address: most find the maximum already there)
+  if (lane == 0 && n_ctx > *reinterpret_cast<volatile int*>(&P.counters->n_rank)) atomicMax(&P.counters->n_rank, n_ctx);
+  __syncwarp();         // the shared arrays are complete
   for (int i = lane; i < N; i += 32) {   // the child lists, written by all lanes
     ChildInfo ci = {i, s_tok[i], __int_as_float(s_uni[i]), (din[i + 1] << 16) | siz[i + 1]};
     kids[s_pos[i]] = ci;

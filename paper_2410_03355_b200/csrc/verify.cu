@@ -666,7 +666,8 @@ static lantern_status verify_impl(const void* target_logits, const void* draft_l
   P.top_k = topk ? top_k : 0;
   P.thr_q = topk ? reinterpret_cast<float*>(ws + L.thrq) : nullptr;
   P.thr_p = topk ? reinterpret_cast<float*>(ws + L.thrp) : nullptr;
-  P.ctx_slots = greedy ? reinterpret_cast<int32_t*>(ws + L.slots) : nullptr;   // only the greedy kernels walk the compact list
+  // only the threshold kernel of greedy decoding with the logit filter walks the compact list
+  P.ctx_slots = (greedy && topk) ? reinterpret_cast<int32_t*>(ws + L.slots) : nullptr;
   P.dead = ws + L.dead;
   P.wait_tries = g_wait_tries;
   P.withhold_item = g_withhold_item;

@@ -114,6 +114,31 @@ def test_long_chain_and_wide_tree():
     check(inp, host, dev, 0.5, min_tested=2)          # the longest supported chain
 
 
+def test_deep_explicit_trees():
+    """Trees whose depth is of the order of their size: the longest chain written as a tree (every level holds
+    one node), and a spine with a leaf hanging off every spine node (the plan's depths, level order, subtree sizes
+    and pre-order positions over hundreds of levels)."""
+    V, k = 256, 16
+    cb = li.codebook_gaussian(V, 8, seed=39)
+    host = oracle.build_neighbors(cb, k)[0]
+    dev = torch.from_numpy(host).cuda()
+    inp = li.verify_inputs(2, 1024, V, dtype=li.BF16, has_uncond=False, cfg_scale=1.0, sigma_draft=0.05, seed=63)
+    a = run_gpu(inp, dev, 0.5)
+    b = run_gpu(dataclasses.replace(inp, tree_parents=li.chain_parents(2, 1024)), dev, 0.5)
+    for f in ("accept_len", "next_token", "accept_path", "status"):
+        assert torch.equal(getattr(a, f), getattr(b, f)), f
+    assert int(a.accept_len.min()) > 20
+    # spine nodes 0, 2, 4, ... (each the child of the spine node before), node 2j + 1 a second child of spine node 2j - 2
+    N = 600
+    par = np.empty((3, N), np.int32)
+    for i in range(N):
+        par[:, i] = i - 2 if i >= 2 else -1
+    inp = li.verify_inputs(3, N, V, dtype=li.BF16, has_uncond=True, cfg_scale=1.5, sigma_target=1.0, sigma_draft=0.15,
+                           rho=0.95, parents=par, seed=64)
+    res = check(inp, host, dev, 0.3, min_tested=3)
+    assert res["accept_mean"] > 3
+
+
 def test_chain_equals_explicit_tree():
     V, k = 1024, 32
     cb = li.codebook_gaussian(V, 8, seed=33)

@@ -236,31 +236,63 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
   const int quads = V >> 2;
   const int G = gridDim.x;
   int n_eval = 0, n_skip = 0, n_test = 0;       // thread 0: work accounting
-  // Thread 0 keeps the staging areas filled.  The CTA walks the slots blockIdx.x, blockIdx.x + G, ... and, as in
+  // Warp 0 keeps the staging areas filled.  The CTA walks the slots blockIdx.x, blockIdx.x + G, ... and, as in
   // the sampling pass, leaves out the empty ones and the contexts known to be unreachable (Algorithm 1 stops at
-  // the first rejection); a context whose parent is still undecided is evaluated anyway.
-  auto refill = [&](int area) {
+  // the first rejection); a context whose parent is still undecided is evaluated anyway.  The warp looks at 32
+  // slots in one round trip (work item and dead mark of each) and keeps the live ones as candidates, one per
+  // lane; when an area falls free, the first candidate's dead mark is read once more -- as late as possible --
+  // and the candidate is taken or dropped.
+  int q_w = -1, q_mark = 0;      // this lane's candidate: its slot and its dead mark's index
+  bool q_live = false;
+  auto refill = [&](int area) {  // called by all lanes of warp 0
     for (;;) {
-      const int w = S.cursor;
-      if (w >= total) {
-        S.item[area].item = -1;
+      unsigned m = __ballot_sync(kFull, q_live);
+      while (m) {
+        const int l = __ffs(m) - 1;
+        m &= m - 1u;
+        const int w = __shfl_sync(kFull, q_w, l), mk = __shfl_sync(kFull, q_mark, l);
+        if (lane == l) q_live = false;
+        int4 lo = make_int4(0, 0, 0, 0), hi = make_int4(0, 0, 0, 0);
+        int dead = 0;
+        if (lane == 0) {           // both round trips at once: the mark, and the item in case it is taken
+          dead = *reinterpret_cast<const volatile unsigned char*>(P.dead + mk);
+          lo = __ldg(reinterpret_cast<const int4*>(P.work + w));
+          hi = __ldg(reinterpret_cast<const int4*>(P.work + w) + 1);
+        }
+        dead = __shfl_sync(kFull, dead, 0);
+        if (dead) {
+          if (lane == 0) ++n_skip;
+          continue;
+        }
+        if (lane == 0) {
+          WorkItem wi;
+          wi.item = lo.x, wi.cbase = lo.y, wi.nchild_node0 = lo.z, wi.span0 = lo.w;
+          wi.tok0 = hi.x, wi.r0 = __int_as_float(hi.y), wi.u_final = __int_as_float(hi.z), wi.mark = hi.w;
+          S.item[area] = wi;
+          greedy_issue_rows<BF16, UNC>(P, wi.item, gsm + static_cast<size_t>(area) * area_bytes, rowbytes, &S.bar_full[area]);
+          ++n_eval;
+        }
         return;
       }
-      S.cursor = w + G;
-      const int4 lo = __ldg(reinterpret_cast<const int4*>(P.work + w));
-      if (lo.x < 0) continue;
-      const int4 hi = __ldg(reinterpret_cast<const int4*>(P.work + w) + 1);
-      if (*reinterpret_cast<const volatile unsigned char*>(P.dead + hi.w) != 0) {
-        ++n_skip;
-        continue;
+      // no candidate left: the next 32 slots of this CTA
+      const int base = S.cursor;
+      if (base >= total) {
+        if (lane == 0) S.item[area].item = -1;
+        return;
       }
-      WorkItem wi;
-      wi.item = lo.x, wi.cbase = lo.y, wi.nchild_node0 = lo.z, wi.span0 = lo.w;
-      wi.tok0 = hi.x, wi.r0 = __int_as_float(hi.y), wi.u_final = __int_as_float(hi.z), wi.mark = hi.w;
-      S.item[area] = wi;
-      greedy_issue_rows<BF16, UNC>(P, wi.item, gsm + static_cast<size_t>(area) * area_bytes, rowbytes, &S.bar_full[area]);
-      ++n_eval;
-      return;
+      __syncwarp();
+      if (lane == 0) S.cursor = base + 32 * G;
+      const long long wl = static_cast<long long>(base) + static_cast<long long>(lane) * G;
+      const bool valid = wl < total;
+      q_w = valid ? static_cast<int>(wl) : -1;
+      const int item = valid ? __ldg(&P.work[q_w].item) : -1;
+      const bool has = item >= 0;
+      q_mark = has ? __ldg(&P.work[q_w].mark) : 0;
+      const bool dead = has && *reinterpret_cast<const volatile unsigned char*>(P.dead + q_mark) != 0;
+      const unsigned gone = __ballot_sync(kFull, dead);
+      if (lane == 0) n_skip += __popc(gone);
+      q_live = has && !dead;
+      __syncwarp();
     }
   };
 
@@ -270,8 +302,10 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
     S.status = 0;
     S.flags[0] = S.flags[1] = 0;
     S.cursor = blockIdx.x;
-    for (int r = 0; r < ring; ++r) refill(r);
   }
+  __syncthreads();
+  if (warp == 0)
+    for (int r = 0; r < ring; ++r) refill(r);
   __syncthreads();
 
   uint32_t phase = 0;
@@ -526,8 +560,8 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
       Record rec = {accepted, finite ? arg : -1, status | S.status, 0};
       P.records[cur.item] = rec;
       S.status = 0;
-      refill(buf);
     }
+    if (warp == 0) refill(buf);
     __syncthreads();   // the area's next context (or the end of the list) is visible to everybody
     if (++buf == ring) {
       buf = 0;

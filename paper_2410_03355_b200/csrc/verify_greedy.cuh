@@ -132,6 +132,7 @@ constexpr int GCW = GCT / 32;
 constexpr int GGT = 256;            // threads that gather: four neighbour slots each per round
 constexpr int GGW = GGT / 32;
 constexpr int GRING_MAX = 4;
+constexpr int GLOOK = 32;           // slots warp 0 looks at per round trip when it has no candidate left (8 and 16 measured slower)
 static_assert(GCW <= 32 && GGT < GCT, "one warp combines the per-warp partials; a thread beyond the gatherers solves the JSD bound");
 
 struct GreedyCtxShared {
@@ -281,9 +282,9 @@ __global__ void __launch_bounds__(GCT, 3) lantern_greedy_context_kernel(VerifyPa
         return;
       }
       __syncwarp();
-      if (lane == 0) S.cursor = base + 32 * G;
+      if (lane == 0) S.cursor = base + GLOOK * G;
       const long long wl = static_cast<long long>(base) + static_cast<long long>(lane) * G;
-      const bool valid = wl < total;
+      const bool valid = lane < GLOOK && wl < total;
       q_w = valid ? static_cast<int>(wl) : -1;
       const int item = valid ? __ldg(&P.work[q_w].item) : -1;
       const bool has = item >= 0;

@@ -104,7 +104,7 @@ def method_work(parents, accept_len, accept_path, N: int):
 # 1024-sequence call of the chain workload, as a ratio to the bytes of the 5348 contexts and nodes that call evaluated;
 # traffic grows in proportion to the contexts evaluated, so a full launch is scaled by its evaluated bytes.
 # Tied to the kernel revision the capture was taken on: any other revision reports null.
-NCU_TRAFFIC = {"kernel_revision": 17, "workload": "batch_chain", "traffic_over_algorithmic": 562767360 / 547121792}
+NCU_TRAFFIC = {"kernel_revision": 18, "workload": "batch_chain", "traffic_over_algorithmic": 564017408 / 548656352}
 
 
 def ncu_traffic(workload, alg_bytes):

@@ -33,7 +33,7 @@
 // evaluated anyway: with few sequences per call that keeps every SM busy (all contexts of a tree run
 // side by side), with many sequences it is rare, and the walk kernel reads only records on the
 // accepted path either way, so the result never depends on what was speculated.
-#define LANTERN_CONTEXT_KERNEL_REVISION 17   // bump on every change to this file
+#define LANTERN_CONTEXT_KERNEL_REVISION 18   // bump on every change to this file
 
 namespace lantern {
 
@@ -933,6 +933,14 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
           break;
         }
         // ---- rejected: residual [q_{k,delta}(.|D = x~) - p]_+ ----
+        // the drafter logits of the first pass: asked for at once, in flight while A is flagged and across the barrier
+        const unsigned char* drow = static_cast<const unsigned char*>(P.draft) + static_cast<size_t>(item) * rowbytes;
+        DraftRaw dnext[CP];
+#pragma unroll
+        for (int c = 0; c < CP; ++c) {
+          const int g = c * GT + gt;
+          dnext[c] = draft_fetch(drow, g * 8 < V ? g : gt);
+        }
         // members of A (x~ included) leave no residual mass: flag them with a negative sign
         for (int base = 0; base < m; base += 4 * GT) {
 #pragma unroll
@@ -969,14 +977,6 @@ __global__ void __launch_bounds__(CTX_THREADS, 1) lantern_context_kernel(VerifyP
             raw_c = ctx_raw_logit<BF16>(P.target, e);
             if (UNC) raw_u = ctx_raw_logit<BF16>(P.target, static_cast<size_t>(P.B) * R * V + e);
           }
-        }
-        // the drafter logits of the first pass, in flight across the barrier
-        const unsigned char* drow = static_cast<const unsigned char*>(P.draft) + static_cast<size_t>(item) * rowbytes;
-        DraftRaw dnext[CP];
-#pragma unroll
-        for (int c = 0; c < CP; ++c) {
-          const int g = c * GT + gt;
-          dnext[c] = draft_fetch(drow, g * 8 < V ? g : gt);
         }
         gbar(grp);   // [flags]
         // w = E - (p'/q' scale ratio) * ep in common units, i.e. E - ratio * ep in the slice's own units

@@ -7,9 +7,14 @@
 // Small D (<= 32): one CTA per code computes its V keys straight into shared memory.
 // Large D: a tiled SIMT kernel writes the keys of a block of rows to global scratch (each
 // (i, j) accumulator still runs over d in order), and the per-row CTA reads its row of keys.
-// Per row: exclude the code itself, radix-select the (k-1)-th smallest key (ties by smaller
-// index), compact the selected (key, index) pairs, bitonic-sort them as 64-bit composites,
-// and store the row with the code itself in slot 0.
+// Per row (the code itself excluded; it goes to slot 0): the keys' range, one 2048-bin histogram of
+// the top 11 bits of key - min, the bin that holds the (k-1)-th smallest key and every bin's offset
+// by one block scan, then a counting sort -- the index of every key up to that bin is scattered to
+// its bin's place, ranked inside its bin by (key, index), and stored at its final position, so that
+// ties at the threshold are taken by smaller index.  A row in which one of those bins holds more
+// than 256 keys (massive ties, an outlier that stretches the range) takes the general path:
+// further histogram passes down to the exact threshold key, compaction of the selected
+// (key, index) pairs, bitonic sort of the 64-bit composites.
 #include <cuda_runtime.h>
 #include <stdint.h>
 
